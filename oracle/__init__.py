@@ -1,0 +1,158 @@
+"""Python face of the CPU oracle (test infrastructure, not product code).
+
+Builds ``castling_oracle.c`` with gcc into a shared object beside it and calls
+it through ctypes on float64 numpy arrays.  Nothing here touches CUDA or the
+``paper_2211_10526_b200`` package, and that package never imports this one.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may use
+this module.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "castling_oracle.c")
+_LIB = os.path.join(_HERE, "libcastling_oracle.so")
+_lib = None
+
+DEFAULT_EPS = 1e-12
+
+_dp = ctypes.POINTER(ctypes.c_double)
+
+
+def build(force: bool = False, src: str = _SRC, lib: str = _LIB) -> str:
+    """Compile the C oracle (-O2, no fast-math) if it is missing or stale."""
+    if force or not os.path.exists(lib) or os.path.getmtime(lib) < os.path.getmtime(src):
+        tmp = f"{lib}.{os.getpid()}.tmp"
+        subprocess.run(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-o", tmp, src, "-lm"], check=True)
+        os.replace(tmp, lib)
+    return lib
+
+
+def _declare(lib: ctypes.CDLL) -> ctypes.CDLL:
+    i, dbl = ctypes.c_int, ctypes.c_double
+    lib.castling_oracle_forward.restype = i
+    lib.castling_oracle_forward.argtypes = [_dp] * 6 + [i] * 6 + [dbl, i, i]
+    lib.castling_oracle_forward_bruteforce.restype = i
+    lib.castling_oracle_forward_bruteforce.argtypes = [_dp] * 6 + [i] * 6 + [dbl]
+    lib.castling_oracle_similarity.restype = i
+    lib.castling_oracle_similarity.argtypes = [_dp] * 3 + [i, i, dbl]
+    lib.castling_oracle_angular_exact.restype = dbl
+    lib.castling_oracle_angular_exact.argtypes = [dbl]
+    lib.castling_oracle_angular_series.restype = dbl
+    lib.castling_oracle_angular_series.argtypes = [dbl, i]
+    lib.castling_oracle_angular_series_coeff.restype = dbl
+    lib.castling_oracle_angular_series_coeff.argtypes = [i]
+    return lib
+
+
+def load(path: Optional[str] = None) -> ctypes.CDLL:
+    """Load (building first if needed) the oracle library; ``path`` loads another build of it."""
+    global _lib
+    if path is not None:
+        return _declare(ctypes.CDLL(path))
+    if _lib is None:
+        _lib = _declare(ctypes.CDLL(build()))
+    return _lib
+
+
+def _f64(a) -> np.ndarray:
+    """float64, C-contiguous numpy view/copy of a numpy array or a CPU torch tensor."""
+    if hasattr(a, "detach"):  # torch tensor, any float dtype
+        a = a.detach().cpu().double().numpy()
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(_dp)
+
+
+def _check_shapes(q, k, v, w, bias, gridH, gridW, ksize):
+    if q.ndim != 4 or q.shape != k.shape or q.shape != v.shape:
+        raise ValueError("q, k, v must share one [B, H, N, d] shape")
+    B, H, N, d = q.shape
+    if N != gridH * gridW:
+        raise ValueError("N != gridH * gridW")
+    if w.shape != (H * d, ksize, ksize):
+        raise ValueError("dw_weight must be [H*d, ksize, ksize]")
+    if bias is not None and bias.shape != (H * d,):
+        raise ValueError("dw_bias must be [H*d]")
+    return B, H, N, d
+
+
+def forward(q, k, v, dw_weight, dw_bias, gridH: int, gridW: int, ksize: int,
+            eps: float = DEFAULT_EPS, threads: int = 1, lib: Optional[ctypes.CDLL] = None) -> np.ndarray:
+    """Linear-angular attention core, re-associated form, float64.  Returns [B,H,N,d].
+
+    ``threads`` > 1 splits the independent (b,h) heads over host threads; each
+    thread runs the same single-threaded C routine on its own slice.
+    """
+    lib = lib or load()
+    q, k, v, w = _f64(q), _f64(k), _f64(v), _f64(dw_weight)
+    bias = None if dw_bias is None else _f64(dw_bias)
+    B, H, N, d = _check_shapes(q, k, v, w, bias, gridH, gridW, ksize)
+    out = np.empty_like(q)
+    BH = B * H
+    threads = max(1, min(int(threads), BH))
+
+    def run(lo: int, hi: int) -> int:
+        return lib.castling_oracle_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(bias), _ptr(out),
+                                           B, H, gridH, gridW, d, ksize, float(eps), lo, hi)
+
+    if threads == 1:
+        rcs = [run(0, BH)]
+    else:
+        cuts = [BH * t // threads for t in range(threads + 1)]
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            rcs = list(pool.map(lambda ab: run(*ab), zip(cuts[:-1], cuts[1:])))
+    if any(rcs):
+        raise RuntimeError("castling_oracle_forward failed")
+    return out
+
+
+def forward_bruteforce(q, k, v, dw_weight, dw_bias, gridH: int, gridW: int, ksize: int,
+                       eps: float = DEFAULT_EPS, lib: Optional[ctypes.CDLL] = None) -> np.ndarray:
+    """Same result from the explicit N x N similarity matrix (Eq. 8 then Eq. 9); small N only."""
+    lib = lib or load()
+    q, k, v, w = _f64(q), _f64(k), _f64(v), _f64(dw_weight)
+    bias = None if dw_bias is None else _f64(dw_bias)
+    B, H, N, d = _check_shapes(q, k, v, w, bias, gridH, gridW, ksize)
+    out = np.empty_like(q)
+    rc = lib.castling_oracle_forward_bruteforce(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(bias), _ptr(out),
+                                                B, H, gridH, gridW, d, ksize, float(eps))
+    if rc:
+        raise RuntimeError("castling_oracle_forward_bruteforce failed")
+    return out
+
+
+def similarity(q, k, eps: float = DEFAULT_EPS, lib: Optional[ctypes.CDLL] = None) -> np.ndarray:
+    """Explicit similarity matrix 1/2 + q^.k^/pi of one head; q, k are [N, d]."""
+    lib = lib or load()
+    q, k = _f64(q), _f64(k)
+    N, d = q.shape
+    sim = np.empty((N, N), dtype=np.float64)
+    if lib.castling_oracle_similarity(_ptr(q), _ptr(k), _ptr(sim), N, d, float(eps)):
+        raise RuntimeError("castling_oracle_similarity failed")
+    return sim
+
+
+def angular_exact(x: float) -> float:
+    """Eq. 5 on a cosine: 1 - arccos(x)/pi."""
+    return load().castling_oracle_angular_exact(float(x))
+
+
+def angular_series(x: float, kmax: int) -> float:
+    """Eq. 8 truncated after the k = kmax residual term (kmax = 0: the kept linear part)."""
+    return load().castling_oracle_angular_series(float(x), int(kmax))
+
+
+def angular_series_coeff(k: int) -> float:
+    """Eq. 8's coefficient (2k)! / (2^(2k) (k!)^2 (2k+1))."""
+    return load().castling_oracle_angular_series_coeff(int(k))
