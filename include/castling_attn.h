@@ -1,0 +1,153 @@
+/*
+ * castling_attn.h -- C ABI of the linear-angular attention core for NVIDIA B200 (sm_100a).
+ *
+ * The library computes, for every batch b and head h independently, the
+ * inference-time attention of Castling-ViT (arXiv 2211.10526, Sec. 3.2.1):
+ *
+ *     out_t = 1/2 * sum_j v_j  +  (1/pi) * q^_t (K^^T V)  +  DWConv(V)_t
+ *
+ * where q^_t = q_t / max(||q_t||_2, eps) and k^_j likewise are the unit rows the
+ * paper prescribes for Q and K (text after Eq. 8; last sentence of Sec. 3.2.1),
+ * 1/2 + (q^_t . k^_j)/pi is the kept "linear-angular" part of the expanded
+ * angular kernel (Eq. 8), the product is re-associated so that only the d x d
+ * state K^^T V and the token sum of V are formed (Eq. 9 and the "kernel-based
+ * linear attention" paragraph of Sec. 3.1), and DWConv is the learnable
+ * depthwise convolution applied to the value tokens on their 2-D grid
+ * (Eq. 9, term M_DW V).  The masked softmax branch of Eq. 9-10 is all zeros at
+ * inference (Sec. 3.2.2, "Castling during ViT inference") and is not computed.
+ *
+ * No row-sum denominator and no 1/sqrt(d) factor appear in Eq. 8-9, and none
+ * is applied.  V is used as given.  The convolution is a cross-correlation
+ * with zero "same" padding and stride 1, one ksize x ksize filter per
+ * head-channel ch = h*d + j, plus an optional bias.
+ *
+ * All tensor arguments are plain pointers; nothing here depends on PyTorch.
+ * Nothing in this library runs the computation on the CPU: without a CUDA
+ * device of compute capability 10.x every forward call returns an error.
+ */
+#ifndef CASTLING_ATTN_H_
+#define CASTLING_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct castling_attn castling_attn_t; /* opaque handle */
+
+typedef enum {
+    CASTLING_F32 = 0, /* fp32 in, fp32 arithmetic, fp32 out                      */
+    CASTLING_BF16 = 1 /* bf16 in, fp32 accumulation (bf16 tensor-core operands), */
+                      /* one round-to-nearest-even to bf16 at the store          */
+} castling_dtype_t;
+
+/* Return codes.  0 is success; everything else is negative. */
+enum {
+    CASTLING_OK = 0,
+    CASTLING_ERR_INVALID_ARG = -1, /* NULL pointer, non-positive size, even ksize, overlap   */
+    CASTLING_ERR_UNSUPPORTED = -2, /* d not a multiple of 16 or > 128, ksize > 7, bad dtype  */
+    CASTLING_ERR_ALIGNMENT = -3,   /* a tensor pointer is not 16-byte aligned                */
+    CASTLING_ERR_ARCH = -4,        /* current device is not compute capability 10.x          */
+    CASTLING_ERR_CUDA = -5,        /* a CUDA call failed; see castling_attn_last_cuda_error  */
+    CASTLING_ERR_OOM = -6,         /* workspace allocation failed or exceeds max_workspace   */
+    CASTLING_ERR_DEVICE = -7       /* a kernel reported a bounded wait that ran out          */
+};
+
+/* Kernel families the dispatcher can be pinned to (testing and benchmarking). */
+enum {
+    CASTLING_PATH_AUTO = 0,
+    CASTLING_PATH_SIMT = 1,   /* CUDA-core FMA kernels: every dtype, d and ksize supported   */
+    CASTLING_PATH_TENSOR = 2  /* tcgen05/TMEM + TMA kernels: bf16, d = 64                    */
+};
+
+typedef struct {
+    int ksize;            /* depthwise filter side: odd, 1..7                                  */
+    double eps;           /* floor on ||q||, ||k||; <= 0 selects the default 1e-12.  A zero    */
+                          /* row therefore has cosine 0 with everything (similarity 1/2).     */
+    int force_path;       /* CASTLING_PATH_*; AUTO picks by dtype, d and N                     */
+    size_t max_workspace; /* cap on handle-owned device memory in bytes; 0 = no cap            */
+} castling_attn_config_t;
+
+/*
+ * castling_attn_create: make a handle bound to the CURRENT CUDA device.
+ *   cfg         host pointer, read once; NULL selects {ksize 3, eps 1e-12, AUTO, no cap}.
+ *   out_handle  host pointer receiving the handle; set to NULL on failure.
+ * Allocates nothing on the device.  Errors: INVALID_ARG, UNSUPPORTED (ksize), ARCH, CUDA.
+ */
+int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** out_handle);
+
+/*
+ * castling_attn_forward: enqueue one forward pass on `stream` and return without
+ * synchronising (Eq. 8-9 as stated at the top of this file).
+ *
+ *   q, k, v     DEVICE pointers, [B, H, N, d] contiguous, d innermost, N = gridH*gridW,
+ *               token t = y*gridW + x.  Read only.  16-byte aligned.
+ *   dw_weight   DEVICE pointer, [H*d, ksize, ksize], same dtype as q.  Read only.
+ *   dw_bias     DEVICE pointer, [H*d], same dtype, or NULL for no bias.
+ *   out         DEVICE pointer, [B, H, N, d], same dtype; every element is written exactly
+ *               once.  Must not overlap any input.  16-byte aligned.
+ *   B,H,gridH,gridW,d   positive; d a multiple of 16, d <= 128.
+ *   dtype       element type of all six tensors.
+ *   stream      a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *
+ * Ownership: the caller owns every tensor; the handle owns a workspace (partial and final
+ * d x d states, token sums) that may be (re)allocated with cudaMalloc on the first call
+ * for a larger shape -- that call synchronises the device; later calls of the same or a
+ * smaller shape allocate nothing.
+ * A handle serves one host thread and one stream at a time; distinct handles are
+ * independent.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, OOM, CUDA.  Nothing aborts
+ * and no exception crosses this boundary.
+ */
+int castling_attn_forward(castling_attn_t* handle,
+                          const void* q, const void* k, const void* v,
+                          const void* dw_weight, const void* dw_bias, void* out,
+                          int B, int H, int gridH, int gridW, int d,
+                          castling_dtype_t dtype, void* stream);
+
+/*
+ * castling_attn_forward_host: the same computation with every tensor in HOST memory.
+ * Copies q, k, v, dw_weight and dw_bias to handle-owned device staging buffers on
+ * `stream`, runs the forward pass, copies `out` back and synchronises the stream
+ * before returning, so on return `out` holds the result.  Pinned host memory makes the
+ * copies asynchronous to each other; pageable memory also works.  Shapes, dtype and
+ * errors as for castling_attn_forward (alignment is not required of host pointers).
+ */
+int castling_attn_forward_host(castling_attn_t* handle,
+                               const void* q, const void* k, const void* v,
+                               const void* dw_weight, const void* dw_bias, void* out,
+                               int B, int H, int gridH, int gridW, int d,
+                               castling_dtype_t dtype, void* stream);
+
+/*
+ * castling_attn_destroy: free the workspace and the handle.  The caller must have
+ * synchronised every stream the handle was used on.  NULL is accepted.
+ */
+int castling_attn_destroy(castling_attn_t* handle);
+
+/* Bytes of handle-owned device workspace a forward of this shape needs (0 on bad arguments). */
+size_t castling_attn_workspace_bytes(int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype);
+
+/* Static, NUL-terminated description of a return code. */
+const char* castling_attn_error_string(int code);
+
+/* The cudaError_t (as int) behind the handle's most recent CASTLING_ERR_CUDA / OOM, else 0. */
+int castling_attn_last_cuda_error(const castling_attn_t* handle);
+
+/*
+ * castling_attn_last_path: which kernel family (CASTLING_PATH_SIMT / _TENSOR) the handle's
+ * most recent successful forward used, and how many kernels it launched (may be NULL).
+ */
+int castling_attn_last_path(const castling_attn_t* handle, int* kernel_launches);
+
+/*
+ * castling_attn_device_status: read back the handle's device-side status word
+ * (synchronises `stream`).  0 = every bounded wait in the kernels completed; otherwise
+ * returns CASTLING_ERR_DEVICE and stores the raw word in *raw (may be NULL).
+ */
+int castling_attn_device_status(castling_attn_t* handle, void* stream, unsigned int* raw);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CASTLING_ATTN_H_ */

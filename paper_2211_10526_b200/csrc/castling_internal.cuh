@@ -1,0 +1,43 @@
+// Internal declarations shared by the host dispatcher and the kernel files of
+// the linear-angular attention library.  Not part of the public ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace castling {
+
+constexpr float kInvPi = 0.31830988618379067154f;
+
+// One forward call, as the kernels see it.
+struct Problem {
+    const void* q;
+    const void* k;
+    const void* v;
+    const void* w;     // [H*d, ksize, ksize]
+    const void* bias;  // [H*d] or nullptr
+    void* out;
+    int B, H, gridH, gridW, d, ksize;
+    int N;             // gridH * gridW
+    int BH;            // B * H
+    bool bf16;
+    float eps2;        // eps^2: the floor under the sum of squares
+};
+
+// Workspace layout (fp32 words):
+//   [0, 64)                          header; word 0 is the device status word
+//   state  [BH][d*d + d]             raw sums: S = sum_n k^_n^T v_n, then s = sum_n v_n
+//   partial[BH][P][d*d + d]          per-split sums when the token range is split P ways
+constexpr size_t kHeaderWords = 64;
+
+inline size_t state_words(int d) { return (size_t)d * d + d; }
+
+// CUDA-core path.  simt_forward returns the cudaError_t of its launches.
+cudaError_t simt_forward(const Problem& p, float* ws_state, float* ws_partial, int P,
+                         cudaStream_t stream, int* launches);
+int simt_choose_splits(int BH, int N);
+bool simt_supports(int d, int ksize);
+
+}  // namespace castling
