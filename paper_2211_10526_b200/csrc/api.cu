@@ -1,0 +1,249 @@
+// Host side of the C ABI declared in include/castling_attn.h: handle, argument
+// validation, workspace, kernel-family dispatch.  No computation happens here.
+#include "castling_attn.h"
+#include "castling_internal.cuh"
+
+#include <new>
+
+using castling::Problem;
+
+struct castling_attn {
+    castling_attn_config_t cfg;
+    int device = 0;
+    int sm_count = 0;
+    float* ws = nullptr;        // header | state | partial
+    size_t ws_bytes = 0;
+    char* stage = nullptr;      // device staging for castling_attn_forward_host
+    size_t stage_bytes = 0;
+    int last_cuda_error = 0;
+    int last_path = 0;
+    int last_launches = 0;
+};
+
+namespace {
+
+size_t elem_bytes(castling_dtype_t t) { return t == CASTLING_F32 ? 4 : 2; }
+
+// header | state [BH] | partial [BH][P] (only when the token range is split)
+size_t workspace_words(int BH, int N, int d) {
+    const int P = castling::simt_choose_splits(BH, N);
+    return castling::kHeaderWords + (size_t)BH * castling::state_words(d) * (1 + (P > 1 ? P : 0));
+}
+
+int fail_cuda(castling_attn* h, cudaError_t e, int code = CASTLING_ERR_CUDA) {
+    if (h) h->last_cuda_error = (int)e;
+    (void)cudaGetLastError();  // reset the runtime's last-error slot
+    return code;
+}
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+    return x < y + nb && y < x + na;
+}
+
+// Shape / dtype checks shared by the device- and host-pointer entry points.
+int check_shape(const castling_attn* h, int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype) {
+    if (!h) return CASTLING_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || gridH <= 0 || gridW <= 0 || d <= 0) return CASTLING_ERR_INVALID_ARG;
+    if (dtype != CASTLING_F32 && dtype != CASTLING_BF16) return CASTLING_ERR_UNSUPPORTED;
+    if (!castling::simt_supports(d, h->cfg.ksize)) return CASTLING_ERR_UNSUPPORTED;
+    const long long N = (long long)gridH * gridW, BH = (long long)B * H;
+    if (N > (1 << 24) || BH > (1 << 20) || BH * ((N + 63) / 64) > 0x7fffffffLL) return CASTLING_ERR_UNSUPPORTED;
+    if (BH * N * d > (1LL << 40)) return CASTLING_ERR_UNSUPPORTED;
+    return CASTLING_OK;
+}
+
+int ensure_workspace(castling_attn* h, int BH, int N, int d) {
+    const size_t need = workspace_words(BH, N, d) * sizeof(float);
+    if (need <= h->ws_bytes) return CASTLING_OK;
+    if (h->cfg.max_workspace && need > h->cfg.max_workspace) return CASTLING_ERR_OOM;
+    cudaError_t e = cudaDeviceSynchronize();  // nothing may still be using the old buffer
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    if (h->ws) cudaFree(h->ws);
+    h->ws = nullptr; h->ws_bytes = 0;
+    e = cudaMalloc((void**)&h->ws, need);
+    if (e != cudaSuccess) return fail_cuda(h, e, CASTLING_ERR_OOM);
+    e = cudaMemset(h->ws, 0, castling::kHeaderWords * sizeof(float));
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->ws_bytes = need;
+    return CASTLING_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** out_handle) {
+    if (!out_handle) return CASTLING_ERR_INVALID_ARG;
+    *out_handle = nullptr;
+    castling_attn_config_t c = {3, 1e-12, CASTLING_PATH_AUTO, 0};
+    if (cfg) c = *cfg;
+    if (c.eps <= 0.0) c.eps = 1e-12;
+    if (c.ksize <= 0 || (c.ksize & 1) == 0) return CASTLING_ERR_INVALID_ARG;
+    if (c.ksize > 7) return CASTLING_ERR_UNSUPPORTED;
+    if (c.force_path < CASTLING_PATH_AUTO || c.force_path > CASTLING_PATH_TENSOR) return CASTLING_ERR_INVALID_ARG;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(nullptr, e);
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) return fail_cuda(nullptr, e);
+    if (prop.major != 10) return CASTLING_ERR_ARCH;
+    castling_attn* h = new (std::nothrow) castling_attn();
+    if (!h) return CASTLING_ERR_OOM;
+    h->cfg = c;
+    h->device = dev;
+    h->sm_count = prop.multiProcessorCount;
+    *out_handle = h;
+    return CASTLING_OK;
+}
+
+int castling_attn_destroy(castling_attn_t* h) {
+    if (!h) return CASTLING_OK;
+    if (h->ws) cudaFree(h->ws);
+    if (h->stage) cudaFree(h->stage);
+    delete h;
+    return CASTLING_OK;
+}
+
+size_t castling_attn_workspace_bytes(int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype) {
+    if (B <= 0 || H <= 0 || gridH <= 0 || gridW <= 0 || d <= 0 || d > 128 || d % 16) return 0;
+    if (dtype != CASTLING_F32 && dtype != CASTLING_BF16) return 0;
+    return workspace_words(B * H, gridH * gridW, d) * sizeof(float);
+}
+
+const char* castling_attn_error_string(int code) {
+    switch (code) {
+        case CASTLING_OK: return "success";
+        case CASTLING_ERR_INVALID_ARG: return "invalid argument (NULL pointer, non-positive size, even ksize or overlapping buffers)";
+        case CASTLING_ERR_UNSUPPORTED: return "unsupported head width, filter size, dtype or problem size";
+        case CASTLING_ERR_ALIGNMENT: return "tensor pointer is not 16-byte aligned";
+        case CASTLING_ERR_ARCH: return "current CUDA device is not compute capability 10.x";
+        case CASTLING_ERR_CUDA: return "a CUDA call failed (see castling_attn_last_cuda_error)";
+        case CASTLING_ERR_OOM: return "workspace allocation failed or exceeds max_workspace";
+        case CASTLING_ERR_DEVICE: return "a kernel gave up on a bounded wait";
+        default: return "unknown castling_attn error code";
+    }
+}
+
+int castling_attn_last_cuda_error(const castling_attn_t* h) { return h ? h->last_cuda_error : 0; }
+
+int castling_attn_last_path(const castling_attn_t* h, int* kernel_launches) {
+    if (!h) return CASTLING_ERR_INVALID_ARG;
+    if (kernel_launches) *kernel_launches = h->last_launches;
+    return h->last_path;
+}
+
+}  // extern "C"
+
+namespace {
+
+// Enqueue the kernels for one validated problem whose tensors are all on the device.
+int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
+    int rc = ensure_workspace(h, p.BH, p.N, p.d);
+    if (rc != CASTLING_OK) return rc;
+    if (h->cfg.force_path == CASTLING_PATH_TENSOR) return CASTLING_ERR_UNSUPPORTED;  // not built yet
+    float* state = h->ws + castling::kHeaderWords;
+    float* partial = state + (size_t)p.BH * castling::state_words(p.d);
+    const int P = castling::simt_choose_splits(p.BH, p.N);
+    int launches = 0;
+    const cudaError_t e = castling::simt_forward(p, state, partial, P, stream, &launches);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->last_path = CASTLING_PATH_SIMT;
+    h->last_launches = launches;
+    return CASTLING_OK;
+}
+
+Problem make_problem(const castling_attn* h, const void* q, const void* k, const void* v, const void* w,
+                     const void* bias, void* out, int B, int H, int gridH, int gridW, int d,
+                     castling_dtype_t dtype) {
+    Problem p;
+    p.q = q; p.k = k; p.v = v; p.w = w; p.bias = bias; p.out = out;
+    p.B = B; p.H = H; p.gridH = gridH; p.gridW = gridW; p.d = d; p.ksize = h->cfg.ksize;
+    p.N = gridH * gridW; p.BH = B * H;
+    p.bf16 = (dtype == CASTLING_BF16);
+    p.eps2 = (float)(h->cfg.eps * h->cfg.eps);
+    return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+int castling_attn_forward(castling_attn_t* h, const void* q, const void* k, const void* v,
+                          const void* dw_weight, const void* dw_bias, void* out,
+                          int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype, void* stream) {
+    int rc = check_shape(h, B, H, gridH, gridW, d, dtype);
+    if (rc != CASTLING_OK) return rc;
+    if (!q || !k || !v || !dw_weight || !out) return CASTLING_ERR_INVALID_ARG;
+    const size_t eb = elem_bytes(dtype);
+    const size_t tensor_bytes = (size_t)B * H * gridH * gridW * d * eb;
+    const size_t w_bytes = (size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb;
+    const size_t b_bytes = (size_t)H * d * eb;
+    const void* ptrs[4] = {q, k, v, out};
+    for (const void* ptr : ptrs)
+        if ((uintptr_t)ptr & 15) return CASTLING_ERR_ALIGNMENT;
+    if (overlaps(out, tensor_bytes, q, tensor_bytes) || overlaps(out, tensor_bytes, k, tensor_bytes) ||
+        overlaps(out, tensor_bytes, v, tensor_bytes) || overlaps(out, tensor_bytes, dw_weight, w_bytes) ||
+        (dw_bias && overlaps(out, tensor_bytes, dw_bias, b_bytes)))
+        return CASTLING_ERR_INVALID_ARG;
+    const Problem p = make_problem(h, q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, dtype);
+    return run_device(h, p, static_cast<cudaStream_t>(stream));
+}
+
+int castling_attn_forward_host(castling_attn_t* h, const void* q, const void* k, const void* v,
+                               const void* dw_weight, const void* dw_bias, void* out,
+                               int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype, void* stream) {
+    int rc = check_shape(h, B, H, gridH, gridW, d, dtype);
+    if (rc != CASTLING_OK) return rc;
+    if (!q || !k || !v || !dw_weight || !out) return CASTLING_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t eb = elem_bytes(dtype);
+    const size_t tb = (((size_t)B * H * gridH * gridW * d * eb) + 255) & ~(size_t)255;
+    const size_t wb = (((size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb) + 255) & ~(size_t)255;
+    const size_t bb = (((size_t)H * d * eb) + 255) & ~(size_t)255;
+    const size_t need = 4 * tb + wb + bb;
+    if (need > h->stage_bytes) {
+        if (h->cfg.max_workspace && need > h->cfg.max_workspace) return CASTLING_ERR_OOM;
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        if (h->stage) cudaFree(h->stage);
+        h->stage = nullptr; h->stage_bytes = 0;
+        e = cudaMalloc((void**)&h->stage, need);
+        if (e != cudaSuccess) return fail_cuda(h, e, CASTLING_ERR_OOM);
+        h->stage_bytes = need;
+    }
+    char* dq = h->stage; char* dk = dq + tb; char* dv = dk + tb; char* dout = dv + tb;
+    char* dw = dout + tb; char* db = dw + wb;
+    const size_t t_exact = (size_t)B * H * gridH * gridW * d * eb;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(dq, q, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaMemcpyAsync(dk, k, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaMemcpyAsync(dv, v, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaMemcpyAsync(dw, dw_weight, (size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb,
+                             cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
+    if (dw_bias &&
+        (e = cudaMemcpyAsync(db, dw_bias, (size_t)H * d * eb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return fail_cuda(h, e);
+    const Problem p = make_problem(h, dq, dk, dv, dw, dw_bias ? db : nullptr, dout, B, H, gridH, gridW, d, dtype);
+    rc = run_device(h, p, st);
+    if (rc != CASTLING_OK) return rc;
+    if ((e = cudaMemcpyAsync(out, dout, t_exact, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(h, e);
+    return CASTLING_OK;
+}
+
+int castling_attn_device_status(castling_attn_t* h, void* stream, unsigned int* raw) {
+    if (!h) return CASTLING_ERR_INVALID_ARG;
+    unsigned int word = 0;
+    if (h->ws) {
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        cudaError_t e = cudaMemcpyAsync(&word, h->ws, sizeof(word), cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(h, e);
+    }
+    if (raw) *raw = word;
+    return word ? CASTLING_ERR_DEVICE : CASTLING_OK;
+}
+
+}  // extern "C"
