@@ -30,6 +30,12 @@
 
 #include <stddef.h>
 
+#if defined(__GNUC__)
+#define CASTLING_API __attribute__((visibility("default")))
+#else
+#define CASTLING_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -75,7 +81,7 @@ typedef struct {
  *   out_handle  host pointer receiving the handle; set to NULL on failure.
  * Allocates nothing on the device.  Errors: INVALID_ARG, UNSUPPORTED (ksize), ARCH, CUDA.
  */
-int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** out_handle);
+CASTLING_API int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** out_handle);
 
 /*
  * castling_attn_forward: enqueue one forward pass on `stream` and return without
@@ -99,7 +105,7 @@ int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** ou
  * independent.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, OOM, CUDA.  Nothing aborts
  * and no exception crosses this boundary.
  */
-int castling_attn_forward(castling_attn_t* handle,
+CASTLING_API int castling_attn_forward(castling_attn_t* handle,
                           const void* q, const void* k, const void* v,
                           const void* dw_weight, const void* dw_bias, void* out,
                           int B, int H, int gridH, int gridW, int d,
@@ -113,7 +119,7 @@ int castling_attn_forward(castling_attn_t* handle,
  * copies asynchronous to each other; pageable memory also works.  Shapes, dtype and
  * errors as for castling_attn_forward (alignment is not required of host pointers).
  */
-int castling_attn_forward_host(castling_attn_t* handle,
+CASTLING_API int castling_attn_forward_host(castling_attn_t* handle,
                                const void* q, const void* k, const void* v,
                                const void* dw_weight, const void* dw_bias, void* out,
                                int B, int H, int gridH, int gridW, int d,
@@ -123,29 +129,29 @@ int castling_attn_forward_host(castling_attn_t* handle,
  * castling_attn_destroy: free the workspace and the handle.  The caller must have
  * synchronised every stream the handle was used on.  NULL is accepted.
  */
-int castling_attn_destroy(castling_attn_t* handle);
+CASTLING_API int castling_attn_destroy(castling_attn_t* handle);
 
 /* Bytes of handle-owned device workspace a forward of this shape needs (0 on bad arguments). */
-size_t castling_attn_workspace_bytes(int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype);
+CASTLING_API size_t castling_attn_workspace_bytes(int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype);
 
 /* Static, NUL-terminated description of a return code. */
-const char* castling_attn_error_string(int code);
+CASTLING_API const char* castling_attn_error_string(int code);
 
 /* The cudaError_t (as int) behind the handle's most recent CASTLING_ERR_CUDA / OOM, else 0. */
-int castling_attn_last_cuda_error(const castling_attn_t* handle);
+CASTLING_API int castling_attn_last_cuda_error(const castling_attn_t* handle);
 
 /*
  * castling_attn_last_path: which kernel family (CASTLING_PATH_SIMT / _TENSOR) the handle's
  * most recent successful forward used, and how many kernels it launched (may be NULL).
  */
-int castling_attn_last_path(const castling_attn_t* handle, int* kernel_launches);
+CASTLING_API int castling_attn_last_path(const castling_attn_t* handle, int* kernel_launches);
 
 /*
  * castling_attn_device_status: read back the handle's device-side status word
  * (synchronises `stream`).  0 = every bounded wait in the kernels completed; otherwise
  * returns CASTLING_ERR_DEVICE and stores the raw word in *raw (may be NULL).
  */
-int castling_attn_device_status(castling_attn_t* handle, void* stream, unsigned int* raw);
+CASTLING_API int castling_attn_device_status(castling_attn_t* handle, void* stream, unsigned int* raw);
 
 #ifdef __cplusplus
 }

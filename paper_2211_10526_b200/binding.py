@@ -1,0 +1,114 @@
+"""ctypes binding of ``include/castling_attn.h``: argument marshalling only.
+
+Function names mirror the C ABI.  Tensors are passed as raw addresses
+(``tensor.data_ptr()``); PyTorch is used by callers for device memory and streams, never
+for arithmetic.  Importing this module loads the compiled CUDA library and raises if it
+is missing: there is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcastling_attn.so")
+
+CASTLING_F32, CASTLING_BF16 = 0, 1
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARCH, ERR_CUDA, ERR_OOM, ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6, -7
+
+
+class castling_attn_config_t(ctypes.Structure):
+    _fields_ = [("ksize", ctypes.c_int), ("eps", ctypes.c_double), ("force_path", ctypes.c_int),
+                ("max_workspace", ctypes.c_size_t)]
+
+
+class CastlingError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {error_string(code)} (code {code})")
+        self.code = code
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is not built; run `python -m paper_2211_10526_b200.build` "
+                          "(needs nvcc; there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.castling_attn_create.restype = i
+    lib.castling_attn_create.argtypes = [ctypes.POINTER(castling_attn_config_t), ctypes.POINTER(vp)]
+    fwd_args = [vp] * 7 + [i] * 5 + [i, vp]
+    lib.castling_attn_forward.restype = i
+    lib.castling_attn_forward.argtypes = fwd_args
+    lib.castling_attn_forward_host.restype = i
+    lib.castling_attn_forward_host.argtypes = fwd_args
+    lib.castling_attn_destroy.restype = i
+    lib.castling_attn_destroy.argtypes = [vp]
+    lib.castling_attn_workspace_bytes.restype = sz
+    lib.castling_attn_workspace_bytes.argtypes = [i] * 6
+    lib.castling_attn_error_string.restype = ctypes.c_char_p
+    lib.castling_attn_error_string.argtypes = [i]
+    lib.castling_attn_last_cuda_error.restype = i
+    lib.castling_attn_last_cuda_error.argtypes = [vp]
+    lib.castling_attn_last_path.restype = i
+    lib.castling_attn_last_path.argtypes = [vp, ctypes.POINTER(i)]
+    lib.castling_attn_device_status.restype = i
+    lib.castling_attn_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint)]
+    return lib
+
+
+lib = _load()
+
+
+def error_string(code: int) -> str:
+    return lib.castling_attn_error_string(int(code)).decode()
+
+
+def castling_attn_create(ksize: int = 3, eps: float = 0.0, force_path: int = PATH_AUTO,
+                         max_workspace: int = 0) -> int:
+    """Returns the handle (an integer address); raises CastlingError on failure."""
+    cfg = castling_attn_config_t(int(ksize), float(eps), int(force_path), int(max_workspace))
+    h = ctypes.c_void_p()
+    rc = lib.castling_attn_create(ctypes.byref(cfg), ctypes.byref(h))
+    if rc != OK:
+        raise CastlingError(rc, "castling_attn_create")
+    return h.value
+
+
+def castling_attn_forward(handle, q: int, k: int, v: int, dw_weight: int, dw_bias: Optional[int], out: int,
+                          B: int, H: int, gridH: int, gridW: int, d: int, dtype: int, stream: int = 0) -> int:
+    """Raw call on device addresses; returns the C return code."""
+    return lib.castling_attn_forward(handle, q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, dtype,
+                                     stream or None)
+
+
+def castling_attn_forward_host(handle, q: int, k: int, v: int, dw_weight: int, dw_bias: Optional[int], out: int,
+                               B: int, H: int, gridH: int, gridW: int, d: int, dtype: int, stream: int = 0) -> int:
+    """Raw call on host addresses (copies in, computes, copies out, synchronises)."""
+    return lib.castling_attn_forward_host(handle, q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, dtype,
+                                          stream or None)
+
+
+def castling_attn_destroy(handle) -> int:
+    return lib.castling_attn_destroy(handle)
+
+
+def castling_attn_workspace_bytes(B, H, gridH, gridW, d, dtype) -> int:
+    return lib.castling_attn_workspace_bytes(B, H, gridH, gridW, d, dtype)
+
+
+def castling_attn_last_cuda_error(handle) -> int:
+    return lib.castling_attn_last_cuda_error(handle)
+
+
+def castling_attn_last_path(handle):
+    n = ctypes.c_int(0)
+    path = lib.castling_attn_last_path(handle, ctypes.byref(n))
+    return path, n.value
+
+
+def castling_attn_device_status(handle, stream: int = 0):
+    raw = ctypes.c_uint(0)
+    rc = lib.castling_attn_device_status(handle, stream or None, ctypes.byref(raw))
+    return rc, raw.value
