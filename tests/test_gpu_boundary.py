@@ -1,0 +1,176 @@
+"""GPU tests of the C-ABI boundary: error codes, ownership, memory safety, determinism."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _b():
+    from paper_2211_10526_b200 import binding
+    return binding
+
+
+def _dev(call):
+    dev = torch.device("cuda:0")
+    return [t.to(dev) for t in (call.q, call.k, call.v, call.dw_weight, call.dw_bias)]
+
+
+def _raw_forward(b, h, q, k, v, w, bias, out, s, dtype_code=None, stream=0):
+    code = (b.CASTLING_F32 if q.dtype == torch.float32 else b.CASTLING_BF16) if dtype_code is None else dtype_code
+    return b.castling_attn_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), w.data_ptr(),
+                                   None if bias is None else bias.data_ptr(), out.data_ptr(),
+                                   s.B, s.H, s.gridH, s.gridW, s.d, code, stream)
+
+
+def test_error_codes():
+    b = _b()
+    c = workloads.custom_call(1, 2, 4, 4, 32, 3, "f32", seed=400)
+    q, k, v, w, bias = _dev(c)
+    out = torch.empty_like(q)
+    s = c.shape
+    h = b.castling_attn_create(3)
+    try:
+        assert _raw_forward(b, h, q, k, v, w, bias, out, s) == b.OK
+        # NULL tensor
+        assert b.castling_attn_forward(h, None, k.data_ptr(), v.data_ptr(), w.data_ptr(), None, out.data_ptr(),
+                                       1, 2, 4, 4, 32, 0) == b.ERR_INVALID_ARG
+        # non-positive dims
+        for dims in ((0, 2, 4, 4, 32), (1, 0, 4, 4, 32), (1, 2, -4, 4, 32), (1, 2, 4, 0, 32), (1, 2, 4, 4, 0)):
+            assert b.castling_attn_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), w.data_ptr(), None,
+                                           out.data_ptr(), *dims, 0) == b.ERR_INVALID_ARG
+        # unsupported head width / dtype
+        for d in (8, 33, 144):
+            assert b.castling_attn_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), w.data_ptr(), None,
+                                           out.data_ptr(), 1, 2, 4, 4, d, 0) == b.ERR_UNSUPPORTED
+        assert _raw_forward(b, h, q, k, v, w, bias, out, s, dtype_code=5) == b.ERR_UNSUPPORTED
+        # misaligned tensor pointer (4 bytes off a 16-byte boundary)
+        flat = torch.empty(q.numel() + 8, dtype=q.dtype, device=q.device)
+        mis = flat[1:1 + q.numel()].view_as(q)
+        assert mis.data_ptr() % 16 != 0
+        assert _raw_forward(b, h, mis, k, v, w, bias, out, s) == b.ERR_ALIGNMENT
+        assert _raw_forward(b, h, q, k, v, w, bias, mis, s) == b.ERR_ALIGNMENT
+        # output overlapping an input
+        assert _raw_forward(b, h, q, k, v, w, bias, v, s) == b.ERR_INVALID_ARG
+        both = torch.empty(2 * q.numel() - 64, dtype=q.dtype, device=q.device)
+        a_in = both[:q.numel()].view_as(q)
+        a_out = both[q.numel() - 64:].view_as(q)
+        assert _raw_forward(b, h, a_in, k, v, w, bias, a_out, s) == b.ERR_INVALID_ARG
+        # workspace cap
+        h2 = b.castling_attn_create(3, max_workspace=128)
+        assert _raw_forward(b, h2, q, k, v, w, bias, out, s) == b.ERR_OOM
+        b.castling_attn_destroy(h2)
+        # the handle still works after every rejected call
+        assert _raw_forward(b, h, q, k, v, w, bias, out, s) == b.OK
+        torch.cuda.synchronize()
+        path, launches = b.castling_attn_last_path(h)
+        assert path in (b.PATH_SIMT, b.PATH_TENSOR) and launches >= 1
+        assert b.castling_attn_device_status(h) == (b.OK, 0)
+    finally:
+        b.castling_attn_destroy(h)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(2, 3, 9, 7, 32, 3), (1, 2, 70, 75, 64, 5), (4, 12, 14, 14, 64, 3)],
+                         ids=["small", "split", "deit"])
+def test_guard_bands_and_inputs_untouched(shape, dtype):
+    """Bytes before and after `out` keep their pattern; inputs are bit-identical afterwards."""
+    b = _b()
+    c = workloads.custom_call(*shape, dtype, seed=410)
+    q, k, v, w, bias = _dev(c)
+    s = c.shape
+    n = q.numel()
+    guard = 4096
+    buf = torch.full((n + 2 * guard,), float("nan"), dtype=q.dtype, device=q.device)
+    out = buf[guard:guard + n].view_as(q)
+    assert out.data_ptr() % 16 == 0
+    before = [t.clone() for t in (q, k, v, w, bias)]
+    h = b.castling_attn_create(s.ksize)
+    try:
+        assert _raw_forward(b, h, q, k, v, w, bias, out, s) == b.OK
+        torch.cuda.synchronize()
+    finally:
+        b.castling_attn_destroy(h)
+    assert torch.isnan(buf[:guard]).all() and torch.isnan(buf[guard + n:]).all()
+    assert torch.isfinite(out.float()).all(), "an output element was never written"
+    for t, t0 in zip((q, k, v, w, bias), before):
+        assert torch.equal(t.view(torch.uint8), t0.view(torch.uint8))
+
+
+@pytest.mark.parametrize("name,idx", [("c1_fp32_tiny", 0), ("c4_detection_bf16", 0), ("c5_sweep_bf16", 1)])
+def test_bitwise_reproducible(name, idx):
+    """Reductions run in a fixed order: two runs give identical bits, also from a second handle."""
+    b = _b()
+    (c,) = list(workloads.iter_workload(name, only=[idx]))
+    q, k, v, w, bias = _dev(c)
+    s = c.shape
+    outs = []
+    for _ in range(2):
+        h = b.castling_attn_create(s.ksize)
+        for _ in range(2):
+            out = torch.empty_like(q)
+            assert _raw_forward(b, h, q, k, v, w, bias, out, s) == b.OK
+            torch.cuda.synchronize()
+            outs.append(out)
+        b.castling_attn_destroy(h)
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.uint8), outs[0].view(torch.uint8))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_host_entry_point_matches_device_entry_point(dtype):
+    from paper_2211_10526_b200 import CastlingAttn
+    c = workloads.custom_call(2, 4, 14, 14, 32, 3, dtype, seed=420)
+    s = c.shape
+    with CastlingAttn(ksize=3) as attn:
+        pinned = [t.pin_memory() for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)]
+        out_h = torch.empty_like(c.q).pin_memory()
+        attn.forward_host(*pinned, s.gridH, s.gridW, out=out_h)
+        out_d = attn.forward(*_dev(c), s.gridH, s.gridW)
+        torch.cuda.synchronize()
+        assert torch.equal(out_d.cpu().view(torch.uint8), out_h.view(torch.uint8))
+        # pageable memory and no bias also work
+        out_p = attn.forward_host(c.q, c.k, c.v, c.dw_weight, None, s.gridH, s.gridW)
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, None, s.gridH, s.gridW, 3)
+    err = np.max(np.abs(out_p.double().numpy() - ref)) / np.max(np.abs(ref))
+    assert err <= (1e-5 if dtype == "f32" else 2e-2)
+
+
+def test_two_handles_two_streams_and_shape_changes():
+    """Distinct handles are independent; one handle may serve shapes of growing and shrinking size."""
+    from paper_2211_10526_b200 import CastlingAttn
+    calls = [workloads.custom_call(1, 2, 6, 6, 32, 3, "bf16", seed=430),
+             workloads.custom_call(2, 4, 40, 40, 64, 3, "bf16", seed=431),
+             workloads.custom_call(1, 1, 3, 5, 64, 3, "bf16", seed=432)]
+    refs = [oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, c.shape.gridH, c.shape.gridW, 3, threads=8)
+            for c in calls]
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    a1, a2 = CastlingAttn(3), CastlingAttn(3)
+    outs = []
+    dev_calls = [_dev(c) for c in calls]
+    torch.cuda.synchronize()
+    for i, (c, d) in enumerate(zip(calls, dev_calls)):
+        with torch.cuda.stream(s1 if i % 2 == 0 else s2):
+            attn = a1 if i % 2 == 0 else a2
+            outs.append(attn.forward(*d, c.shape.gridH, c.shape.gridW))
+    # and the same handle across all shapes on one stream
+    with torch.cuda.stream(s1):
+        outs2 = [a1.forward(*d, c.shape.gridH, c.shape.gridW) for c, d in zip(calls, dev_calls)]
+    torch.cuda.synchronize()
+    for o, o2, ref in zip(outs, outs2, refs):
+        for t in (o, o2):
+            err = np.max(np.abs(t.double().cpu().numpy() - ref)) / np.max(np.abs(ref))
+            assert err <= 2e-2
+    a1.close(); a2.close()
+
+
+def test_create_destroy_cycles():
+    b = _b()
+    for _ in range(50):
+        h = b.castling_attn_create(5)
+        assert b.castling_attn_destroy(h) == b.OK

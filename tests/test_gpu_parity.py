@@ -1,0 +1,188 @@
+"""GPU parity: the CUDA library against the float64 CPU oracle, through the C ABI.
+
+Error metric (both tolerances come with the method's acceptance bar): per call,
+``max_i |gpu_i - ref_i| / max_i |ref_i|`` must be <= 1e-5 for fp32 I/O and <= 2e-2 for
+bf16 I/O.  The oracle consumes the already-rounded fp32/bf16 inputs widened to float64
+and its output is not rounded.  Term-isolation cases make one term of Eq. 9 the whole
+output so that a defect in a small term cannot hide under a large one.
+"""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-2}
+
+
+def _lib():
+    import paper_2211_10526_b200 as pkg
+    return pkg
+
+
+def rel_err(got: torch.Tensor, ref: np.ndarray) -> float:
+    g = got.detach().double().cpu().numpy()
+    assert np.all(np.isfinite(g)), "non-finite GPU output"
+    return float(np.max(np.abs(g - ref)) / max(np.max(np.abs(ref)), 1e-30))
+
+
+def run_gpu(call: workloads.CallInputs, force_path: int = 0, bias: bool = True) -> torch.Tensor:
+    pkg = _lib()
+    s = call.shape
+    dev = torch.device("cuda:0")
+    q, k, v, w = (t.to(dev) for t in (call.q, call.k, call.v, call.dw_weight))
+    b = call.dw_bias.to(dev) if (bias and call.dw_bias is not None) else None
+    with pkg.CastlingAttn(ksize=s.ksize, force_path=force_path) as attn:
+        out = attn.forward(q, k, v, w, b, s.gridH, s.gridW)
+        torch.cuda.synchronize()
+        rc, raw = attn.device_status()
+        assert rc == 0, f"device status word {raw:#x}"
+    return out
+
+
+def run_oracle(call: workloads.CallInputs, bias: bool = True, threads: int = 8) -> np.ndarray:
+    s = call.shape
+    return oracle.forward(call.q, call.k, call.v, call.dw_weight, call.dw_bias if bias else None,
+                          s.gridH, s.gridW, s.ksize, threads=threads)
+
+
+def check(call, force_path=0, bias=True, tol=None):
+    ref = run_oracle(call, bias)
+    got = run_gpu(call, force_path, bias)
+    err = rel_err(got, ref)
+    tol = TOL[call.shape.dtype] if tol is None else tol
+    assert err <= tol, f"{call.shape.label()}: max-rel error {err:.3e} > {tol:.1e}"
+    return err
+
+
+# ---------------------------------------------------------------------------
+# the five configurations
+# ---------------------------------------------------------------------------
+CONFIG_CALLS = [("c1_fp32_tiny", 0), ("c2_levit_bf16", 0), ("c2_levit_bf16", 1), ("c2_levit_bf16", 2),
+                ("c3_deit_base_bf16", 0), ("c4_detection_bf16", 0), ("c5_sweep_bf16", 0), ("c5_sweep_bf16", 1)]
+
+
+@pytest.mark.parametrize("name,idx", CONFIG_CALLS, ids=[f"{n}-{i}" for n, i in CONFIG_CALLS])
+def test_config_parity(name, idx):
+    (call,) = list(workloads.iter_workload(name, only=[idx]))
+    check(call)
+
+
+@pytest.mark.parametrize("idx", [2, 3], ids=["side128", "side256"])
+def test_long_sequence_full_size(idx):
+    """Largest sweep points, every element compared."""
+    (call,) = list(workloads.iter_workload("c5_sweep_bf16", only=[idx]))
+    check(call)
+
+
+# ---------------------------------------------------------------------------
+# term isolation (Eq. 9 one term at a time)
+# ---------------------------------------------------------------------------
+def _iso_call(dtype, seed, B=2, H=3, gh=9, gw=11, d=32, ks=3):
+    return workloads.custom_call(B, H, gh, gw, d, ks, dtype, seed)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d", [32, 64])
+def test_linear_term_alone(dtype, d):
+    """Zero filters, zero bias and V with zero token-sum: only (1/pi) q^ (K^^T V) is left."""
+    c = _iso_call(dtype, 201, d=d)
+    v = c.v.float()
+    v = v - v.mean(dim=2, keepdim=True)
+    c.v = v.to(c.v.dtype)
+    c.dw_weight.zero_(); c.dw_bias.zero_()
+    check(c)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_half_sum_term_alone(dtype):
+    """Constant V: output is c (N/2 + q^ . sum k^ / pi); dominated by the 1/2 term."""
+    c = _iso_call(dtype, 202)
+    c.v[:] = c.v[:, :, :1, :].clone()
+    c.dw_weight.zero_(); c.dw_bias.zero_()
+    check(c)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("ks", [3, 5])
+def test_conv_term_alone(dtype, ks):
+    """K = 0 (cosine 0) and zero-sum V: attention part vanishes, the convolution is the output."""
+    c = _iso_call(dtype, 203, ks=ks)
+    v = c.v.float()
+    v = v - v.mean(dim=2, keepdim=True)
+    c.v = v.to(c.v.dtype)
+    # the token sum of the rounded V is not exactly zero; make the conv term dominate it
+    c.dw_weight = (c.dw_weight.float() * 30).to(c.dw_weight.dtype)
+    c.k.zero_()
+    check(c)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_delta_filter_is_identity(dtype):
+    c = _iso_call(dtype, 204)
+    c.dw_weight.zero_(); c.dw_weight[:, 1, 1] = 1.0
+    c.dw_bias.zero_()
+    c.k.zero_()
+    v = c.v.float(); v = v - v.mean(dim=2, keepdim=True); c.v = v.to(c.v.dtype)
+    got = run_gpu(c).double().cpu().numpy()
+    half_sum = 0.5 * c.v.double().sum(dim=2, keepdim=True).numpy()
+    np.testing.assert_allclose(got, c.v.double().numpy() + half_sum, rtol=0, atol=2e-2 if dtype == "bf16" else 1e-5)
+
+
+# ---------------------------------------------------------------------------
+# shapes, edges
+# ---------------------------------------------------------------------------
+EDGE = [
+    # B, H, gridH, gridW, d, ksize
+    (1, 1, 1, 1, 32, 3), (1, 1, 1, 1, 16, 7), (1, 2, 4, 4, 32, 5), (2, 1, 2, 2, 64, 7), (1, 3, 3, 17, 32, 3),
+    (1, 1, 13, 5, 64, 3), (3, 2, 8, 8, 16, 1), (1, 1, 33, 31, 64, 3), (2, 2, 5, 13, 48, 5), (1, 2, 7, 9, 80, 3),
+    (1, 1, 6, 11, 96, 3), (1, 2, 10, 3, 112, 3), (1, 1, 12, 12, 128, 3), (1, 1, 65, 63, 32, 5), (1, 1, 40, 52, 64, 7),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", EDGE, ids=lambda s: "x".join(map(str, s)))
+def test_edge_shapes(shape, dtype):
+    c = workloads.custom_call(*shape, dtype, seed=300 + sum(shape))
+    check(c)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_no_bias(dtype):
+    c = workloads.custom_call(2, 2, 6, 7, 32, 3, dtype, seed=310)
+    check(c, bias=False)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_zero_rows(dtype):
+    """A zero query or key row has cosine 0 with everything (eps floor), never NaN."""
+    c = workloads.custom_call(1, 2, 5, 5, 32, 3, dtype, seed=311)
+    c.q[0, 0, 3] = 0
+    c.k[0, 1, 7] = 0
+    c.k[0, 0, 0] = 0
+    check(c)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_scale_invariance_large_dynamic_range(dtype):
+    """Per-token scales over several orders of magnitude leave the result unchanged."""
+    c = workloads.custom_call(1, 2, 8, 8, 64, 3, dtype, seed=312, qk_lognormal_sigma=3.0)
+    check(c)
+
+
+def test_many_heads_small_grid():
+    c = workloads.custom_call(32, 12, 4, 4, 32, 3, "bf16", seed=313)
+    check(c)
+
+
+def test_split_state_path_fp32():
+    """N large enough that the state kernel splits the token range (partials + reduce)."""
+    c = workloads.custom_call(1, 2, 48, 50, 32, 3, "f32", seed=314)
+    check(c)
+    c = workloads.custom_call(1, 1, 70, 77, 64, 5, "f32", seed=315)
+    check(c)
