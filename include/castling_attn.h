@@ -153,6 +153,21 @@ CASTLING_API int castling_attn_last_path(const castling_attn_t* handle, int* ker
  */
 CASTLING_API int castling_attn_device_status(castling_attn_t* handle, void* stream, unsigned int* raw);
 
+/*
+ * castling_attn_set_profiling: with enable != 0 every later forward on this handle records a
+ * CUDA event on its stream before its first kernel and after each kernel.  Off by default;
+ * the events add a little latency between kernels, so time whole forwards with it off.
+ */
+CASTLING_API int castling_attn_set_profiling(castling_attn_t* handle, int enable);
+
+/*
+ * castling_attn_kernel_times: per-kernel durations of the handle's most recent forward.
+ * Waits for that forward to finish, writes up to `capacity` durations in milliseconds to
+ * ms[] (host) and, if names is not NULL, static kernel-name strings to names[]; returns the
+ * number written (0 when profiling is off), or a negative error code.
+ */
+CASTLING_API int castling_attn_kernel_times(castling_attn_t* handle, float* ms, const char** names, int capacity);
+
 #ifdef __cplusplus
 }
 #endif

@@ -2,9 +2,18 @@
 
 The computation lives in the CUDA library built from ``csrc/``; ``binding`` marshals
 arguments to its C ABI and ``CastlingAttn`` is a small convenience wrapper over torch
-tensors.  Nothing here computes on the CPU.
+tensors.  Nothing here computes on the CPU.  The library is loaded on first use of
+``binding`` or ``CastlingAttn`` (so that ``python -m paper_2211_10526_b200.build`` can
+run before it exists) and loading raises if it has not been built.
 """
-from . import binding
-from .attn import CastlingAttn
+import importlib
 
-__all__ = ["binding", "CastlingAttn"]
+__all__ = ["binding", "CastlingAttn", "build"]
+
+
+def __getattr__(name):
+    if name == "CastlingAttn":
+        return importlib.import_module(".attn", __name__).CastlingAttn
+    if name in ("binding", "build", "attn"):
+        return importlib.import_module("." + name, __name__)
+    raise AttributeError(f"module {__name__!r} has no attribute {name!r}")

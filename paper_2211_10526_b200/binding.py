@@ -55,6 +55,10 @@ def _load() -> ctypes.CDLL:
     lib.castling_attn_last_path.argtypes = [vp, ctypes.POINTER(i)]
     lib.castling_attn_device_status.restype = i
     lib.castling_attn_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint)]
+    lib.castling_attn_set_profiling.restype = i
+    lib.castling_attn_set_profiling.argtypes = [vp, i]
+    lib.castling_attn_kernel_times.restype = i
+    lib.castling_attn_kernel_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_char_p), i]
     return lib
 
 
@@ -112,3 +116,18 @@ def castling_attn_device_status(handle, stream: int = 0):
     raw = ctypes.c_uint(0)
     rc = lib.castling_attn_device_status(handle, stream or None, ctypes.byref(raw))
     return rc, raw.value
+
+
+def castling_attn_set_profiling(handle, enable: bool) -> int:
+    return lib.castling_attn_set_profiling(handle, 1 if enable else 0)
+
+
+def castling_attn_kernel_times(handle):
+    """[(kernel name, milliseconds)] of the handle's most recent forward (empty when profiling is off)."""
+    cap = 8
+    ms = (ctypes.c_float * cap)()
+    names = (ctypes.c_char_p * cap)()
+    n = lib.castling_attn_kernel_times(handle, ms, names, cap)
+    if n < 0:
+        raise CastlingError(n, "castling_attn_kernel_times")
+    return [(names[i].decode(), float(ms[i])) for i in range(n)]

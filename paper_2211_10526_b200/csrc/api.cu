@@ -18,6 +18,7 @@ struct castling_attn {
     int last_cuda_error = 0;
     int last_path = 0;
     int last_launches = 0;
+    castling::KernelTimer timer;
 };
 
 namespace {
@@ -102,6 +103,8 @@ int castling_attn_destroy(castling_attn_t* h) {
     if (!h) return CASTLING_OK;
     if (h->ws) cudaFree(h->ws);
     if (h->stage) cudaFree(h->stage);
+    for (auto& e : h->timer.ev)
+        if (e) cudaEventDestroy(e);
     delete h;
     return CASTLING_OK;
 }
@@ -147,7 +150,8 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     float* partial = state + (size_t)p.BH * castling::state_words(p.d);
     const int P = castling::simt_choose_splits(p.BH, p.N);
     int launches = 0;
-    const cudaError_t e = castling::simt_forward(p, state, partial, P, stream, &launches);
+    h->timer.begin(stream);
+    const cudaError_t e = castling::simt_forward(p, state, partial, P, stream, &launches, &h->timer);
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->last_path = CASTLING_PATH_SIMT;
     h->last_launches = launches;
@@ -244,6 +248,27 @@ int castling_attn_device_status(castling_attn_t* h, void* stream, unsigned int* 
     }
     if (raw) *raw = word;
     return word ? CASTLING_ERR_DEVICE : CASTLING_OK;
+}
+
+int castling_attn_set_profiling(castling_attn_t* h, int enable) {
+    if (!h) return CASTLING_ERR_INVALID_ARG;
+    h->timer.on = enable != 0;
+    h->timer.n = 0;
+    return CASTLING_OK;
+}
+
+int castling_attn_kernel_times(castling_attn_t* h, float* ms, const char** names, int capacity) {
+    if (!h || capacity < 0 || (capacity > 0 && !ms)) return CASTLING_ERR_INVALID_ARG;
+    if (!h->timer.on || h->timer.n == 0) return 0;
+    cudaError_t e = cudaEventSynchronize(h->timer.ev[h->timer.n]);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    const int n = h->timer.n < capacity ? h->timer.n : capacity;
+    for (int i = 0; i < n; ++i) {
+        e = cudaEventElapsedTime(&ms[i], h->timer.ev[i], h->timer.ev[i + 1]);
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        if (names) names[i] = h->timer.name[i];
+    }
+    return n;
 }
 
 }  // extern "C"

@@ -34,9 +34,30 @@ constexpr size_t kHeaderWords = 64;
 
 inline size_t state_words(int d) { return (size_t)d * d + d; }
 
+// Optional per-kernel timing: when `on`, an event is recorded on the stream before the first
+// kernel of a forward and after every kernel, so the host can read each kernel's duration.
+struct KernelTimer {
+    static constexpr int kMax = 8;
+    bool on = false;
+    int n = 0;                       // kernels recorded by the most recent forward
+    cudaEvent_t ev[kMax + 1] = {};   // created lazily
+    const char* name[kMax] = {};
+    void begin(cudaStream_t st) {
+        n = 0;
+        if (!on) return;
+        if (!ev[0]) for (auto& e : ev) cudaEventCreate(&e);
+        cudaEventRecord(ev[0], st);
+    }
+    void mark(cudaStream_t st, const char* kernel_name) {
+        if (!on || n >= kMax) return;
+        name[n] = kernel_name;
+        cudaEventRecord(ev[++n], st);
+    }
+};
+
 // CUDA-core path.  simt_forward returns the cudaError_t of its launches.
 cudaError_t simt_forward(const Problem& p, float* ws_state, float* ws_partial, int P,
-                         cudaStream_t stream, int* launches);
+                         cudaStream_t stream, int* launches, KernelTimer* timer);
 int simt_choose_splits(int BH, int N);
 bool simt_supports(int d, int ksize);
 

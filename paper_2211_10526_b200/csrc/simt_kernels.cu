@@ -259,7 +259,7 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
 
 template <typename T, int D>
 cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, int P,
-                        cudaStream_t stream, int* launches) {
+                        cudaStream_t stream, int* launches, KernelTimer* timer) {
     const int tiles = (p.N + kStateTile - 1) / kStateTile;
     const int chunk = ((tiles + P - 1) / P) * kStateTile;
     float* dst = (P > 1) ? ws_partial : ws_state;
@@ -268,11 +268,13 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     *launches = 1;
+    timer->mark(stream, "simt_state");
     if (P > 1) {
         simt_reduce_kernel<<<p.BH, kThreads, 0, stream>>>(ws_partial, ws_state, D * D + D, P);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         ++*launches;
+        timer->mark(stream, "simt_reduce");
     }
     const size_t smem = simt_apply_smem<D>(p.ksize);
     e = cudaFuncSetAttribute(simt_apply_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -283,12 +285,15 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
         static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.gridH, p.gridW, p.ksize, p.eps2);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
+    timer->mark(stream, "simt_apply");
     return e;
 }
 
 template <int D>
-cudaError_t launch_simt_dtype(const Problem& p, float* s, float* part, int P, cudaStream_t st, int* n) {
-    return p.bf16 ? launch_simt<__nv_bfloat16, D>(p, s, part, P, st, n) : launch_simt<float, D>(p, s, part, P, st, n);
+cudaError_t launch_simt_dtype(const Problem& p, float* s, float* part, int P, cudaStream_t st, int* n,
+                              KernelTimer* t) {
+    return p.bf16 ? launch_simt<__nv_bfloat16, D>(p, s, part, P, st, n, t)
+                  : launch_simt<float, D>(p, s, part, P, st, n, t);
 }
 
 }  // namespace
@@ -309,17 +314,17 @@ int simt_choose_splits(int BH, int N) {
 }
 
 cudaError_t simt_forward(const Problem& p, float* ws_state, float* ws_partial, int P,
-                         cudaStream_t stream, int* launches) {
+                         cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
     switch (p.d) {
-        case 16: return launch_simt_dtype<16>(p, ws_state, ws_partial, P, stream, launches);
-        case 32: return launch_simt_dtype<32>(p, ws_state, ws_partial, P, stream, launches);
-        case 48: return launch_simt_dtype<48>(p, ws_state, ws_partial, P, stream, launches);
-        case 64: return launch_simt_dtype<64>(p, ws_state, ws_partial, P, stream, launches);
-        case 80: return launch_simt_dtype<80>(p, ws_state, ws_partial, P, stream, launches);
-        case 96: return launch_simt_dtype<96>(p, ws_state, ws_partial, P, stream, launches);
-        case 112: return launch_simt_dtype<112>(p, ws_state, ws_partial, P, stream, launches);
-        case 128: return launch_simt_dtype<128>(p, ws_state, ws_partial, P, stream, launches);
+        case 16: return launch_simt_dtype<16>(p, ws_state, ws_partial, P, stream, launches, timer);
+        case 32: return launch_simt_dtype<32>(p, ws_state, ws_partial, P, stream, launches, timer);
+        case 48: return launch_simt_dtype<48>(p, ws_state, ws_partial, P, stream, launches, timer);
+        case 64: return launch_simt_dtype<64>(p, ws_state, ws_partial, P, stream, launches, timer);
+        case 80: return launch_simt_dtype<80>(p, ws_state, ws_partial, P, stream, launches, timer);
+        case 96: return launch_simt_dtype<96>(p, ws_state, ws_partial, P, stream, launches, timer);
+        case 112: return launch_simt_dtype<112>(p, ws_state, ws_partial, P, stream, launches, timer);
+        case 128: return launch_simt_dtype<128>(p, ws_state, ws_partial, P, stream, launches, timer);
         default: return cudaErrorInvalidValue;
     }
 }
