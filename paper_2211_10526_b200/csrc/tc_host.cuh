@@ -1,0 +1,34 @@
+// Host-side interface of the tensor-core (tcgen05 + TMA) path.
+#pragma once
+
+#include "castling_internal.cuh"
+#include <cuda.h>
+
+namespace castling {
+namespace tc {
+
+bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+                          const uint32_t* box, bool swizzle128);
+
+// True when the tensor-core kernels can take this problem (bf16, d = 64, 3x3 or 5x5 filters).
+bool supports(const Problem& p);
+
+// Token splits of the tensor-core state kernel and the workspace words it needs beyond the state.
+int choose_splits(int BH, int N);
+
+// Enqueue state build, split reduction and apply for one problem.  `status` is the device status
+// word.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
+// be built.
+cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, int P, unsigned* status,
+                    cudaStream_t stream, int* launches, KernelTimer* timer);
+
+// Launchers of the individual kernels (each in its own file).
+cudaError_t launch_state(const Problem& p, float* dst, int P, int tiles_per_cta, unsigned* status, cudaStream_t st);
+cudaError_t launch_apply(const Problem& p, const float* state, unsigned* status, cudaStream_t st);
+
+}  // namespace tc
+
+// Shared with the CUDA-core path: sums P partial states per (b,h) in index order.
+cudaError_t launch_reduce(const float* partial, float* state, int BH, int words, int P, cudaStream_t st);
+
+}  // namespace castling
