@@ -2,6 +2,7 @@
 // validation, workspace, kernel-family dispatch.  No computation happens here.
 #include "castling_attn.h"
 #include "castling_internal.cuh"
+#include "tc_host.cuh"
 
 #include <new>
 
@@ -27,7 +28,8 @@ size_t elem_bytes(castling_dtype_t t) { return t == CASTLING_F32 ? 4 : 2; }
 
 // header | state [BH] | partial [BH][P] (only when the token range is split)
 size_t workspace_words(int BH, int N, int d) {
-    const int P = castling::simt_choose_splits(BH, N);
+    int P = castling::simt_choose_splits(BH, N);
+    if (d == 64) P = P > castling::tc::choose_splits(BH, N) ? P : castling::tc::choose_splits(BH, N);
     return castling::kHeaderWords + (size_t)BH * castling::state_words(d) * (1 + (P > 1 ? P : 0));
 }
 
@@ -145,15 +147,23 @@ namespace {
 int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     int rc = ensure_workspace(h, p.BH, p.N, p.d);
     if (rc != CASTLING_OK) return rc;
-    if (h->cfg.force_path == CASTLING_PATH_TENSOR) return CASTLING_ERR_UNSUPPORTED;  // not built yet
+    const bool tensor_ok = castling::tc::supports(p);
+    if (h->cfg.force_path == CASTLING_PATH_TENSOR && !tensor_ok) return CASTLING_ERR_UNSUPPORTED;
+    const bool use_tensor = tensor_ok && h->cfg.force_path != CASTLING_PATH_SIMT;
     float* state = h->ws + castling::kHeaderWords;
     float* partial = state + (size_t)p.BH * castling::state_words(p.d);
-    const int P = castling::simt_choose_splits(p.BH, p.N);
     int launches = 0;
     h->timer.begin(stream);
-    const cudaError_t e = castling::simt_forward(p, state, partial, P, stream, &launches, &h->timer);
+    cudaError_t e;
+    if (use_tensor) {
+        e = castling::tc::forward(p, state, partial, castling::tc::choose_splits(p.BH, p.N),
+                                  reinterpret_cast<unsigned*>(h->ws), stream, &launches, &h->timer);
+    } else {
+        e = castling::simt_forward(p, state, partial, castling::simt_choose_splits(p.BH, p.N), stream, &launches,
+                                   &h->timer);
+    }
     if (e != cudaSuccess) return fail_cuda(h, e);
-    h->last_path = CASTLING_PATH_SIMT;
+    h->last_path = use_tensor ? CASTLING_PATH_TENSOR : CASTLING_PATH_SIMT;
     h->last_launches = launches;
     return CASTLING_OK;
 }

@@ -8,6 +8,7 @@
 //   reduce kernel : sums the token splits in a fixed order (only when P > 1)
 //   apply kernel  : out_t = (1/pi) q^_t S + 1/2 s + bias + DWConv(V)_t    (Eq. 9)
 #include "castling_internal.cuh"
+#include "tc_host.cuh"
 
 namespace castling {
 namespace {
@@ -297,6 +298,11 @@ cudaError_t launch_simt_dtype(const Problem& p, float* s, float* part, int P, cu
 }
 
 }  // namespace
+
+cudaError_t launch_reduce(const float* partial, float* state, int BH, int words, int P, cudaStream_t st) {
+    simt_reduce_kernel<<<BH, kThreads, 0, st>>>(partial, state, words, P);
+    return cudaGetLastError();
+}
 
 bool simt_supports(int d, int ksize) {
     return d >= 16 && d <= 128 && d % 16 == 0 && ksize >= 1 && ksize <= 7 && (ksize & 1);

@@ -1,0 +1,324 @@
+// Apply kernel of the tensor-core path (bf16, d = 64):
+//     out_t = (1/pi) q^_t S + 1/2 s + bias + DWConv(V)_t                         (Eq. 9)
+// Persistent CTAs walk a contiguous range of 8 x 16-token patches of the token grid.  Per patch
+//   warp 0      TMA: the raw Q patch (128 rows of 128 B, 128-byte swizzle) and the V patch with
+//               its halo; out-of-grid rows and columns are zero-filled by TMA, which is exactly
+//               the convolution's zero padding
+//   warp 1      one thread issues four UMMAs: acc[128 x 64] = Q[128 x 64] * S'[64 x 64] into TMEM,
+//               S' = S / pi in bf16; the row scale 1/||q|| commutes and is applied afterwards
+//   warps 6..9  depthwise convolution on CUDA cores, one lane per channel pair, filters in
+//               registers, sliding window along x, packed fp32x2 FMAs, result (+ 1/2 s + bias)
+//               staged in shared memory as fp32
+//   warps 2..5  one thread per token: ||q|| from the Q patch, accumulator row from TMEM,
+//               out = acc / max(||q||, eps) + staged, one rounding to bf16, patch written to
+//               shared memory and stored with TMA (clipped at the grid edge)
+#include "tc_common.cuh"
+#include "tc_host.cuh"
+
+namespace castling {
+namespace tc {
+namespace {
+
+constexpr int kD = 64;
+constexpr int kTY = 8, kTX = 16;            // patch: 8 rows x 16 columns = 128 tokens
+constexpr int kTile = kTY * kTX;
+constexpr int kQBytes = kTile * kD * 2;     // 16 KiB
+constexpr int kStgStride = kD * 4 + 16;     // fp32 row + 16 B pad: conflict-free row-per-thread reads
+constexpr int kStgBytes = kTile * kStgStride;
+constexpr int kThreads = 320;
+constexpr int kTmemCols = 128;              // two 64-column accumulators
+
+template <int KS> struct Geo {
+    static constexpr int R = KS / 2;
+    static constexpr int HY = kTY + 2 * R, HX = kTX + 2 * R;
+    static constexpr int kVBytes = HY * HX * kD * 2;
+    static constexpr int kStage = ((kQBytes + kVBytes + 1023) / 1024) * 1024;
+    static constexpr int kStages = (KS == 3) ? 3 : 2;
+    // S' | out patch | stages | staging x2 | barriers
+    static constexpr int kOffS = 0, kOffOut = 8192, kOffStages = kOffOut + kQBytes;
+    static constexpr int kOffStg = kOffStages + kStages * kStage;
+    static constexpr int kOffBar = kOffStg + 2 * kStgBytes;
+    static constexpr size_t kSmem = 1024 + kOffBar + 256;
+};
+
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+
+struct ApplyParams {
+    const float* state;            // [BH][64*64 + 64] raw sums
+    const __nv_bfloat16* w;        // [H*64][KS][KS]
+    const __nv_bfloat16* bias;     // [H*64] or nullptr
+    int H, bh0, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
+    float eps2;
+    unsigned* status;
+};
+
+template <int KS>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmV,
+                const __grid_constant__ CUtensorMap tmO, const ApplyParams prm) {
+    using G = Geo<KS>;
+    constexpr int NS = G::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* S_s = smem + G::kOffS;
+    uint8_t* out_s = smem + G::kOffOut;
+    uint8_t* stages = smem + G::kOffStages;
+    uint8_t* stg = smem + G::kOffStg;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + G::kOffBar);  // [NS] TMA landed
+    uint64_t* empty = full + NS;                                      // [NS] stage consumed (128 arrivals)
+    uint64_t* acc_full = empty + NS;                                  // [2]  UMMAs retired
+    uint64_t* conv_full = acc_full + 2;                               // [2]  staging written (128 arrivals)
+    uint64_t* buf_free = conv_full + 2;                               // [2]  accumulator + staging read (128)
+    uint64_t* s_ready = buf_free + 2;                                 // S' of the current (b,h) written (128)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_ready + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tiles_per_bh = prm.tilesX * prm.tilesY;
+    // contiguous share of the patches for this CTA
+    const int g_begin = (int)((long long)prm.n_tiles * blockIdx.x / gridDim.x);
+    const int g_end = (int)((long long)prm.n_tiles * (blockIdx.x + 1) / gridDim.x);
+    const int my_tiles = g_end - g_begin;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kTile); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], kTile); mbar_init(&buf_free[b], kTile); }
+        mbar_init(s_ready, kTile);
+        *abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    constexpr unsigned kBit = kStatusApplyTimeout;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int it = 0; it < my_tiles; ++it) {
+                const int s = it % NS, use = it / NS;
+                if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) break;
+                const int g = g_begin + it, bh = g / tiles_per_bh, rem = g % tiles_per_bh;
+                const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
+                uint8_t* qs = stages + s * G::kStage;
+                mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
+                tma_load_4d(qs, &tmQ, &full[s], 0, x0, y0, bh);
+                tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::R, y0 - G::R, bh);
+                ++issued;
+            }
+            if (*abort_flag) {
+                for (int i = max(0, issued - NS); i < issued; ++i)
+                    for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[i % NS], (i / NS) & 1); ++spin) {}
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, kD, false, true);
+            const uint32_t s_addr = smem_u32(S_s);
+            int prev_bh = -1, seg = 0;
+            for (int it = 0; it < my_tiles; ++it) {
+                const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
+                const int bh = (g_begin + it) / tiles_per_bh;
+                if (bh != prev_bh) {
+                    if (!mbar_wait(s_ready, seg & 1, abort_flag, prm.status, kBit)) break;
+                    ++seg; prev_bh = bh;
+                }
+                if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
+                if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
+                tcgen05_fence_after_sync();
+                const uint32_t q_addr = smem_u32(stages + s * G::kStage);
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k) {
+                    const uint64_t a = umma_desc_sw128(q_addr + k * 32, 0, 1024);        // K-major rows of 128 B
+                    const uint64_t bd = umma_desc_sw128(s_addr + k * 2048, 0, 1024);     // N-major, 16 K-rows per step
+                    umma_bf16(tmem + b * kD, a, bd, idesc, k != 0);
+                }
+                umma_commit(&acc_full[b]);
+            }
+        }
+    } else if (warp < 6) {
+        // ---------------- epilogue: one thread per token of the patch ----------------
+        const int quarter = warp & 3, row = quarter * 32 + lane, et = tid - 64;
+        const bool leader = (et == 0);
+        int prev_bh = -1;
+        for (int it = 0; it < my_tiles; ++it) {
+            const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
+            const int g = g_begin + it, bh = g / tiles_per_bh, rem = g % tiles_per_bh;
+            const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
+            if (bh != prev_bh) {
+                // every UMMA that read the previous S' has retired (its acc_full was waited on below)
+                prev_bh = bh;
+                const int i = et >> 1, half = et & 1;
+                const float4* src = reinterpret_cast<const float4*>(prm.state + (size_t)(prm.bh0 + bh) * (kD * kD + kD) + i * kD + half * 32);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float4 lo = __ldg(src + 2 * c), hi = __ldg(src + 2 * c + 1);
+                    uint4 o;
+                    o.x = pack_bf16x2(lo.x * kInvPi, lo.y * kInvPi); o.y = pack_bf16x2(lo.z * kInvPi, lo.w * kInvPi);
+                    o.z = pack_bf16x2(hi.x * kInvPi, hi.y * kInvPi); o.w = pack_bf16x2(hi.z * kInvPi, hi.w * kInvPi);
+                    *reinterpret_cast<uint4*>(S_s + i * 128 + (((half * 4 + c) ^ (i & 7)) << 4)) = o;
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(s_ready);
+            }
+            if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
+            // 1 / max(||q||, eps) of this thread's token
+            const uint8_t* qrow = stages + s * G::kStage + row * 128;
+            float ss = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint4 c = *reinterpret_cast<const uint4*>(qrow + ((j ^ (row & 7)) << 4));
+                const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float lo = bf16lo(w4[e]), hi = bf16hi(w4[e]);
+                    ss = fmaf(lo, lo, ss); ss = fmaf(hi, hi, ss);
+                }
+            }
+            const float rq = 1.0f / sqrtf(fmaxf(ss, prm.eps2));
+            if (!mbar_wait(&acc_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
+            if (!mbar_wait(&conv_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
+            tcgen05_fence_after_sync();
+            if (it > 0) {  // the previous patch's TMA store must have read out_s before it is rewritten
+                if (leader) tma_store_wait_read();
+                named_barrier_sync(1, kTile);
+            }
+            const uint8_t* srow = stg + b * kStgBytes + row * kStgStride;
+            uint8_t* orow = out_s + row * 128;
+#pragma unroll
+            for (int cc = 0; cc < kD / 16; ++cc) {
+                float a[16];
+                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kD + cc * 16, a);
+                tmem_ld_wait();
+                float o[16];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float4 c4 = *reinterpret_cast<const float4*>(srow + cc * 64 + e * 16);
+                    o[4 * e + 0] = fmaf(a[4 * e + 0], rq, c4.x); o[4 * e + 1] = fmaf(a[4 * e + 1], rq, c4.y);
+                    o[4 * e + 2] = fmaf(a[4 * e + 2], rq, c4.z); o[4 * e + 3] = fmaf(a[4 * e + 3], rq, c4.w);
+                }
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    uint4 pk;
+                    pk.x = pack_bf16x2(o[8 * e + 0], o[8 * e + 1]); pk.y = pack_bf16x2(o[8 * e + 2], o[8 * e + 3]);
+                    pk.z = pack_bf16x2(o[8 * e + 4], o[8 * e + 5]); pk.w = pack_bf16x2(o[8 * e + 6], o[8 * e + 7]);
+                    *reinterpret_cast<uint4*>(orow + (((2 * cc + e) ^ (row & 7)) << 4)) = pk;
+                }
+            }
+            tcgen05_fence_before_sync();
+            mbar_arrive(&buf_free[b]);
+            mbar_arrive(&empty[s]);
+            fence_proxy_async_smem();
+            named_barrier_sync(1, kTile);
+            if (leader) {
+                tma_store_4d(&tmO, out_s, 0, x0, y0, bh);
+                tma_store_commit();
+            }
+        }
+        if (leader) tma_store_wait_all();
+    } else {
+        // ---------------- depthwise convolution: lane = channel pair, warp = two patch rows ----------------
+        const int cw = warp - 6;
+        constexpr int R = G::R, ROWS = 2 + 2 * R;
+        float2 wreg[KS][KS];
+        float2 cinit = make_float2(0.f, 0.f);
+        int prev_bh = -1;
+        for (int it = 0; it < my_tiles; ++it) {
+            const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
+            const int bh = (g_begin + it) / tiles_per_bh;
+            if (bh != prev_bh) {
+                prev_bh = bh;
+                const int gbh = prm.bh0 + bh, ch = (gbh % prm.H) * kD + 2 * lane;
+                const float* sv = prm.state + (size_t)gbh * (kD * kD + kD) + kD * kD + 2 * lane;
+                cinit.x = 0.5f * __ldg(sv); cinit.y = 0.5f * __ldg(sv + 1);
+                if (prm.bias) { cinit.x += __bfloat162float(prm.bias[ch]); cinit.y += __bfloat162float(prm.bias[ch + 1]); }
+#pragma unroll
+                for (int dy = 0; dy < KS; ++dy)
+#pragma unroll
+                    for (int dx = 0; dx < KS; ++dx)
+                        wreg[dy][dx] = make_float2(__bfloat162float(prm.w[(size_t)ch * KS * KS + dy * KS + dx]),
+                                                   __bfloat162float(prm.w[(size_t)(ch + 1) * KS * KS + dy * KS + dx]));
+            }
+            if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
+            if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
+            const uint8_t* vh = stages + s * G::kStage + kQBytes + (2 * cw) * G::HX * 128 + lane * 4;
+            uint8_t* so = stg + b * kStgBytes + (2 * cw) * kTX * kStgStride + lane * 8;
+            float2 win[ROWS][KS];  // window columns x .. x+KS-1, rotating
+#pragma unroll
+            for (int dx = 0; dx < KS - 1; ++dx)
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + (r * G::HX + dx) * 128);
+                    win[r][dx] = make_float2(bf16lo(wv), bf16hi(wv));
+                }
+#pragma unroll
+            for (int x = 0; x < kTX; ++x) {
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + (r * G::HX + x + KS - 1) * 128);
+                    win[r][(x + KS - 1) % KS] = make_float2(bf16lo(wv), bf16hi(wv));
+                }
+                float2 a0 = cinit, a1 = cinit;
+#pragma unroll
+                for (int dy = 0; dy < KS; ++dy)
+#pragma unroll
+                    for (int dx = 0; dx < KS; ++dx) {
+                        a0 = ffma2(wreg[dy][dx], win[dy][(x + dx) % KS], a0);
+                        a1 = ffma2(wreg[dy][dx], win[dy + 1][(x + dx) % KS], a1);
+                    }
+                *reinterpret_cast<float2*>(so + x * kStgStride) = a0;
+                *reinterpret_cast<float2*>(so + (kTX + x) * kStgStride) = a1;
+            }
+            mbar_arrive(&conv_full[b]);
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+}
+
+template <int KS>
+cudaError_t launch_apply_ks(const Problem& p, const float* state, unsigned* status, cudaStream_t st) {
+    using G = Geo<KS>;
+    CUtensorMap tmQ, tmV, tmO;
+    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)p.gridW, (uint64_t)p.gridH, (uint64_t)p.BH};
+    const uint32_t box[4] = {kD, kTX, kTY, 1};
+    const uint32_t boxv[4] = {kD, (uint32_t)G::HX, (uint32_t)G::HY, 1};
+    if (!make_tensor_map_bf16(&tmQ, p.q, 4, dims, box, true) || !make_tensor_map_bf16(&tmO, p.out, 4, dims, box, true) ||
+        !make_tensor_map_bf16(&tmV, p.v, 4, dims, boxv, false))
+        return cudaErrorNotSupported;
+    ApplyParams prm;
+    prm.state = state;
+    prm.w = static_cast<const __nv_bfloat16*>(p.w);
+    prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
+    prm.H = p.H; prm.bh0 = 0;
+    prm.tilesX = (p.gridW + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
+    prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
+    prm.eps2 = p.eps2; prm.status = status;
+    cudaError_t e = cudaFuncSetAttribute(tc_apply_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmem);
+    if (e != cudaSuccess) return e;
+    const int grid = prm.n_tiles < 148 ? prm.n_tiles : 148;
+    tc_apply_kernel<KS><<<grid, kThreads, G::kSmem, st>>>(tmQ, tmV, tmO, prm);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_apply(const Problem& p, const float* state, unsigned* status, cudaStream_t st) {
+    return p.ksize == 3 ? launch_apply_ks<3>(p, state, status, st) : launch_apply_ks<5>(p, state, status, st);
+}
+
+}  // namespace tc
+}  // namespace castling

@@ -1,0 +1,50 @@
+// Orchestration of the tensor-core path: state build -> split reduction -> apply, in stream order
+// (the stream is the only synchronisation between the phases; no kernel waits on another).
+#include "tc_host.cuh"
+
+namespace castling {
+namespace tc {
+
+namespace {
+constexpr int kStateTile = 128;  // tokens per UMMA stage of the state kernel
+}
+
+bool supports(const Problem& p) {
+    return p.bf16 && p.d == 64 && (p.ksize == 3 || p.ksize == 5);
+}
+
+// Enough CTAs to cover the 148 SMs once, every split non-empty, at most 64 splits.
+int choose_splits(int BH, int N) {
+    const int tiles = (N + kStateTile - 1) / kStateTile;
+    int P = (148 + BH - 1) / BH;
+    if (P > tiles) P = tiles;
+    if (P > 64) P = 64;
+    if (P < 1) P = 1;
+    const int per = (tiles + P - 1) / P;
+    return (tiles + per - 1) / per;
+}
+
+cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, int P, unsigned* status,
+                    cudaStream_t stream, int* launches, KernelTimer* timer) {
+    *launches = 0;
+    const int tiles = (p.N + kStateTile - 1) / kStateTile;
+    const int per = (tiles + P - 1) / P;
+    cudaError_t e = launch_state(p, P > 1 ? ws_partial : ws_state, P, per, status, stream);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    timer->mark(stream, "tc_state");
+    if (P > 1) {
+        e = launch_reduce(ws_partial, ws_state, p.BH, p.d * p.d + p.d, P, stream);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        timer->mark(stream, "reduce");
+    }
+    e = launch_apply(p, ws_state, status, stream);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    timer->mark(stream, "tc_apply");
+    return cudaSuccess;
+}
+
+}  // namespace tc
+}  // namespace castling

@@ -1,0 +1,195 @@
+// State kernel of the tensor-core path (bf16, d = 64): per (b,h) and token split,
+//     S = sum_n k^_n^T v_n  (64 x 64)   and   s = sum_n v_n  (64)            (Eq. 9)
+// as one tcgen05 contraction over tokens.  Per 128-token stage TMA brings the K and V tiles
+// into 128-byte-swizzled shared memory; four warps scale every K row by 1 / max(||k||, eps) in
+// place (the scale sits on the contracted index, so it cannot wait for an epilogue); one thread
+// issues UMMAs with A = [K^ ; 1 0 0 ...] (128 x tokens, M-major: rows 0..63 are the key
+// features, row 64 is all ones, which makes row 64 of the accumulator the token sum of V) and
+// B = V (tokens x 64, N-major).  The fp32 accumulator lives in TMEM for the CTA's whole token
+// range and is written once, as this split's partial state.
+#include "tc_common.cuh"
+#include "tc_host.cuh"
+
+namespace castling {
+namespace tc {
+namespace {
+
+constexpr int kD = 64;
+constexpr int kTile = 128;                   // tokens per stage
+constexpr int kStages = 4;
+constexpr int kTileBytes = kTile * kD * 2;   // 16 KiB per operand tile
+constexpr int kStageBytes = 2 * kTileBytes;  // K then V
+constexpr int kOnesBytes = 2048;             // 16 token rows x 128 B: feature 64 = 1, 65..127 = 0
+constexpr int kThreads = 192;                // warp 0 TMA, warp 1 UMMA, warps 2..5 scale + epilogue
+constexpr int kTmemCols = 64;
+constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                float* __restrict__ dst, int N, int tiles_per_cta, int P, float eps2, unsigned* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* ones = smem + kStages * kStageBytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(ones + kOnesBytes);  // TMA bytes landed
+    uint64_t* scaled = full + kStages;                                // K rows normalised (128 arrivals)
+    uint64_t* empty = scaled + kStages;                               // UMMAs of the stage retired
+    uint64_t* accum = empty + kStages;                                // whole accumulation retired
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int p = blockIdx.x % P, bh = blockIdx.x / P;
+    const int total_tiles = (N + kTile - 1) / kTile;
+    const int t_begin = p * tiles_per_cta;
+    const int n_tiles = min(total_tiles, t_begin + tiles_per_cta) - t_begin;
+    float* out = dst + ((size_t)bh * P + p) * (kD * kD + kD);
+    if (n_tiles <= 0) {  // the host never makes such a split; keep the partial well defined anyway
+        for (int i = tid; i < kD * kD + kD; i += kThreads) out[i] = 0.f;
+        return;
+    }
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&scaled[s], kTile);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(accum, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp >= 2) {
+        // constant block of A: for each of 16 token rows, element 64 (first of the second 64-wide
+        // block along M) is 1.0 and the rest 0; 16-byte chunk c of row r sits at chunk c ^ (r & 7)
+        const int t = tid - 64;  // 0..127 -> one 16-byte chunk each
+        const int r = t >> 3, c = t & 7;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if ((c ^ (r & 7)) == 0) val.x = 0x3f80u;  // logical chunk 0: bf16 1.0 in its first element
+        *reinterpret_cast<uint4*>(ones + r * 128 + c * 16) = val;
+        fence_proxy_async_smem();
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int it = 0; it < n_tiles; ++it) {
+                const int s = it % kStages, use = it / kStages;
+                if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, status, kStatusStateTimeout)) break;
+                uint8_t* ks = smem + s * kStageBytes;
+                mbar_expect_tx(&full[s], kStageBytes);
+                tma_load_3d(ks, &tmK, &full[s], 0, (t_begin + it) * kTile, bh);
+                tma_load_3d(ks + kTileBytes, &tmV, &full[s], 0, (t_begin + it) * kTile, bh);
+                ++issued;
+            }
+            if (*abort_flag) {
+                // giving up: let copies already in flight land before the CTA's shared memory goes away
+                for (int i = max(0, issued - kStages); i < issued; ++i)
+                    for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[i % kStages], (i / kStages) & 1); ++spin) {}
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, kD, true, true);
+            const uint32_t ones_addr = smem_u32(ones);
+            bool ok = true;
+            for (int it = 0; it < n_tiles && ok; ++it) {
+                const int s = it % kStages, use = it / kStages;
+                ok = mbar_wait(&scaled[s], use & 1, abort_flag, status, kStatusStateTimeout);
+                if (!ok) break;
+                tcgen05_fence_after_sync();
+                const uint32_t ka = smem_u32(smem + s * kStageBytes), va = ka + kTileBytes;
+#pragma unroll
+                for (int j = 0; j < kTile / 16; ++j) {  // one UMMA per 16 tokens (K = 16)
+                    const uint32_t a0 = ka + j * 2048, b0 = va + j * 2048;
+                    const uint64_t a = umma_desc_sw128(a0, ones_addr - a0, 1024);
+                    const uint64_t b = umma_desc_sw128(b0, 0, 1024);
+                    umma_bf16(tmem, a, b, idesc, (it | j) != 0);
+                }
+                umma_commit(&empty[s]);
+            }
+            if (ok) umma_commit(accum);
+        }
+    } else {
+        const int t = tid - 64;  // token row of the stage handled by this thread
+        bool ok = true;
+        for (int it = 0; it < n_tiles; ++it) {
+            const int s = it % kStages, use = it / kStages;
+            ok = mbar_wait(&full[s], use & 1, abort_flag, status, kStatusStateTimeout);
+            if (!ok) break;
+            uint8_t* row = smem + s * kStageBytes + t * 128;
+            uint4 c[8];
+            float ss = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                c[j] = *reinterpret_cast<const uint4*>(row + ((j ^ (t & 7)) << 4));
+                const uint32_t w[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float lo = bf16lo(w[e]), hi = bf16hi(w[e]);
+                    ss = fmaf(lo, lo, ss);
+                    ss = fmaf(hi, hi, ss);
+                }
+            }
+            const float rk = 1.0f / sqrtf(fmaxf(ss, eps2));
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint4 o;
+                o.x = pack_bf16x2(bf16lo(c[j].x) * rk, bf16hi(c[j].x) * rk);
+                o.y = pack_bf16x2(bf16lo(c[j].y) * rk, bf16hi(c[j].y) * rk);
+                o.z = pack_bf16x2(bf16lo(c[j].z) * rk, bf16hi(c[j].z) * rk);
+                o.w = pack_bf16x2(bf16lo(c[j].w) * rk, bf16hi(c[j].w) * rk);
+                *reinterpret_cast<uint4*>(row + ((j ^ (t & 7)) << 4)) = o;
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&scaled[s]);
+        }
+        // epilogue: accumulator rows 0..63 are S, row 64 is s; a warp reads TMEM lanes 32*(warp%4)..+31
+        const int quarter = warp & 3;
+        if (ok && quarter < 3) {
+            ok = mbar_wait(accum, 0, abort_flag, status, kStatusStateTimeout);
+            if (ok) {
+                tcgen05_fence_after_sync();
+                const int row = quarter * 32 + lane;
+#pragma unroll
+                for (int cc = 0; cc < kD / 16; ++cc) {
+                    float v[16];
+                    tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + cc * 16, v);
+                    tmem_ld_wait();
+                    if (row <= kD) {
+                        float4* o4 = reinterpret_cast<float4*>(out + row * kD + cc * 16);  // row 64 lands on s
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o4[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                    }
+                }
+            }
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace
+
+cudaError_t launch_state(const Problem& p, float* dst, int P, int tiles_per_cta, unsigned* status, cudaStream_t st) {
+    CUtensorMap tmK, tmV;
+    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)p.N, (uint64_t)p.BH};
+    const uint32_t box[3] = {kD, kTile, 1};
+    if (!make_tensor_map_bf16(&tmK, p.k, 3, dims, box, true) || !make_tensor_map_bf16(&tmV, p.v, 3, dims, box, true))
+        return cudaErrorNotSupported;
+    cudaError_t e = cudaFuncSetAttribute(tc_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    tc_state_kernel<<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(tmK, tmV, dst, p.N, tiles_per_cta, P, p.eps2,
+                                                                        status);
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+}  // namespace castling

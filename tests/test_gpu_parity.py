@@ -186,3 +186,70 @@ def test_split_state_path_fp32():
     check(c)
     c = workloads.custom_call(1, 1, 70, 77, 64, 5, "f32", seed=315)
     check(c)
+
+
+# ---------------------------------------------------------------------------
+# kernel families: the tensor-core path must be the one that runs where it applies
+# ---------------------------------------------------------------------------
+TENSOR_SHAPES = [(2, 8, 32, 32, 64, 3), (1, 2, 8, 16, 64, 3), (1, 1, 1, 1, 64, 3), (2, 3, 14, 14, 64, 3),
+                 (1, 2, 37, 53, 64, 3), (1, 2, 24, 40, 64, 5), (1, 1, 3, 130, 64, 3), (1, 1, 200, 5, 64, 5),
+                 (3, 5, 64, 64, 64, 3)]
+
+
+@pytest.mark.parametrize("shape", TENSOR_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_tensor_path_parity(shape):
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    c = workloads.custom_call(*shape, "bf16", seed=500 + sum(shape))
+    ref = run_oracle(c)
+    s = c.shape
+    dev = torch.device("cuda:0")
+    args = [t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)]
+    errs = {}
+    for path in (binding.PATH_TENSOR, binding.PATH_SIMT, binding.PATH_AUTO):
+        with CastlingAttn(ksize=s.ksize, force_path=path) as attn:
+            out = attn.forward(*args, s.gridH, s.gridW)
+            torch.cuda.synchronize()
+            assert attn.device_status() == (0, 0)
+            used, launches = attn.last_path()
+        if path != binding.PATH_AUTO:
+            assert used == path
+        else:
+            assert used == binding.PATH_TENSOR, "bf16, d = 64 must run on the tensor-core kernels by default"
+        errs[path] = rel_err(out, ref)
+    assert max(errs.values()) <= TOL["bf16"], errs
+
+
+def test_tensor_path_term_isolation():
+    """Each term of Eq. 9 alone, on the tensor-core kernels."""
+    from paper_2211_10526_b200 import binding
+    base = lambda seed: workloads.custom_call(2, 2, 24, 20, 64, 3, "bf16", seed=seed)
+    # linear term alone
+    c = base(601)
+    v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+    c.dw_weight.zero_(); c.dw_bias.zero_()
+    check(c, force_path=binding.PATH_TENSOR)
+    # 1/2 sum alone (plus its linear companion)
+    c = base(602)
+    c.v[:] = c.v[:, :, :1, :].clone()
+    c.dw_weight.zero_(); c.dw_bias.zero_()
+    check(c, force_path=binding.PATH_TENSOR)
+    # convolution alone
+    c = base(603)
+    v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+    c.dw_weight = (c.dw_weight.float() * 30).to(torch.bfloat16)
+    c.k.zero_()
+    check(c, force_path=binding.PATH_TENSOR)
+    # zero rows
+    c = base(604)
+    c.q[0, 0, 5] = 0; c.k[1, 1, 17] = 0
+    check(c, force_path=binding.PATH_TENSOR)
+
+
+def test_tensor_path_rejects_what_it_cannot_take():
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    c = workloads.custom_call(1, 1, 4, 4, 32, 3, "f32", seed=605)
+    dev = torch.device("cuda:0")
+    with CastlingAttn(ksize=3, force_path=binding.PATH_TENSOR) as attn:
+        with pytest.raises(binding.CastlingError) as ei:
+            attn.forward(*[t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)], 4, 4)
+        assert ei.value.code == binding.ERR_UNSUPPORTED
