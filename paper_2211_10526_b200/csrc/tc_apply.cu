@@ -53,7 +53,8 @@ __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
 }
 
 struct ApplyParams {
-    const float* state;            // [BH][64*64 + 64] raw sums
+    const float* state;            // [BH][P][64*64 + 64] raw sums of the P token splits
+    int P;
     const __nv_bfloat16* w;        // [H*64][KS][KS]
     const __nv_bfloat16* bias;     // [H*64] or nullptr
     int H, bh0, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
@@ -161,10 +162,16 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 // every UMMA that read the previous S' has retired (its acc_full was waited on below)
                 prev_bh = bh;
                 const int i = et >> 1, half = et & 1;
-                const float4* src = reinterpret_cast<const float4*>(prm.state + (size_t)(prm.bh0 + bh) * (kD * kD + kD) + i * kD + half * 32);
+                const float4* src = reinterpret_cast<const float4*>(prm.state + (size_t)(prm.bh0 + bh) * prm.P * (kD * kD + kD) + i * kD + half * 32);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const float4 lo = __ldg(src + 2 * c), hi = __ldg(src + 2 * c + 1);
+                    float4 lo = __ldg(src + 2 * c), hi = __ldg(src + 2 * c + 1);
+                    for (int pp = 1; pp < prm.P; ++pp) {  // fixed order: bitwise reproducible
+                        const float4 l2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c);
+                        const float4 h2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c + 1);
+                        lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
+                        hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
+                    }
                     uint4 o;
                     o.x = pack_bf16x2(lo.x * kInvPi, lo.y * kInvPi); o.y = pack_bf16x2(lo.z * kInvPi, lo.w * kInvPi);
                     o.z = pack_bf16x2(hi.x * kInvPi, hi.y * kInvPi); o.w = pack_bf16x2(hi.z * kInvPi, hi.w * kInvPi);
@@ -241,8 +248,13 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (bh != prev_bh) {
                 prev_bh = bh;
                 const int gbh = prm.bh0 + bh, ch = (gbh % prm.H) * kD + 2 * lane;
-                const float* sv = prm.state + (size_t)gbh * (kD * kD + kD) + kD * kD + 2 * lane;
-                cinit.x = 0.5f * __ldg(sv); cinit.y = 0.5f * __ldg(sv + 1);
+                const float* sv = prm.state + (size_t)gbh * prm.P * (kD * kD + kD) + kD * kD + 2 * lane;
+                float s0 = __ldg(sv), s1 = __ldg(sv + 1);
+                for (int pp = 1; pp < prm.P; ++pp) {
+                    s0 += __ldg(sv + pp * (kD * kD + kD));
+                    s1 += __ldg(sv + pp * (kD * kD + kD) + 1);
+                }
+                cinit.x = 0.5f * s0; cinit.y = 0.5f * s1;
                 if (prm.bias) { cinit.x += __bfloat162float(prm.bias[ch]); cinit.y += __bfloat162float(prm.bias[ch + 1]); }
 #pragma unroll
                 for (int dy = 0; dy < KS; ++dy)
@@ -290,7 +302,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 }
 
 template <int KS>
-cudaError_t launch_apply_ks(const Problem& p, const float* state, unsigned* status, cudaStream_t st) {
+cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigned* status, cudaStream_t st) {
     using G = Geo<KS>;
     CUtensorMap tmQ, tmV, tmO;
     const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)p.gridW, (uint64_t)p.gridH, (uint64_t)p.BH};
@@ -301,6 +313,7 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, unsigned* stat
         return cudaErrorNotSupported;
     ApplyParams prm;
     prm.state = state;
+    prm.P = P;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.H = p.H; prm.bh0 = 0;
@@ -316,8 +329,8 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, unsigned* stat
 
 }  // namespace
 
-cudaError_t launch_apply(const Problem& p, const float* state, unsigned* status, cudaStream_t st) {
-    return p.ksize == 3 ? launch_apply_ks<3>(p, state, status, st) : launch_apply_ks<5>(p, state, status, st);
+cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st) {
+    return p.ksize == 3 ? launch_apply_ks<3>(p, partial, P, status, st) : launch_apply_ks<5>(p, partial, P, status, st);
 }
 
 }  // namespace tc

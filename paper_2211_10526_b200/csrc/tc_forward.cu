@@ -13,10 +13,11 @@ bool supports(const Problem& p) {
     return p.bf16 && p.d == 64 && (p.ksize == 3 || p.ksize == 5);
 }
 
-// Enough CTAs to cover the 148 SMs once, every split non-empty, at most 64 splits.
+// Two state CTAs fit on an SM: as many splits as keep all CTAs of the launch resident at once
+// (2 x 148), every split non-empty, at most 64 splits.
 int choose_splits(int BH, int N) {
     const int tiles = (N + kStateTile - 1) / kStateTile;
-    int P = (148 + BH - 1) / BH;
+    int P = (2 * 148) / BH;
     if (P > tiles) P = tiles;
     if (P > 64) P = 64;
     if (P < 1) P = 1;
@@ -29,17 +30,14 @@ cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, int P,
     *launches = 0;
     const int tiles = (p.N + kStateTile - 1) / kStateTile;
     const int per = (tiles + P - 1) / P;
-    cudaError_t e = launch_state(p, P > 1 ? ws_partial : ws_state, P, per, status, stream);
+    // the splits' partial states [BH][P][d*d + d] start at the state area; the apply kernel sums
+    // them in index order while it converts S to its bf16 operand
+    (void)ws_partial;
+    cudaError_t e = launch_state(p, ws_state, P, per, status, stream);
     if (e != cudaSuccess) return e;
     ++*launches;
     timer->mark(stream, "tc_state");
-    if (P > 1) {
-        e = launch_reduce(ws_partial, ws_state, p.BH, p.d * p.d + p.d, P, stream);
-        if (e != cudaSuccess) return e;
-        ++*launches;
-        timer->mark(stream, "reduce");
-    }
-    e = launch_apply(p, ws_state, status, stream);
+    e = launch_apply(p, ws_state, P, status, stream);
     if (e != cudaSuccess) return e;
     ++*launches;
     timer->mark(stream, "tc_apply");

@@ -24,7 +24,7 @@ cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, int P,
 
 // Launchers of the individual kernels (each in its own file).
 cudaError_t launch_state(const Problem& p, float* dst, int P, int tiles_per_cta, unsigned* status, cudaStream_t st);
-cudaError_t launch_apply(const Problem& p, const float* state, unsigned* status, cudaStream_t st);
+cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st);
 
 }  // namespace tc
 

@@ -16,7 +16,7 @@ namespace {
 
 constexpr int kD = 64;
 constexpr int kTile = 128;                   // tokens per stage
-constexpr int kStages = 4;
+constexpr int kStages = 3;                  // 3 x 32 KiB: two CTAs fit on one SM
 constexpr int kTileBytes = kTile * kD * 2;   // 16 KiB per operand tile
 constexpr int kStageBytes = 2 * kTileBytes;  // K then V
 constexpr int kOnesBytes = 2048;             // 16 token rows x 128 B: feature 64 = 1, 65..127 = 0
@@ -24,7 +24,7 @@ constexpr int kThreads = 192;                // warp 0 TMA, warp 1 UMMA, warps 2
 constexpr int kTmemCols = 64;
 constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 float* __restrict__ dst, int N, int tiles_per_cta, int P, float eps2, unsigned* status) {
     extern __shared__ uint8_t smem_raw[];
