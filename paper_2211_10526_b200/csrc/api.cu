@@ -14,6 +14,8 @@ struct castling_attn {
     int sm_count = 0;
     float* ws = nullptr;        // header | state | partial
     size_t ws_bytes = 0;
+    unsigned* counters = nullptr;  // one arrival counter per (b,h), zero between calls
+    size_t counters_cap = 0;
     char* stage = nullptr;      // device staging for castling_attn_forward_host
     size_t stage_bytes = 0;
     int last_cuda_error = 0;
@@ -72,6 +74,22 @@ int ensure_workspace(castling_attn* h, int BH, int N, int d) {
     return CASTLING_OK;
 }
 
+int ensure_counters(castling_attn* h, int BH) {
+    if ((size_t)BH <= h->counters_cap) return CASTLING_OK;
+    size_t cap = 1024;
+    while (cap < (size_t)BH) cap *= 2;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    if (h->counters) cudaFree(h->counters);
+    h->counters = nullptr; h->counters_cap = 0;
+    e = cudaMalloc((void**)&h->counters, cap * sizeof(unsigned));
+    if (e != cudaSuccess) return fail_cuda(h, e, CASTLING_ERR_OOM);
+    e = cudaMemset(h->counters, 0, cap * sizeof(unsigned));
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->counters_cap = cap;
+    return CASTLING_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -105,6 +123,7 @@ int castling_attn_destroy(castling_attn_t* h) {
     if (!h) return CASTLING_OK;
     if (h->ws) cudaFree(h->ws);
     if (h->stage) cudaFree(h->stage);
+    if (h->counters) cudaFree(h->counters);
     for (auto& e : h->timer.ev)
         if (e) cudaEventDestroy(e);
     delete h;
@@ -156,7 +175,9 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     h->timer.begin(stream);
     cudaError_t e;
     if (use_tensor) {
-        e = castling::tc::forward(p, state, partial, castling::tc::choose_splits(p.BH, p.N),
+        rc = ensure_counters(h, p.BH);
+        if (rc != CASTLING_OK) return rc;
+        e = castling::tc::forward(p, state, partial, h->counters, castling::tc::choose_splits(p.BH, p.N),
                                   reinterpret_cast<unsigned*>(h->ws), stream, &launches, &h->timer);
     } else {
         e = castling::simt_forward(p, state, partial, castling::simt_choose_splits(p.BH, p.N), stream, &launches,
@@ -257,6 +278,8 @@ int castling_attn_device_status(castling_attn_t* h, void* stream, unsigned int* 
         if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(h, e);
     }
     if (raw) *raw = word;
+    if (word && h->counters)  // a kernel that gave up may have left arrival counters half way
+        cudaMemset(h->counters, 0, h->counters_cap * sizeof(unsigned));
     return word ? CASTLING_ERR_DEVICE : CASTLING_OK;
 }
 

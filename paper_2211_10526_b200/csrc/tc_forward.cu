@@ -25,19 +25,16 @@ int choose_splits(int BH, int N) {
     return (tiles + per - 1) / per;
 }
 
-cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, int P, unsigned* status,
-                    cudaStream_t stream, int* launches, KernelTimer* timer) {
+cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsigned* counters, int P,
+                    unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
     const int tiles = (p.N + kStateTile - 1) / kStateTile;
     const int per = (tiles + P - 1) / P;
-    // the splits' partial states [BH][P][d*d + d] start at the state area; the apply kernel sums
-    // them in index order while it converts S to its bf16 operand
-    (void)ws_partial;
-    cudaError_t e = launch_state(p, ws_state, P, per, status, stream);
+    cudaError_t e = launch_state(p, ws_partial, ws_state, counters, P, per, status, stream);
     if (e != cudaSuccess) return e;
     ++*launches;
     timer->mark(stream, "tc_state");
-    e = launch_apply(p, ws_state, P, status, stream);
+    e = launch_apply(p, ws_state, 1, status, stream);
     if (e != cudaSuccess) return e;
     ++*launches;
     timer->mark(stream, "tc_apply");

@@ -17,13 +17,14 @@ bool supports(const Problem& p);
 int choose_splits(int BH, int N);
 
 // Enqueue state build, split reduction and apply for one problem.  `status` is the device status
-// word.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
+// word; `counters` holds one zero-initialised arrival counter per (b,h), left at zero by every call.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
 // be built.
-cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, int P, unsigned* status,
-                    cudaStream_t stream, int* launches, KernelTimer* timer);
+cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsigned* counters, int P,
+                    unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer);
 
 // Launchers of the individual kernels (each in its own file).
-cudaError_t launch_state(const Problem& p, float* dst, int P, int tiles_per_cta, unsigned* status, cudaStream_t st);
+cudaError_t launch_state(const Problem& p, float* partial, float* final_state, unsigned* counters, int P,
+                         int tiles_per_cta, unsigned* status, cudaStream_t st);
 cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st);
 
 }  // namespace tc

@@ -26,7 +26,8 @@ constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
 __global__ void __launch_bounds__(kThreads, 2)
 tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                float* __restrict__ dst, int N, int tiles_per_cta, int P, float eps2, unsigned* status) {
+                float* __restrict__ dst, float* __restrict__ final_state, unsigned* __restrict__ counters,
+                int N, int tiles_per_cta, int P, float eps2, unsigned* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* ones = smem + kStages * kStageBytes;
@@ -172,13 +173,40 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
     }
     tcgen05_fence_before_sync();
+    __threadfence();  // this split's partial state is visible device-wide before the arrival below
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+
+    // Cross-split reduction without a second launch and without any waiting: every CTA of a (b,h)
+    // counts itself in; the one that arrives last sums the P partial states in index order (so the
+    // result does not depend on which CTA that is) and re-arms the counter for the next call.
+    if (P > 1 && !*abort_flag) {
+        __shared__ int is_last;
+        if (tid == 0) is_last = (atomicAdd(&counters[bh], 1u) == (unsigned)(P - 1));
+        __syncthreads();
+        if (is_last) {
+            __threadfence();
+            constexpr int kWords4 = (kD * kD + kD) / 4;
+            const float4* src = reinterpret_cast<const float4*>(dst + (size_t)bh * P * (kD * kD + kD));
+            float4* fin = reinterpret_cast<float4*>(final_state + (size_t)bh * (kD * kD + kD));
+            for (int i = tid; i < kWords4; i += kThreads) {
+                float4 a = __ldcg(src + i);
+#pragma unroll 6
+                for (int pp = 1; pp < P; ++pp) {
+                    const float4 b = __ldcg(src + (size_t)pp * kWords4 + i);
+                    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                }
+                fin[i] = a;
+            }
+            if (tid == 0) counters[bh] = 0;
+        }
+    }
 }
 
 }  // namespace
 
-cudaError_t launch_state(const Problem& p, float* dst, int P, int tiles_per_cta, unsigned* status, cudaStream_t st) {
+cudaError_t launch_state(const Problem& p, float* partial, float* final_state, unsigned* counters, int P,
+                         int tiles_per_cta, unsigned* status, cudaStream_t st) {
     CUtensorMap tmK, tmV;
     const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)p.N, (uint64_t)p.BH};
     const uint32_t box[3] = {kD, kTile, 1};
@@ -186,8 +214,8 @@ cudaError_t launch_state(const Problem& p, float* dst, int P, int tiles_per_cta,
         return cudaErrorNotSupported;
     cudaError_t e = cudaFuncSetAttribute(tc_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    tc_state_kernel<<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(tmK, tmV, dst, p.N, tiles_per_cta, P, p.eps2,
-                                                                        status);
+    tc_state_kernel<<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(
+        tmK, tmV, P > 1 ? partial : final_state, final_state, counters, p.N, tiles_per_cta, P, p.eps2, status);
     return cudaGetLastError();
 }
 
