@@ -14,7 +14,7 @@ struct castling_attn {
     int sm_count = 0;
     float* ws = nullptr;        // header | state | partial
     size_t ws_bytes = 0;
-    unsigned* counters = nullptr;  // one arrival counter per (b,h), zero between calls
+    unsigned* counters = nullptr;  // arrival counters of the split reduction, zero between calls
     size_t counters_cap = 0;
     char* stage = nullptr;      // device staging for castling_attn_forward_host
     size_t stage_bytes = 0;
@@ -75,9 +75,10 @@ int ensure_workspace(castling_attn* h, int BH, int N, int d) {
 }
 
 int ensure_counters(castling_attn* h, int BH) {
-    if ((size_t)BH <= h->counters_cap) return CASTLING_OK;
-    size_t cap = 1024;
-    while (cap < (size_t)BH) cap *= 2;
+    const size_t want = (size_t)BH * castling::tc::kCountersPerHead;
+    if (want <= h->counters_cap) return CASTLING_OK;
+    size_t cap = 4096;
+    while (cap < want) cap *= 2;
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return fail_cuda(h, e);
     if (h->counters) cudaFree(h->counters);

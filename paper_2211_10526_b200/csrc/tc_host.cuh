@@ -7,6 +7,9 @@
 namespace castling {
 namespace tc {
 
+// Arrival counters per (b,h): one per group of splits (at most 64 / 4 groups) and one for the groups.
+constexpr int kCountersPerHead = 17;
+
 bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
                           const uint32_t* box, bool swizzle128);
 
@@ -17,7 +20,7 @@ bool supports(const Problem& p);
 int choose_splits(int BH, int N);
 
 // Enqueue state build, split reduction and apply for one problem.  `status` is the device status
-// word; `counters` holds one zero-initialised arrival counter per (b,h), left at zero by every call.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
+// word; `counters` holds kCountersPerHead zero-initialised arrival counters per (b,h), left at zero by every call.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
 // be built.
 cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer);

@@ -22,6 +22,7 @@ constexpr int kStageBytes = 2 * kTileBytes;  // K then V
 constexpr int kOnesBytes = 2048;             // 16 token rows x 128 B: feature 64 = 1, 65..127 = 0
 constexpr int kThreads = 192;                // warp 0 TMA, warp 1 UMMA, warps 2..5 scale + epilogue
 constexpr int kTmemCols = 64;
+constexpr int kGroup = 4;                    // splits per first-level reduction group
 constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -177,29 +178,78 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 
-    // Cross-split reduction without a second launch and without any waiting: every CTA of a (b,h)
-    // counts itself in; the one that arrives last sums the P partial states in index order (so the
-    // result does not depend on which CTA that is) and re-arms the counter for the next call.
+    // Cross-split reduction without a second launch and without any waiting, as a two-level tree
+    // driven by arrival counters: the splits of a (b,h) form groups of kGroup; the CTA that arrives
+    // last in its group sums the group's partial states in index order into the group's first slot,
+    // then the group that arrives last sums the group results in index order into the final state.
+    // The order of the additions is fixed, so the result does not depend on which CTAs came last.
+    // Every counter is put back to zero by the CTA that consumed it.
     if (P > 1 && !*abort_flag) {
         __shared__ int is_last;
-        if (tid == 0) is_last = (atomicAdd(&counters[bh], 1u) == (unsigned)(P - 1));
+        constexpr int kWords = kD * kD + kD, kWords4 = kWords / 4, kIter = (kWords4 + kThreads - 1) / kThreads;
+        unsigned* cnt = counters + (size_t)bh * kCountersPerHead;
+        const int n_groups = (P + kGroup - 1) / kGroup, grp = p / kGroup;
+        const int first = grp * kGroup, members = min(kGroup, P - first);
+        float4* base = reinterpret_cast<float4*>(dst + (size_t)bh * P * kWords);
+        if (tid == 0) is_last = (atomicAdd(&cnt[grp], 1u) == (unsigned)(members - 1));
         __syncthreads();
-        if (is_last) {
-            __threadfence();
-            constexpr int kWords4 = (kD * kD + kD) / 4;
-            const float4* src = reinterpret_cast<const float4*>(dst + (size_t)bh * P * (kD * kD + kD));
-            float4* fin = reinterpret_cast<float4*>(final_state + (size_t)bh * (kD * kD + kD));
-            for (int i = tid; i < kWords4; i += kThreads) {
-                float4 a = __ldcg(src + i);
-#pragma unroll 6
-                for (int pp = 1; pp < P; ++pp) {
-                    const float4 b = __ldcg(src + (size_t)pp * kWords4 + i);
-                    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-                }
-                fin[i] = a;
+        if (!is_last) return;
+        __threadfence();
+        if (members > 1) {
+            float4 acc[kIter];
+#pragma unroll
+            for (int j = 0; j < kIter; ++j) {
+                const int i = tid + j * kThreads;
+                if (i < kWords4) acc[j] = __ldcg(base + (size_t)first * kWords4 + i);
             }
-            if (tid == 0) counters[bh] = 0;
+            for (int m = 1; m < members; ++m) {
+                float4 v[kIter];
+#pragma unroll
+                for (int j = 0; j < kIter; ++j) {
+                    const int i = tid + j * kThreads;
+                    if (i < kWords4) v[j] = __ldcg(base + (size_t)(first + m) * kWords4 + i);
+                }
+#pragma unroll
+                for (int j = 0; j < kIter; ++j) { acc[j].x += v[j].x; acc[j].y += v[j].y; acc[j].z += v[j].z; acc[j].w += v[j].w; }
+            }
+#pragma unroll
+            for (int j = 0; j < kIter; ++j) {
+                const int i = tid + j * kThreads;
+                if (i < kWords4) base[(size_t)first * kWords4 + i] = acc[j];
+            }
         }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            cnt[grp] = 0;
+            is_last = (atomicAdd(&cnt[kCountersPerHead - 1], 1u) == (unsigned)(n_groups - 1));
+        }
+        __syncthreads();
+        if (!is_last) return;
+        __threadfence();
+        float4* fin = reinterpret_cast<float4*>(final_state + (size_t)bh * kWords);
+        float4 acc[kIter];
+#pragma unroll
+        for (int j = 0; j < kIter; ++j) {
+            const int i = tid + j * kThreads;
+            if (i < kWords4) acc[j] = __ldcg(base + i);
+        }
+        for (int g = 1; g < n_groups; ++g) {
+            float4 v[kIter];
+#pragma unroll
+            for (int j = 0; j < kIter; ++j) {
+                const int i = tid + j * kThreads;
+                if (i < kWords4) v[j] = __ldcg(base + (size_t)g * kGroup * kWords4 + i);
+            }
+#pragma unroll
+            for (int j = 0; j < kIter; ++j) { acc[j].x += v[j].x; acc[j].y += v[j].y; acc[j].z += v[j].z; acc[j].w += v[j].w; }
+        }
+#pragma unroll
+        for (int j = 0; j < kIter; ++j) {
+            const int i = tid + j * kThreads;
+            if (i < kWords4) fin[i] = acc[j];
+        }
+        if (tid == 0) cnt[kCountersPerHead - 1] = 0;
     }
 }
 
