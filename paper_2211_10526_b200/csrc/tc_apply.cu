@@ -108,6 +108,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 0) {
         if (lane == 0) {
             int issued = 0;
+            const uint64_t pol_q = l2_policy_evict_first();  // Q is read once
             for (int it = 0; it < my_tiles; ++it) {
                 const int s = it % NS, use = it / NS;
                 if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) break;
@@ -115,7 +116,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
                 uint8_t* qs = stages + s * G::kStage;
                 mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
-                tma_load_4d(qs, &tmQ, &full[s], 0, x0, y0, bh);
+                tma_load_4d_hint(qs, &tmQ, &full[s], 0, x0, y0, bh, pol_q);
                 tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::R, y0 - G::R, bh);
                 ++issued;
             }
@@ -153,7 +154,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ---------------- epilogue: one thread per token of the patch ----------------
         const int quarter = warp & 3, row = quarter * 32 + lane, et = tid - 64;
         const bool leader = (et == 0);
+        const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
         int prev_bh = -1;
+        pdl_wait_primary();  // the state kernel's results are read below
         for (int it = 0; it < my_tiles; ++it) {
             const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
             const int g = g_begin + it, bh = g / tiles_per_bh, rem = g % tiles_per_bh;
@@ -230,7 +233,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             fence_proxy_async_smem();
             named_barrier_sync(1, kTile);
             if (leader) {
-                tma_store_4d(&tmO, out_s, 0, x0, y0, bh);
+                tma_store_4d_hint(&tmO, out_s, 0, x0, y0, bh, pol_o);
                 tma_store_commit();
             }
         }
@@ -242,6 +245,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         float2 wreg[KS][KS];
         float2 cinit = make_float2(0.f, 0.f);
         int prev_bh = -1;
+        pdl_wait_primary();  // the token sums of the state kernel are read below
         for (int it = 0; it < my_tiles; ++it) {
             const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
             const int bh = (g_begin + it) / tiles_per_bh;
@@ -323,8 +327,15 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     cudaError_t e = cudaFuncSetAttribute(tc_apply_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmem);
     if (e != cudaSuccess) return e;
     const int grid = prm.n_tiles < 148 ? prm.n_tiles : 148;
-    tc_apply_kernel<KS><<<grid, kThreads, G::kSmem, st>>>(tmQ, tmV, tmO, prm);
-    return cudaGetLastError();
+    // programmatic dependent launch: this grid's prologue and first Q / V loads overlap the tail of
+    // the state kernel; the warps that read its results wait for it (griddepcontrol.wait) first
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = G::kSmem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS>, tmQ, tmV, tmO, prm);
 }
 
 }  // namespace

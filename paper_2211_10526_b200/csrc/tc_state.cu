@@ -50,6 +50,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         return;
     }
 
+    pdl_launch_dependents();  // the apply kernel may begin its prologue while this grid drains
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&full[s], 1);
@@ -81,13 +82,15 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (warp == 0) {
         if (lane == 0) {
             int issued = 0;
+            // K is read once; V is read again by the apply kernel: keep it in L2 as long as possible
+            const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_last();
             for (int it = 0; it < n_tiles; ++it) {
                 const int s = it % kStages, use = it / kStages;
                 if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, status, kStatusStateTimeout)) break;
                 uint8_t* ks = smem + s * kStageBytes;
                 mbar_expect_tx(&full[s], kStageBytes);
-                tma_load_3d(ks, &tmK, &full[s], 0, (t_begin + it) * kTile, bh);
-                tma_load_3d(ks + kTileBytes, &tmV, &full[s], 0, (t_begin + it) * kTile, bh);
+                tma_load_3d_hint(ks, &tmK, &full[s], 0, (t_begin + it) * kTile, bh, pol_k);
+                tma_load_3d_hint(ks + kTileBytes, &tmV, &full[s], 0, (t_begin + it) * kTile, bh, pol_v);
                 ++issued;
             }
             if (*abort_flag) {
