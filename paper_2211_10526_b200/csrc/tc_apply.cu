@@ -6,12 +6,12 @@
 //               the convolution's zero padding
 //   warp 1      one thread issues four UMMAs: acc[128 x 64] = Q[128 x 64] * S'[64 x 64] into TMEM,
 //               S' = S / pi in bf16; the row scale 1/||q|| commutes and is applied afterwards
-//   warps 6..9  depthwise convolution on CUDA cores, one lane per channel pair, filters in
-//               registers, sliding window along x, packed fp32x2 FMAs, result (+ 1/2 s + bias)
-//               staged in shared memory as fp32
-//   warps 2..5  one thread per token: ||q|| from the Q patch, accumulator row from TMEM,
-//               out = acc / max(||q||, eps) + staged, one rounding to bf16, patch written to
-//               shared memory and stored with TMA (clipped at the grid edge)
+//   warps 10..17 depthwise convolution on CUDA cores, one lane per channel pair, filters in
+//               registers, sliding window along x (two rows x eight columns per warp), packed
+//               fp32x2 FMAs, result (+ 1/2 s + bias) staged in shared memory as fp32
+//   warps 2..9  one thread per token and half of its channels: ||q|| from the Q patch,
+//               accumulator row from TMEM, out = acc / max(||q||, eps) + staged, one rounding to
+//               bf16, patch written to shared memory and stored with TMA (clipped at the grid edge)
 #include "tc_common.cuh"
 #include "tc_host.cuh"
 
@@ -25,7 +25,9 @@ constexpr int kTile = kTY * kTX;
 constexpr int kQBytes = kTile * kD * 2;     // 16 KiB
 constexpr int kStgStride = kD * 4 + 16;     // fp32 row + 16 B pad: conflict-free row-per-thread reads
 constexpr int kStgBytes = kTile * kStgStride;
-constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8, kConvWarps = 8;   // two warps per TMEM lane quarter / per pair of patch rows
+constexpr int kEpiThreads = kEpiWarps * 32, kConvThreads = kConvWarps * 32;
+constexpr int kThreads = 64 + kEpiThreads + kConvThreads;
 constexpr int kTmemCols = 128;              // two 64-column accumulators
 
 template <int KS> struct Geo {
@@ -34,10 +36,11 @@ template <int KS> struct Geo {
     static constexpr int kVBytes = HY * HX * kD * 2;
     static constexpr int kStage = ((kQBytes + kVBytes + 1023) / 1024) * 1024;
     static constexpr int kStages = (KS == 3) ? 3 : 2;
-    // S' | out patch | stages | staging x2 | barriers
+    // S' | out patch | stages | staging x2 | rq x2 | barriers
     static constexpr int kOffS = 0, kOffOut = 8192, kOffStages = kOffOut + kQBytes;
     static constexpr int kOffStg = kOffStages + kStages * kStage;
-    static constexpr int kOffBar = kOffStg + 2 * kStgBytes;
+    static constexpr int kOffRq = kOffStg + 2 * kStgBytes;   // 1 / ||q|| per token, two buffers
+    static constexpr int kOffBar = kOffRq + 2 * kTile * 4;
     static constexpr size_t kSmem = 1024 + kOffBar + 256;
 };
 
@@ -74,10 +77,11 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     uint8_t* out_s = smem + G::kOffOut;
     uint8_t* stages = smem + G::kOffStages;
     uint8_t* stg = smem + G::kOffStg;
+    float* rq_s = reinterpret_cast<float*>(smem + G::kOffRq);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + G::kOffBar);  // [NS] TMA landed
-    uint64_t* empty = full + NS;                                      // [NS] stage consumed (128 arrivals)
+    uint64_t* empty = full + NS;                                      // [NS] stage consumed (conv warps + UMMA commit)
     uint64_t* acc_full = empty + NS;                                  // [2]  UMMAs retired
-    uint64_t* conv_full = acc_full + 2;                               // [2]  staging written (128 arrivals)
+    uint64_t* conv_full = acc_full + 2;                               // [2]  staging and 1/||q|| written (conv warps)
     uint64_t* buf_free = conv_full + 2;                               // [2]  accumulator + staging read (128)
     uint64_t* s_ready = buf_free + 2;                                 // S' of the current (b,h) written (128)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_ready + 1);
@@ -91,9 +95,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int my_tiles = g_end - g_begin;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kTile); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], kTile); mbar_init(&buf_free[b], kTile); }
-        mbar_init(s_ready, kTile);
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConvThreads + 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], kConvThreads); mbar_init(&buf_free[b], kEpiThreads); }
+        mbar_init(s_ready, kEpiThreads);
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO);
@@ -148,26 +152,28 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     umma_bf16(tmem + b * kD, a, bd, idesc, k != 0);
                 }
                 umma_commit(&acc_full[b]);
+                umma_commit(&empty[s]);  // the same UMMAs have finished reading the Q patch
             }
         }
-    } else if (warp < 6) {
-        // ---------------- epilogue: one thread per token of the patch ----------------
+    } else if (warp < 2 + kEpiWarps) {
+        // ------- epilogue: thread = (token of the patch, half of the channels) -------
         const int quarter = warp & 3, row = quarter * 32 + lane, et = tid - 64;
+        const int half = (warp - 2) >> 2;  // channels half*32 .. half*32 + 31
         const bool leader = (et == 0);
         const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
         int prev_bh = -1;
         pdl_wait_primary();  // the state kernel's results are read below
         for (int it = 0; it < my_tiles; ++it) {
-            const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
+            const int b = it & 1, ub = it >> 1;
             const int g = g_begin + it, bh = g / tiles_per_bh, rem = g % tiles_per_bh;
             const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
             if (bh != prev_bh) {
                 // every UMMA that read the previous S' has retired (its acc_full was waited on below)
                 prev_bh = bh;
-                const int i = et >> 1, half = et & 1;
-                const float4* src = reinterpret_cast<const float4*>(prm.state + (size_t)(prm.bh0 + bh) * prm.P * (kD * kD + kD) + i * kD + half * 32);
+                const int i = et >> 2, part = et & 3;  // row i of S, 16 columns part*16 ..
+                const float4* src = reinterpret_cast<const float4*>(prm.state + (size_t)(prm.bh0 + bh) * prm.P * (kD * kD + kD) + i * kD + part * 16);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     float4 lo = __ldg(src + 2 * c), hi = __ldg(src + 2 * c + 1);
                     for (int pp = 1; pp < prm.P; ++pp) {  // fixed order: bitwise reproducible
                         const float4 l2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c);
@@ -178,60 +184,45 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     uint4 o;
                     o.x = pack_bf16x2(lo.x * kInvPi, lo.y * kInvPi); o.y = pack_bf16x2(lo.z * kInvPi, lo.w * kInvPi);
                     o.z = pack_bf16x2(hi.x * kInvPi, hi.y * kInvPi); o.w = pack_bf16x2(hi.z * kInvPi, hi.w * kInvPi);
-                    *reinterpret_cast<uint4*>(S_s + i * 128 + (((half * 4 + c) ^ (i & 7)) << 4)) = o;
+                    *reinterpret_cast<uint4*>(S_s + i * 128 + (((part * 2 + c) ^ (i & 7)) << 4)) = o;
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(s_ready);
             }
-            if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
-            // 1 / max(||q||, eps) of this thread's token
-            const uint8_t* qrow = stages + s * G::kStage + row * 128;
-            float ss = 0.f;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint4 c = *reinterpret_cast<const uint4*>(qrow + ((j ^ (row & 7)) << 4));
-                const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float lo = bf16lo(w4[e]), hi = bf16hi(w4[e]);
-                    ss = fmaf(lo, lo, ss); ss = fmaf(hi, hi, ss);
-                }
-            }
-            const float rq = 1.0f / sqrtf(fmaxf(ss, prm.eps2));
             if (!mbar_wait(&acc_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
-            if (!mbar_wait(&conv_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
             tcgen05_fence_after_sync();
+            float a[32];
+            {
+                float a0[16], a1[16];
+                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kD + half * 32, a0);
+                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kD + half * 32 + 16, a1);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 16; ++e) { a[e] = a0[e]; a[16 + e] = a1[e]; }
+            }
+            if (!mbar_wait(&conv_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
+            const float rq = rq_s[b * kTile + row];
             if (it > 0) {  // the previous patch's TMA store must have read out_s before it is rewritten
                 if (leader) tma_store_wait_read();
-                named_barrier_sync(1, kTile);
+                named_barrier_sync(1, kEpiThreads);
             }
-            const uint8_t* srow = stg + b * kStgBytes + row * kStgStride;
+            const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
             uint8_t* orow = out_s + row * 128;
 #pragma unroll
-            for (int cc = 0; cc < kD / 16; ++cc) {
-                float a[16];
-                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kD + cc * 16, a);
-                tmem_ld_wait();
-                float o[16];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float4 c4 = *reinterpret_cast<const float4*>(srow + cc * 64 + e * 16);
-                    o[4 * e + 0] = fmaf(a[4 * e + 0], rq, c4.x); o[4 * e + 1] = fmaf(a[4 * e + 1], rq, c4.y);
-                    o[4 * e + 2] = fmaf(a[4 * e + 2], rq, c4.z); o[4 * e + 3] = fmaf(a[4 * e + 3], rq, c4.w);
-                }
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    uint4 pk;
-                    pk.x = pack_bf16x2(o[8 * e + 0], o[8 * e + 1]); pk.y = pack_bf16x2(o[8 * e + 2], o[8 * e + 3]);
-                    pk.z = pack_bf16x2(o[8 * e + 4], o[8 * e + 5]); pk.w = pack_bf16x2(o[8 * e + 6], o[8 * e + 7]);
-                    *reinterpret_cast<uint4*>(orow + (((2 * cc + e) ^ (row & 7)) << 4)) = pk;
-                }
+            for (int e = 0; e < 4; ++e) {  // 8 channels -> one 16-byte chunk of the bf16 row
+                const float4 c0 = *reinterpret_cast<const float4*>(srow + e * 32);
+                const float4 c1 = *reinterpret_cast<const float4*>(srow + e * 32 + 16);
+                uint4 pk;
+                pk.x = pack_bf16x2(fmaf(a[8 * e + 0], rq, c0.x), fmaf(a[8 * e + 1], rq, c0.y));
+                pk.y = pack_bf16x2(fmaf(a[8 * e + 2], rq, c0.z), fmaf(a[8 * e + 3], rq, c0.w));
+                pk.z = pack_bf16x2(fmaf(a[8 * e + 4], rq, c1.x), fmaf(a[8 * e + 5], rq, c1.y));
+                pk.w = pack_bf16x2(fmaf(a[8 * e + 6], rq, c1.z), fmaf(a[8 * e + 7], rq, c1.w));
+                *reinterpret_cast<uint4*>(orow + (((half * 4 + e) ^ (row & 7)) << 4)) = pk;
             }
             tcgen05_fence_before_sync();
             mbar_arrive(&buf_free[b]);
-            mbar_arrive(&empty[s]);
             fence_proxy_async_smem();
-            named_barrier_sync(1, kTile);
+            named_barrier_sync(1, kEpiThreads);
             if (leader) {
                 tma_store_4d_hint(&tmO, out_s, 0, x0, y0, bh, pol_o);
                 tma_store_commit();
@@ -239,8 +230,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         if (leader) tma_store_wait_all();
     } else {
-        // ---------------- depthwise convolution: lane = channel pair, warp = two patch rows ----------------
-        const int cw = warp - 6;
+        // ------- depthwise convolution: lane = channel pair, warp = two patch rows x eight columns -------
+        const int cw = (warp - 2 - kEpiWarps) >> 1, xh = (warp - 2 - kEpiWarps) & 1;
+        constexpr int kCX = kTX / 2;
         constexpr int R = G::R, ROWS = 2 + 2 * R;
         float2 wreg[KS][KS];
         float2 cinit = make_float2(0.f, 0.f);
@@ -269,8 +261,27 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
             if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
-            const uint8_t* vh = stages + s * G::kStage + kQBytes + (2 * cw) * G::HX * 128 + lane * 4;
-            uint8_t* so = stg + b * kStgBytes + (2 * cw) * kTX * kStgStride + lane * 8;
+            {   // 1 / max(||q||, eps) of this warp's 16 tokens: two lanes per token, 32 elements each
+                const int tl = lane >> 1, hf = lane & 1;
+                const int tok = (2 * cw + (tl >> 3)) * kTX + xh * kCX + (tl & 7);
+                const uint8_t* qrow = stages + s * G::kStage + tok * 128;
+                float ss[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 c = *reinterpret_cast<const uint4*>(qrow + (((4 * hf + j) ^ (tok & 7)) << 4));
+                    const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float lo = bf16lo(w4[e]), hi = bf16hi(w4[e]);
+                        ss[e] = fmaf(lo, lo, ss[e]); ss[e] = fmaf(hi, hi, ss[e]);
+                    }
+                }
+                float tot = (ss[0] + ss[1]) + (ss[2] + ss[3]);
+                tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+                if (hf == 0) rq_s[b * kTile + tok] = 1.0f / sqrtf(fmaxf(tot, prm.eps2));
+            }
+            const uint8_t* vh = stages + s * G::kStage + kQBytes + ((2 * cw) * G::HX + xh * kCX) * 128 + lane * 4;
+            uint8_t* so = stg + b * kStgBytes + ((2 * cw) * kTX + xh * kCX) * kStgStride + lane * 8;
             float2 win[ROWS][KS];  // window columns x .. x+KS-1, rotating
 #pragma unroll
             for (int dx = 0; dx < KS - 1; ++dx)
@@ -280,7 +291,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     win[r][dx] = make_float2(bf16lo(wv), bf16hi(wv));
                 }
 #pragma unroll
-            for (int x = 0; x < kTX; ++x) {
+            for (int x = 0; x < kCX; ++x) {
 #pragma unroll
                 for (int r = 0; r < ROWS; ++r) {
                     const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + (r * G::HX + x + KS - 1) * 128);
@@ -297,6 +308,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 *reinterpret_cast<float2*>(so + x * kStgStride) = a0;
                 *reinterpret_cast<float2*>(so + (kTX + x) * kStgStride) = a1;
             }
+            mbar_arrive(&empty[s]);      // Q rows and V patch of this stage are no longer needed
             mbar_arrive(&conv_full[b]);
         }
     }
