@@ -57,7 +57,8 @@ enum {
     CASTLING_ERR_ARCH = -4,        /* current device is not compute capability 10.x          */
     CASTLING_ERR_CUDA = -5,        /* a CUDA call failed; see castling_attn_last_cuda_error  */
     CASTLING_ERR_OOM = -6,         /* workspace allocation failed or exceeds max_workspace   */
-    CASTLING_ERR_DEVICE = -7       /* a kernel reported a bounded wait that ran out          */
+    CASTLING_ERR_DEVICE = -7,      /* a kernel reported a bounded wait that ran out          */
+    CASTLING_ERR_SCRATCH_LIMIT = -8 /* problem needs more than the built-in static scratch    */
 };
 
 /* Kernel families the dispatcher can be pinned to (testing and benchmarking). */
@@ -167,6 +168,38 @@ CASTLING_API int castling_attn_set_profiling(castling_attn_t* handle, int enable
  * number written (0 when profiling is off), or a negative error code.
  */
 CASTLING_API int castling_attn_kernel_times(castling_attn_t* handle, float* ms, const char** names, int capacity);
+
+/*
+ * castling_attn_forward_static: the same forward pass for callers that cannot allocate device
+ * memory -- code running inside a region where cudaMalloc is forbidden or would stall everything
+ * (a latency-critical serving loop, a plug-in that is handed a fixed memory budget by its host
+ * application, a process whose allocator owns the whole GPU).  It takes no handle and calls no
+ * cudaMalloc, cudaFree or any other allocating routine.  (The paper has no counterpart to this
+ * entry point; it exists only for such callers.)
+ *
+ * The d x d states that pass from the state kernel to the apply kernel are kept in a fixed
+ * CASTLING_STATIC_SCRATCH_BYTES (4 MiB) array that is part of the library's device image: every
+ * GPU on which the library is loaded holds that array until the process exits.  A problem fits
+ * when B*H*(d*d + d)*4 bytes <= CASTLING_STATIC_SCRATCH_BYTES (e.g. d = 64: B*H <= 252;
+ * d = 32: B*H <= 992); larger ones return CASTLING_ERR_SCRATCH_LIMIT and nothing is launched.
+ * The CUDA-core kernels are used for every dtype.
+ *
+ * Arguments as for castling_attn_forward, with the handle's configuration passed directly:
+ * ksize (odd, 1..7) and eps (<= 0 selects 1e-12).  Tensors are DEVICE pointers, 16-byte aligned;
+ * the call only enqueues on `stream`.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) with
+ * that device current; make that first call outside any stream capture.  All calls on a device
+ * share the one array and it keeps the last call's contents: nothing in it needs clearing
+ * between calls (every word that is read is first overwritten by the same call), but two calls
+ * whose kernels overlap on the GPU -- different streams, or the same problem from two threads --
+ * race on it.  Serialise them on one stream.
+ */
+#define CASTLING_STATIC_SCRATCH_BYTES (4u << 20)
+CASTLING_API int castling_attn_forward_static(const void* q, const void* k, const void* v,
+                                              const void* dw_weight, const void* dw_bias, void* out,
+                                              int B, int H, int gridH, int gridW, int d,
+                                              int ksize, double eps, castling_dtype_t dtype, void* stream);
 
 #ifdef __cplusplus
 }

@@ -17,6 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libcastling_attn.so")
 CASTLING_F32, CASTLING_BF16 = 0, 1
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARCH, ERR_CUDA, ERR_OOM, ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6, -7
+ERR_SCRATCH_LIMIT = -8
+STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class castling_attn_config_t(ctypes.Structure):
@@ -59,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.castling_attn_set_profiling.argtypes = [vp, i]
     lib.castling_attn_kernel_times.restype = i
     lib.castling_attn_kernel_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_char_p), i]
+    lib.castling_attn_forward_static.restype = i
+    lib.castling_attn_forward_static.argtypes = [vp] * 6 + [i] * 6 + [ctypes.c_double, i, vp]
     return lib
 
 
@@ -131,3 +135,12 @@ def castling_attn_kernel_times(handle):
     if n < 0:
         raise CastlingError(n, "castling_attn_kernel_times")
     return [(names[i].decode(), float(ms[i])) for i in range(n)]
+
+
+def castling_attn_forward_static(q: int, k: int, v: int, dw_weight: int, dw_bias: Optional[int], out: int,
+                                 B: int, H: int, gridH: int, gridW: int, d: int, ksize: int, eps: float,
+                                 dtype: int, stream: int = 0) -> int:
+    """Forward pass that allocates nothing (scratch is a fixed array inside the library); raw device
+    addresses in, C return code out.  See the header for the size limit and the sharing rules."""
+    return lib.castling_attn_forward_static(q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, ksize,
+                                            float(eps), dtype, stream or None)

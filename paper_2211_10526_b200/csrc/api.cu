@@ -147,6 +147,7 @@ const char* castling_attn_error_string(int code) {
         case CASTLING_ERR_CUDA: return "a CUDA call failed (see castling_attn_last_cuda_error)";
         case CASTLING_ERR_OOM: return "workspace allocation failed or exceeds max_workspace";
         case CASTLING_ERR_DEVICE: return "a kernel gave up on a bounded wait";
+        case CASTLING_ERR_SCRATCH_LIMIT: return "problem needs more than the library's static scratch (use castling_attn_forward with a handle)";
         default: return "unknown castling_attn error code";
     }
 }
