@@ -35,6 +35,10 @@ METRIC = "tokens/sec and achieved HBM GB/s (% of B200 peak) for linear-angular a
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "c5_sweep_bf16:3"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
+# one ncu capture of this command at full size (profiles/tc_kernels_c5_sweep.md); None for workloads
+# or kernels without a capture of the current code.
+NCU_TRAFFIC_BYTES = {("c5_sweep_bf16:3", "tc_apply"): 252.5e6 + 99.8e6}
 
 
 def parse_args():
@@ -277,7 +281,8 @@ def main():
         achieved = alg[top] / (kernels[top] * 1e-3) / 1e9
         path_gbs = s.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                    "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get((args.workload, top)),
+                    "traffic_unit": "bytes per launch, ncu", "peak_source": peak_src,
                     "kernel_ms": kernels, "path_achieved": path_gbs, "path_frac": path_gbs / peak,
                     "path_frac_of_8000": path_gbs / 8000.0}
 
