@@ -9,7 +9,8 @@
 //   warps 10..17 depthwise convolution on CUDA cores, one lane per channel pair, filters in
 //               registers, sliding window along x (two rows x eight columns per warp), packed
 //               fp32x2 FMAs, result (+ 1/2 s + bias) staged in shared memory as fp32
-//   warps 2..9  one thread per token and half of its channels: ||q|| from the Q patch,
+//   warps 2..9  one thread per token and half of its channels: ||q|| from the Q patch (each of
+//               the two warps of a token sums half of the row, exchanged through shared memory),
 //               accumulator row from TMEM, out = acc / max(||q||, eps) + staged, one rounding to
 //               bf16, patch written to shared memory and stored with TMA (clipped at the grid edge)
 #include "tc_common.cuh"
@@ -39,7 +40,7 @@ template <int KS> struct Geo {
     // S' | out patch | stages | staging x2 | rq x2 | barriers
     static constexpr int kOffS = 0, kOffOut = 8192, kOffStages = kOffOut + kQBytes;
     static constexpr int kOffStg = kOffStages + kStages * kStage;
-    static constexpr int kOffRq = kOffStg + 2 * kStgBytes;   // 1 / ||q|| per token, two buffers
+    static constexpr int kOffRq = kOffStg + 2 * kStgBytes;   // sum of squares of each half of a Q row
     static constexpr int kOffBar = kOffRq + 2 * kTile * 4;
     static constexpr size_t kSmem = 1024 + kOffBar + 256;
 };
@@ -79,9 +80,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     uint8_t* stg = smem + G::kOffStg;
     float* rq_s = reinterpret_cast<float*>(smem + G::kOffRq);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + G::kOffBar);  // [NS] TMA landed
-    uint64_t* empty = full + NS;                                      // [NS] stage consumed (conv warps + UMMA commit)
+    uint64_t* empty = full + NS;                                      // [NS] stage consumed (conv + epilogue warps, UMMA commit)
     uint64_t* acc_full = empty + NS;                                  // [2]  UMMAs retired
-    uint64_t* conv_full = acc_full + 2;                               // [2]  staging and 1/||q|| written (conv warps)
+    uint64_t* conv_full = acc_full + 2;                               // [2]  staging written (conv warps)
     uint64_t* buf_free = conv_full + 2;                               // [2]  accumulator + staging read (128)
     uint64_t* s_ready = buf_free + 2;                                 // S' of the current (b,h) written (128)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_ready + 1);
@@ -95,7 +96,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int my_tiles = g_end - g_begin;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConvThreads + 1); }
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConvThreads + kEpiThreads + 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], kConvThreads); mbar_init(&buf_free[b], kEpiThreads); }
         mbar_init(s_ready, kEpiThreads);
         *abort_flag = 0;
@@ -189,6 +190,24 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 fence_proxy_async_smem();
                 mbar_arrive(s_ready);
             }
+            {   // this thread's half of sum(q^2) for its token; the other half comes from the partner warp
+                const int s = it % NS, use = it / NS;
+                if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
+                const uint8_t* qrow = stages + s * G::kStage + row * 128;
+                float ss[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 c = *reinterpret_cast<const uint4*>(qrow + (((4 * half + j) ^ (row & 7)) << 4));
+                    const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float lo = bf16lo(w4[e]), hi = bf16hi(w4[e]);
+                        ss[e] = fmaf(lo, lo, ss[e]); ss[e] = fmaf(hi, hi, ss[e]);
+                    }
+                }
+                rq_s[half * kTile + row] = (ss[0] + ss[1]) + (ss[2] + ss[3]);
+                mbar_arrive(&empty[s]);  // the Q rows of this stage have been read
+            }
             if (!mbar_wait(&acc_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
             tcgen05_fence_after_sync();
             float a[32];
@@ -201,11 +220,11 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int e = 0; e < 16; ++e) { a[e] = a0[e]; a[16 + e] = a1[e]; }
             }
             if (!mbar_wait(&conv_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
-            const float rq = rq_s[b * kTile + row];
-            if (it > 0) {  // the previous patch's TMA store must have read out_s before it is rewritten
-                if (leader) tma_store_wait_read();
-                named_barrier_sync(1, kEpiThreads);
-            }
+            // the previous patch's TMA store must have read out_s before it is rewritten; the same
+            // barrier makes both halves of every row's sum of squares visible
+            if (it > 0 && leader) tma_store_wait_read();
+            named_barrier_sync(1, kEpiThreads);
+            const float rq = rsqrtf(fmaxf(rq_s[row] + rq_s[kTile + row], prm.eps2));
             const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
             uint8_t* orow = out_s + row * 128;
 #pragma unroll
@@ -261,25 +280,6 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
             if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
-            {   // 1 / max(||q||, eps) of this warp's 16 tokens: two lanes per token, 32 elements each
-                const int tl = lane >> 1, hf = lane & 1;
-                const int tok = (2 * cw + (tl >> 3)) * kTX + xh * kCX + (tl & 7);
-                const uint8_t* qrow = stages + s * G::kStage + tok * 128;
-                float ss[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 c = *reinterpret_cast<const uint4*>(qrow + (((4 * hf + j) ^ (tok & 7)) << 4));
-                    const uint32_t w4[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float lo = bf16lo(w4[e]), hi = bf16hi(w4[e]);
-                        ss[e] = fmaf(lo, lo, ss[e]); ss[e] = fmaf(hi, hi, ss[e]);
-                    }
-                }
-                float tot = (ss[0] + ss[1]) + (ss[2] + ss[3]);
-                tot += __shfl_xor_sync(0xffffffffu, tot, 1);
-                if (hf == 0) rq_s[b * kTile + tok] = 1.0f / sqrtf(fmaxf(tot, prm.eps2));
-            }
             const uint8_t* vh = stages + s * G::kStage + kQBytes + ((2 * cw) * G::HX + xh * kCX) * 128 + lane * 4;
             uint8_t* so = stg + b * kStgBytes + ((2 * cw) * kTX + xh * kCX) * kStgStride + lane * 8;
             float2 win[ROWS][KS];  // window columns x .. x+KS-1, rotating
@@ -308,7 +308,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 *reinterpret_cast<float2*>(so + x * kStgStride) = a0;
                 *reinterpret_cast<float2*>(so + (kTX + x) * kStgStride) = a1;
             }
-            mbar_arrive(&empty[s]);      // Q rows and V patch of this stage are no longer needed
+            mbar_arrive(&empty[s]);      // the V patch of this stage is no longer needed
             mbar_arrive(&conv_full[b]);
         }
     }
