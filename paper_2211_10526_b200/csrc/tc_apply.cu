@@ -336,8 +336,12 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.tilesX = (p.gridW + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
     prm.eps2 = p.eps2; prm.status = status;
-    cudaError_t e = cudaFuncSetAttribute(tc_apply_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmem);
-    if (e != cudaSuccess) return e;
+    static bool attr_set = false;  // one flag per KS instantiation
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_apply_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
     const int grid = prm.n_tiles < 148 ? prm.n_tiles : 148;
     // programmatic dependent launch: this grid's prologue and first Q / V loads overlap the tail of
     // the state kernel; the warps that read its results wait for it (griddepcontrol.wait) first

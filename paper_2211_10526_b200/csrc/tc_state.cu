@@ -265,8 +265,12 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
     const uint32_t box[3] = {kD, kTile, 1};
     if (!make_tensor_map_bf16(&tmK, p.k, 3, dims, box, true) || !make_tensor_map_bf16(&tmV, p.v, 3, dims, box, true))
         return cudaErrorNotSupported;
-    cudaError_t e = cudaFuncSetAttribute(tc_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
+    static bool attr_set = false;  // per process; the attribute belongs to the function, not to a call
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
     tc_state_kernel<<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(
         tmK, tmV, P > 1 ? partial : final_state, final_state, counters, p.N, tiles_per_cta, P, p.eps2, status);
     return cudaGetLastError();

@@ -19,13 +19,56 @@ void lookup() {
         qres == cudaDriverEntryPointSuccess)
         g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
 }
+
+// A few recently built maps are kept: a serving loop calls with the same tensors and shapes over
+// and over, and encoding five maps per forward costs more host time than the launches.
+struct CacheEntry {
+    bool valid = false;
+    const void* base = nullptr;
+    int rank = 0;
+    uint64_t dims[5] = {};
+    uint32_t box[5] = {};
+    bool swizzle = false;
+    CUtensorMap map;
+};
+constexpr int kCacheSize = 32;
+CacheEntry g_cache[kCacheSize];
+int g_cache_next = 0;
+std::mutex g_cache_mutex;
+
+bool same_key(const CacheEntry& e, const void* base, int rank, const uint64_t* dims, const uint32_t* box, bool sw) {
+    if (!e.valid || e.base != base || e.rank != rank || e.swizzle != sw) return false;
+    for (int i = 0; i < rank; ++i)
+        if (e.dims[i] != dims[i] || e.box[i] != box[i]) return false;
+    return true;
+}
 }  // namespace
+
+namespace {
+bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+                            const uint32_t* box, bool swizzle128);
+}
 
 // dims/box are innermost-first, in elements; the innermost dimension is contiguous.
 bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
                           const uint32_t* box, bool swizzle128) {
+    if (rank < 2 || rank > 5) return false;
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    for (const CacheEntry& e : g_cache)
+        if (same_key(e, base, rank, dims, box, swizzle128)) { *out = e.map; return true; }
+    if (!encode_tensor_map_bf16(out, base, rank, dims, box, swizzle128)) return false;
+    CacheEntry& e = g_cache[g_cache_next];
+    g_cache_next = (g_cache_next + 1) % kCacheSize;
+    e.valid = true; e.base = base; e.rank = rank; e.swizzle = swizzle128; e.map = *out;
+    for (int i = 0; i < rank; ++i) { e.dims[i] = dims[i]; e.box[i] = box[i]; }
+    return true;
+}
+
+namespace {
+bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+                            const uint32_t* box, bool swizzle128) {
     std::call_once(g_once, lookup);
-    if (!g_encode || rank < 2 || rank > 5) return false;
+    if (!g_encode) return false;
     cuuint64_t gdim[5];
     cuuint64_t gstride[4];
     cuuint32_t bdim[5], estride[5];
@@ -43,6 +86,7 @@ bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const ui
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
+}  // namespace
 
 }  // namespace tc
 }  // namespace castling
