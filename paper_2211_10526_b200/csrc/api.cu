@@ -29,10 +29,15 @@ namespace {
 size_t elem_bytes(castling_dtype_t t) { return t == CASTLING_F32 ? 4 : 2; }
 
 // header | state [BH] | partial [BH][P] (only when the token range is split)
-size_t workspace_words(int BH, int N, int d) {
+size_t workspace_words(int BH, int N, int d, bool bf16) {
     int P = castling::simt_choose_splits(BH, N);
-    if (d == 64) P = P > castling::tc::choose_splits(BH, N) ? P : castling::tc::choose_splits(BH, N);
-    return castling::kHeaderWords + (size_t)BH * castling::state_words(d) * (1 + (P > 1 ? P : 0));
+    size_t words = castling::state_words(d);
+    if (bf16 && (d == 64 || d == 32)) {  // shapes the tensor-core kernels may take: they keep 64-wide states
+        const int Pt = castling::tc::choose_splits(BH, castling::tc::rows_per_head(N, d));
+        if (Pt > P) P = Pt;
+        words = castling::tc::kStateWords;
+    }
+    return castling::kHeaderWords + (size_t)BH * words * (1 + (P > 1 ? P : 0));
 }
 
 int fail_cuda(castling_attn* h, cudaError_t e, int code = CASTLING_ERR_CUDA) {
@@ -58,8 +63,8 @@ int check_shape(const castling_attn* h, int B, int H, int gridH, int gridW, int 
     return CASTLING_OK;
 }
 
-int ensure_workspace(castling_attn* h, int BH, int N, int d) {
-    const size_t need = workspace_words(BH, N, d) * sizeof(float);
+int ensure_workspace(castling_attn* h, int BH, int N, int d, bool bf16) {
+    const size_t need = workspace_words(BH, N, d, bf16) * sizeof(float);
     if (need <= h->ws_bytes) return CASTLING_OK;
     if (h->cfg.max_workspace && need > h->cfg.max_workspace) return CASTLING_ERR_OOM;
     cudaError_t e = cudaDeviceSynchronize();  // nothing may still be using the old buffer
@@ -134,7 +139,7 @@ int castling_attn_destroy(castling_attn_t* h) {
 size_t castling_attn_workspace_bytes(int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype) {
     if (B <= 0 || H <= 0 || gridH <= 0 || gridW <= 0 || d <= 0 || d > 128 || d % 16) return 0;
     if (dtype != CASTLING_F32 && dtype != CASTLING_BF16) return 0;
-    return workspace_words(B * H, gridH * gridW, d) * sizeof(float);
+    return workspace_words(B * H, gridH * gridW, d, dtype == CASTLING_BF16) * sizeof(float);
 }
 
 const char* castling_attn_error_string(int code) {
@@ -166,20 +171,20 @@ namespace {
 
 // Enqueue the kernels for one validated problem whose tensors are all on the device.
 int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
-    int rc = ensure_workspace(h, p.BH, p.N, p.d);
+    int rc = ensure_workspace(h, p.BH, p.N, p.d, p.bf16);
     if (rc != CASTLING_OK) return rc;
     const bool tensor_ok = castling::tc::supports(p);
     if (h->cfg.force_path == CASTLING_PATH_TENSOR && !tensor_ok) return CASTLING_ERR_UNSUPPORTED;
     const bool use_tensor = tensor_ok && h->cfg.force_path != CASTLING_PATH_SIMT;
     float* state = h->ws + castling::kHeaderWords;
-    float* partial = state + (size_t)p.BH * castling::state_words(p.d);
+    float* partial = state + (size_t)p.BH * (use_tensor ? (size_t)castling::tc::kStateWords : castling::state_words(p.d));
     int launches = 0;
     h->timer.begin(stream);
     cudaError_t e;
     if (use_tensor) {
         rc = ensure_counters(h, p.BH);
         if (rc != CASTLING_OK) return rc;
-        e = castling::tc::forward(p, state, partial, h->counters, castling::tc::choose_splits(p.BH, p.N),
+        e = castling::tc::forward(p, state, partial, h->counters, castling::tc::choose_splits(p.BH, castling::tc::rows_per_head(p.N, p.d)),
                                   reinterpret_cast<unsigned*>(h->ws), stream, &launches, &h->timer);
     } else {
         e = castling::simt_forward(p, state, partial, castling::simt_choose_splits(p.BH, p.N), stream, &launches,

@@ -31,9 +31,12 @@ constexpr int kEpiThreads = kEpiWarps * 32, kConvThreads = kConvWarps * 32;
 constexpr int kThreads = 64 + kEpiThreads + kConvThreads;
 constexpr int kTmemCols = 128;              // two 64-column accumulators
 
-template <int KS> struct Geo {
+// PAIR = true serves head width 32: a 128-byte row holds two horizontally adjacent tokens, so a
+// "column" of the patch is a token pair and the 8 x 16-column patch covers 8 x 32 tokens.
+template <int KS, bool PAIR> struct Geo {
     static constexpr int R = KS / 2;
-    static constexpr int HY = kTY + 2 * R, HX = kTX + 2 * R;
+    static constexpr int HC = PAIR ? (R + 1) / 2 : R;   // halo columns on each side
+    static constexpr int HY = kTY + 2 * R, HX = kTX + 2 * HC;
     static constexpr int kVBytes = HY * HX * kD * 2;
     static constexpr int kStage = ((kQBytes + kVBytes + 1023) / 1024) * 1024;
     static constexpr int kStages = (KS == 3) ? 3 : 2;
@@ -59,18 +62,18 @@ __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
 struct ApplyParams {
     const float* state;            // [BH][P][64*64 + 64] raw sums of the P token splits
     int P;
-    const __nv_bfloat16* w;        // [H*64][KS][KS]
-    const __nv_bfloat16* bias;     // [H*64] or nullptr
+    const __nv_bfloat16* w;        // [H*d][KS][KS]
+    const __nv_bfloat16* bias;     // [H*d] or nullptr
     int H, bh0, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
 };
 
-template <int KS>
+template <int KS, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmO, const ApplyParams prm) {
-    using G = Geo<KS>;
+    using G = Geo<KS, PAIR>;
     constexpr int NS = G::kStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -122,7 +125,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 uint8_t* qs = stages + s * G::kStage;
                 mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
                 tma_load_4d_hint(qs, &tmQ, &full[s], 0, x0, y0, bh, pol_q);
-                tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::R, y0 - G::R, bh);
+                tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, bh);
                 ++issued;
             }
             if (*abort_flag) {
@@ -171,16 +174,33 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (bh != prev_bh) {
                 // every UMMA that read the previous S' has retired (its acc_full was waited on below)
                 prev_bh = bh;
-                const int i = et >> 2, part = et & 3;  // row i of S, 16 columns part*16 ..
-                const float4* src = reinterpret_cast<const float4*>(prm.state + (size_t)(prm.bh0 + bh) * prm.P * (kD * kD + kD) + i * kD + part * 16);
+                const int i = et >> 2, part = et & 3;  // row i of the operand, 16 columns part*16 ..
+                const float* st = prm.state + (size_t)(prm.bh0 + bh) * prm.P * (kD * kD + kD);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    float4 lo = __ldg(src + 2 * c), hi = __ldg(src + 2 * c + 1);
-                    for (int pp = 1; pp < prm.P; ++pp) {  // fixed order: bitwise reproducible
-                        const float4 l2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c);
-                        const float4 h2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c + 1);
-                        lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
-                        hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
+                    float4 lo, hi;
+                    if (!PAIR) {
+                        const float4* src = reinterpret_cast<const float4*>(st + i * kD + part * 16);
+                        lo = __ldg(src + 2 * c); hi = __ldg(src + 2 * c + 1);
+                        for (int pp = 1; pp < prm.P; ++pp) {  // fixed order: bitwise reproducible
+                            const float4 l2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c);
+                            const float4 h2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c + 1);
+                            lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
+                            hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
+                        }
+                    } else {
+                        // operand = blockdiag(S32, S32) with S32 = block(0,0) + block(1,1) of the paired sums
+                        const int col = part * 16 + c * 8;  // first of 8 columns
+                        if ((i < 32) == (col < 32)) {
+                            const int a = i & 31, bcol = col & 31;
+                            const float4* s0 = reinterpret_cast<const float4*>(st + a * kD + bcol);
+                            const float4* s1 = reinterpret_cast<const float4*>(st + (32 + a) * kD + 32 + bcol);
+                            const float4 l0 = __ldg(s0), h0 = __ldg(s0 + 1), l1 = __ldg(s1), h1 = __ldg(s1 + 1);
+                            lo = make_float4(l0.x + l1.x, l0.y + l1.y, l0.z + l1.z, l0.w + l1.w);
+                            hi = make_float4(h0.x + h1.x, h0.y + h1.y, h0.z + h1.z, h0.w + h1.w);
+                        } else {
+                            lo = make_float4(0.f, 0.f, 0.f, 0.f); hi = lo;
+                        }
                     }
                     uint4 o;
                     o.x = pack_bf16x2(lo.x * kInvPi, lo.y * kInvPi); o.y = pack_bf16x2(lo.z * kInvPi, lo.w * kInvPi);
@@ -224,7 +244,8 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             // barrier makes both halves of every row's sum of squares visible
             if (it > 0 && leader) tma_store_wait_read();
             named_barrier_sync(1, kEpiThreads);
-            const float rq = rsqrtf(fmaxf(rq_s[row] + rq_s[kTile + row], prm.eps2));
+            const float rq = PAIR ? rsqrtf(fmaxf(rq_s[half * kTile + row], prm.eps2))   // half row = one token
+                                  : rsqrtf(fmaxf(rq_s[row] + rq_s[kTile + row], prm.eps2));
             const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
             uint8_t* orow = out_s + row * 128;
 #pragma unroll
@@ -262,12 +283,22 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const int bh = (g_begin + it) / tiles_per_bh;
             if (bh != prev_bh) {
                 prev_bh = bh;
-                const int gbh = prm.bh0 + bh, ch = (gbh % prm.H) * kD + 2 * lane;
-                const float* sv = prm.state + (size_t)gbh * prm.P * (kD * kD + kD) + kD * kD + 2 * lane;
-                float s0 = __ldg(sv), s1 = __ldg(sv + 1);
-                for (int pp = 1; pp < prm.P; ++pp) {
-                    s0 += __ldg(sv + pp * (kD * kD + kD));
-                    s1 += __ldg(sv + pp * (kD * kD + kD) + 1);
+                // this lane's channel pair: 2*lane of 64 channels, or (PAIR) 2*(lane & 15) of 32 channels
+                // for the token of parity lane >> 4
+                const int gbh = prm.bh0 + bh;
+                const int cp2 = PAIR ? 2 * (lane & 15) : 2 * lane;
+                const int ch = (gbh % prm.H) * (PAIR ? 32 : kD) + cp2;
+                const float* sv = prm.state + (size_t)gbh * prm.P * (kD * kD + kD) + kD * kD;
+                float s0, s1;
+                if (PAIR) {  // token sum = sum of the two halves of the paired sums
+                    s0 = __ldg(sv + cp2) + __ldg(sv + 32 + cp2);
+                    s1 = __ldg(sv + cp2 + 1) + __ldg(sv + 32 + cp2 + 1);
+                } else {
+                    s0 = __ldg(sv + cp2); s1 = __ldg(sv + cp2 + 1);
+                    for (int pp = 1; pp < prm.P; ++pp) {
+                        s0 += __ldg(sv + pp * (kD * kD + kD) + cp2);
+                        s1 += __ldg(sv + pp * (kD * kD + kD) + cp2 + 1);
+                    }
                 }
                 cinit.x = 0.5f * s0; cinit.y = 0.5f * s1;
                 if (prm.bias) { cinit.x += __bfloat162float(prm.bias[ch]); cinit.y += __bfloat162float(prm.bias[ch + 1]); }
@@ -280,30 +311,41 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             if (!mbar_wait(&full[s], use & 1, abort_flag, prm.status, kBit)) break;
             if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
-            const uint8_t* vh = stages + s * G::kStage + kQBytes + ((2 * cw) * G::HX + xh * kCX) * 128 + lane * 4;
+            // Window of KS tokens per halo row, sliding along x.  Token t (relative to the first token this
+            // lane needs) sits U bytes after token t-1: U = 128, one token per column, or (PAIR) 64.
+            // One output column advances the window by STEP tokens (2 when PAIR: the lane's token keeps
+            // its parity).  Slot of token t in the rotating window: t % KS (t is a compile-time value).
+            constexpr int U = PAIR ? 64 : 128, STEP = PAIR ? 2 : 1;
+            const int tok0 = PAIR ? 2 * (xh * kCX + G::HC) + (lane >> 4) - R : xh * kCX;
+            const uint8_t* vh = stages + s * G::kStage + kQBytes + (2 * cw) * G::HX * 128 + tok0 * U +
+                                (PAIR ? (lane & 15) * 4 : lane * 4);
             uint8_t* so = stg + b * kStgBytes + ((2 * cw) * kTX + xh * kCX) * kStgStride + lane * 8;
-            float2 win[ROWS][KS];  // window columns x .. x+KS-1, rotating
+            float2 win[ROWS][KS];
 #pragma unroll
-            for (int dx = 0; dx < KS - 1; ++dx)
+            for (int t = 0; t < KS - STEP; ++t)
 #pragma unroll
                 for (int r = 0; r < ROWS; ++r) {
-                    const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + (r * G::HX + dx) * 128);
-                    win[r][dx] = make_float2(bf16lo(wv), bf16hi(wv));
+                    const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + r * G::HX * 128 + t * U);
+                    win[r][t % KS] = make_float2(bf16lo(wv), bf16hi(wv));
                 }
 #pragma unroll
             for (int x = 0; x < kCX; ++x) {
 #pragma unroll
-                for (int r = 0; r < ROWS; ++r) {
-                    const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + (r * G::HX + x + KS - 1) * 128);
-                    win[r][(x + KS - 1) % KS] = make_float2(bf16lo(wv), bf16hi(wv));
+                for (int n = 0; n < STEP; ++n) {
+                    const int t = STEP * x + KS - STEP + n;  // compile-time after unrolling
+#pragma unroll
+                    for (int r = 0; r < ROWS; ++r) {
+                        const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + r * G::HX * 128 + t * U);
+                        win[r][t % KS] = make_float2(bf16lo(wv), bf16hi(wv));
+                    }
                 }
                 float2 a0 = cinit, a1 = cinit;
 #pragma unroll
                 for (int dy = 0; dy < KS; ++dy)
 #pragma unroll
                     for (int dx = 0; dx < KS; ++dx) {
-                        a0 = ffma2(wreg[dy][dx], win[dy][(x + dx) % KS], a0);
-                        a1 = ffma2(wreg[dy][dx], win[dy + 1][(x + dx) % KS], a1);
+                        a0 = ffma2(wreg[dy][dx], win[dy][(STEP * x + dx) % KS], a0);
+                        a1 = ffma2(wreg[dy][dx], win[dy + 1][(STEP * x + dx) % KS], a1);
                     }
                 *reinterpret_cast<float2*>(so + x * kStgStride) = a0;
                 *reinterpret_cast<float2*>(so + (kTX + x) * kStgStride) = a1;
@@ -317,11 +359,12 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int KS>
+template <int KS, bool PAIR>
 cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigned* status, cudaStream_t st) {
-    using G = Geo<KS>;
+    using G = Geo<KS, PAIR>;
     CUtensorMap tmQ, tmV, tmO;
-    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)p.gridW, (uint64_t)p.gridH, (uint64_t)p.BH};
+    const int cols = PAIR ? p.gridW / 2 : p.gridW;  // 128-byte columns per grid row
+    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)cols, (uint64_t)p.gridH, (uint64_t)p.BH};
     const uint32_t box[4] = {kD, kTX, kTY, 1};
     const uint32_t boxv[4] = {kD, (uint32_t)G::HX, (uint32_t)G::HY, 1};
     if (!make_tensor_map_bf16(&tmQ, p.q, 4, dims, box, true) || !make_tensor_map_bf16(&tmO, p.out, 4, dims, box, true) ||
@@ -333,12 +376,12 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.H = p.H; prm.bh0 = 0;
-    prm.tilesX = (p.gridW + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
+    prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
     prm.eps2 = p.eps2; prm.status = status;
-    static bool attr_set = false;  // one flag per KS instantiation
+    static bool attr_set = false;  // one flag per instantiation
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_apply_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmem);
+        cudaError_t e = cudaFuncSetAttribute(tc_apply_kernel<KS, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -351,13 +394,17 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS>, tmQ, tmV, tmO, prm);
+    return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS, PAIR>, tmQ, tmV, tmO, prm);
 }
 
 }  // namespace
 
 cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st) {
-    return p.ksize == 3 ? launch_apply_ks<3>(p, partial, P, status, st) : launch_apply_ks<5>(p, partial, P, status, st);
+    if (p.d == 32)
+        return p.ksize == 3 ? launch_apply_ks<3, true>(p, partial, P, status, st)
+                            : launch_apply_ks<5, true>(p, partial, P, status, st);
+    return p.ksize == 3 ? launch_apply_ks<3, false>(p, partial, P, status, st)
+                        : launch_apply_ks<5, false>(p, partial, P, status, st);
 }
 
 }  // namespace tc

@@ -9,14 +9,20 @@ namespace {
 constexpr int kStateTile = 128;  // tokens per UMMA stage of the state kernel
 }
 
+// bf16 with head width 64, or head width 32 on a grid of even width (two tokens share one
+// 128-byte row there); 3x3 or 5x5 filters.
 bool supports(const Problem& p) {
-    return p.bf16 && p.d == 64 && (p.ksize == 3 || p.ksize == 5);
+    if (!p.bf16 || (p.ksize != 3 && p.ksize != 5)) return false;
+    return p.d == 64 || (p.d == 32 && p.gridW % 2 == 0);
 }
+
+int rows_per_head(int N, int d) { return d == 32 ? N / 2 : N; }
 
 // Two state CTAs fit on an SM: as many splits as keep all CTAs of the launch resident at once
 // (2 x 148), every split non-empty, at most 64 splits.
 int choose_splits(int BH, int N) {
     const int tiles = (N + kStateTile - 1) / kStateTile;
+    if (tiles < 1) return 1;
     int P = (2 * 148) / BH;
     if (P > tiles) P = tiles;
     if (P > 64) P = 64;
@@ -28,7 +34,7 @@ int choose_splits(int BH, int N) {
 cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
-    const int tiles = (p.N + kStateTile - 1) / kStateTile;
+    const int tiles = (rows_per_head(p.N, p.d) + kStateTile - 1) / kStateTile;
     const int per = (tiles + P - 1) / P;
     cudaError_t e = launch_state(p, ws_partial, ws_state, counters, P, per, status, stream);
     if (e != cudaSuccess) return e;

@@ -13,8 +13,15 @@ constexpr int kCountersPerHead = 17;
 bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
                           const uint32_t* box, bool swizzle128);
 
-// True when the tensor-core kernels can take this problem (bf16, d = 64, 3x3 or 5x5 filters).
+// True when the tensor-core kernels can take this problem (bf16; d = 64, or d = 32 with even gridW;
+// 3x3 or 5x5 filters).
 bool supports(const Problem& p);
+
+// 128-byte rows per (b,h): N for d = 64, N / 2 for d = 32 (two tokens per row).
+int rows_per_head(int N, int d);
+
+// Words of one (b,h) state as the tensor-core kernels store it (always the 64-wide form).
+constexpr int kStateWords = 64 * 64 + 64;
 
 // Token splits of the tensor-core state kernel and the workspace words it needs beyond the state.
 int choose_splits(int BH, int N);

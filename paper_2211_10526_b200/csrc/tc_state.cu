@@ -25,6 +25,12 @@ constexpr int kTmemCols = 64;
 constexpr int kGroup = 4;                    // splits per first-level reduction group
 constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
+// PAIR = true serves head width 32: the [N][32] tensors are viewed as [N/2][64], one 128-byte row
+// holding two consecutive tokens.  The same contraction then yields the four 32 x 32 blocks
+// [k_even^T v_even, k_even^T v_odd; k_odd^T v_even, k_odd^T v_odd]; the state is the sum of the two
+// diagonal blocks (and s the sum of the two halves of row 64), which the apply kernel folds when it
+// reads them.  Each half row is normalised by its own token's norm.
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 2)
 tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 float* __restrict__ dst, float* __restrict__ final_state, unsigned* __restrict__ counters,
@@ -130,21 +136,30 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             if (!ok) break;
             uint8_t* row = smem + s * kStageBytes + t * 128;
             uint4 c[8];
-            float ss = 0.f;
+            float ssa = 0.f, ssb = 0.f;  // first / second half of the row (two tokens when PAIR)
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 c[j] = *reinterpret_cast<const uint4*>(row + ((j ^ (t & 7)) << 4));
                 const uint32_t w[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
+                float part = 0.f;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const float lo = bf16lo(w[e]), hi = bf16hi(w[e]);
-                    ss = fmaf(lo, lo, ss);
-                    ss = fmaf(hi, hi, ss);
+                    part = fmaf(lo, lo, part);
+                    part = fmaf(hi, hi, part);
                 }
+                if (j < 4) ssa += part; else ssb += part;
             }
-            const float rk = 1.0f / sqrtf(fmaxf(ss, eps2));
+            float rka, rkb;
+            if (PAIR) {
+                rka = 1.0f / sqrtf(fmaxf(ssa, eps2));
+                rkb = 1.0f / sqrtf(fmaxf(ssb, eps2));
+            } else {
+                rka = rkb = 1.0f / sqrtf(fmaxf(ssa + ssb, eps2));
+            }
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
+                const float rk = j < 4 ? rka : rkb;
                 uint4 o;
                 o.x = pack_bf16x2(bf16lo(c[j].x) * rk, bf16hi(c[j].x) * rk);
                 o.y = pack_bf16x2(bf16lo(c[j].y) * rk, bf16hi(c[j].y) * rk);
@@ -260,19 +275,28 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
 cudaError_t launch_state(const Problem& p, float* partial, float* final_state, unsigned* counters, int P,
                          int tiles_per_cta, unsigned* status, cudaStream_t st) {
+    const bool pair = (p.d == 32);
+    const int rows = pair ? p.N / 2 : p.N;  // 128-byte rows per (b,h)
     CUtensorMap tmK, tmV;
-    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)p.N, (uint64_t)p.BH};
+    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)rows, (uint64_t)p.BH};
     const uint32_t box[3] = {kD, kTile, 1};
     if (!make_tensor_map_bf16(&tmK, p.k, 3, dims, box, true) || !make_tensor_map_bf16(&tmV, p.v, 3, dims, box, true))
         return cudaErrorNotSupported;
     static bool attr_set = false;  // per process; the attribute belongs to the function, not to a call
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(tc_state_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc_state_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    tc_state_kernel<<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(
-        tmK, tmV, P > 1 ? partial : final_state, final_state, counters, p.N, tiles_per_cta, P, p.eps2, status);
+    float* dst = P > 1 ? partial : final_state;
+    if (pair)
+        tc_state_kernel<true><<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(
+            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.eps2, status);
+    else
+        tc_state_kernel<false><<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(
+            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.eps2, status);
     return cudaGetLastError();
 }
 

@@ -46,6 +46,8 @@ def test_error_strings_and_workspace_query_need_no_gpu():
     assert "unknown" in b.error_string(-99)
     # state + no partials for a small grid: header + BH * (d*d + d) floats
     assert b.castling_attn_workspace_bytes(2, 4, 14, 14, 32, b.CASTLING_F32) == 4 * (64 + 8 * (32 * 32 + 32))
+    # bf16 with d = 32 may run the tensor-core kernels, which keep 64-wide states
+    assert b.castling_attn_workspace_bytes(2, 4, 14, 14, 32, b.CASTLING_BF16) >= 4 * (64 + 8 * (64 * 64 + 64))
     big = b.castling_attn_workspace_bytes(2, 8, 256, 256, 64, b.CASTLING_BF16)
     assert big > 4 * (64 + 16 * (64 * 64 + 64))  # token range is split: partial states too
     assert b.castling_attn_workspace_bytes(0, 4, 14, 14, 32, 0) == 0

@@ -193,7 +193,10 @@ def test_split_state_path_fp32():
 # ---------------------------------------------------------------------------
 TENSOR_SHAPES = [(2, 8, 32, 32, 64, 3), (1, 2, 8, 16, 64, 3), (1, 1, 1, 1, 64, 3), (2, 3, 14, 14, 64, 3),
                  (1, 2, 37, 53, 64, 3), (1, 2, 24, 40, 64, 5), (1, 1, 3, 130, 64, 3), (1, 1, 200, 5, 64, 5),
-                 (3, 5, 64, 64, 64, 3)]
+                 (3, 5, 64, 64, 64, 3),
+                 # head width 32 on even-width grids: two tokens share a 128-byte row
+                 (2, 4, 14, 14, 32, 3), (1, 2, 64, 64, 32, 5), (1, 3, 9, 22, 32, 3), (1, 1, 5, 2, 32, 5),
+                 (2, 2, 40, 66, 32, 5), (1, 1, 1, 2, 32, 3), (1, 2, 33, 34, 32, 3), (64, 12, 4, 4, 32, 3)]
 
 
 @pytest.mark.parametrize("shape", TENSOR_SHAPES, ids=lambda s: "x".join(map(str, s)))
@@ -214,7 +217,7 @@ def test_tensor_path_parity(shape):
         if path != binding.PATH_AUTO:
             assert used == path
         else:
-            assert used == binding.PATH_TENSOR, "bf16, d = 64 must run on the tensor-core kernels by default"
+            assert used == binding.PATH_TENSOR, "these shapes must run on the tensor-core kernels by default"
         errs[path] = rel_err(out, ref)
     assert max(errs.values()) <= TOL["bf16"], errs
 
@@ -243,6 +246,36 @@ def test_tensor_path_term_isolation():
     c = base(604)
     c.q[0, 0, 5] = 0; c.k[1, 1, 17] = 0
     check(c, force_path=binding.PATH_TENSOR)
+
+
+def test_tensor_path_term_isolation_head_width_32():
+    from paper_2211_10526_b200 import binding
+    base = lambda seed, ks: workloads.custom_call(2, 2, 24, 20, 32, ks, "bf16", seed=seed)
+    for ks in (3, 5):
+        c = base(611, ks)   # linear term alone
+        v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+        c.dw_weight.zero_(); c.dw_bias.zero_()
+        check(c, force_path=binding.PATH_TENSOR)
+        c = base(612, ks)   # 1/2 sum (constant V)
+        c.v[:] = c.v[:, :, :1, :].clone()
+        c.dw_weight.zero_(); c.dw_bias.zero_()
+        check(c, force_path=binding.PATH_TENSOR)
+        c = base(613, ks)   # convolution alone
+        v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+        c.dw_weight = (c.dw_weight.float() * 30).to(torch.bfloat16)
+        c.k.zero_()
+        check(c, force_path=binding.PATH_TENSOR)
+
+
+def test_odd_grid_width_head_width_32_uses_cuda_cores():
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    c = workloads.custom_call(2, 2, 7, 7, 32, 3, "bf16", seed=614)
+    dev = torch.device("cuda:0")
+    with CastlingAttn(ksize=3) as attn:
+        attn.forward(*[t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)], 7, 7)
+        torch.cuda.synchronize()
+        assert attn.last_path()[0] == binding.PATH_SIMT
+    check(c)
 
 
 def test_tensor_path_rejects_what_it_cannot_take():
