@@ -175,7 +175,8 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     if (rc != CASTLING_OK) return rc;
     const bool tensor_ok = castling::tc::supports(p);
     if (h->cfg.force_path == CASTLING_PATH_TENSOR && !tensor_ok) return CASTLING_ERR_UNSUPPORTED;
-    const bool use_tensor = tensor_ok && h->cfg.force_path != CASTLING_PATH_SIMT;
+    const bool use_tensor = h->cfg.force_path == CASTLING_PATH_TENSOR ||
+                            (h->cfg.force_path == CASTLING_PATH_AUTO && castling::tc::preferred(p));
     float* state = h->ws + castling::kHeaderWords;
     float* partial = state + (size_t)p.BH * (use_tensor ? (size_t)castling::tc::kStateWords : castling::state_words(p.d));
     int launches = 0;

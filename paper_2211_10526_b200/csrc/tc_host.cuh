@@ -17,6 +17,9 @@ bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const ui
 // 3x3 or 5x5 filters).
 bool supports(const Problem& p);
 
+// True when automatic dispatch should pick them (enough rows per (b,h) to fill their tiles).
+bool preferred(const Problem& p);
+
 // 128-byte rows per (b,h): N for d = 64, N / 2 for d = 32 (two tokens per row).
 int rows_per_head(int N, int d);
 
