@@ -21,7 +21,7 @@ constexpr int kTileBytes = kTile * kD * 2;   // 16 KiB per operand tile
 constexpr int kStageBytes = 2 * kTileBytes;  // K then V
 constexpr int kOnesBytes = 2048;             // 16 token rows x 128 B: feature 64 = 1, 65..127 = 0
 constexpr int kThreads = 192;                // warp 0 TMA, warp 1 UMMA, warps 2..5 scale + epilogue
-constexpr int kTmemCols = 64;
+constexpr int kTmemCols = 128;                // two 64-column accumulators: a CTA may serve several (b,h)
 constexpr int kGroup = 4;                    // splits per first-level reduction group
 constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
@@ -34,25 +34,34 @@ template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 2)
 tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 float* __restrict__ dst, float* __restrict__ final_state, unsigned* __restrict__ counters,
-                int N, int tiles_per_cta, int P, float eps2, unsigned* status) {
+                int N, int tiles_per_cta, int P, int BH, int items_per_cta, float eps2, unsigned* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* ones = smem + kStages * kStageBytes;
     uint64_t* full = reinterpret_cast<uint64_t*>(ones + kOnesBytes);  // TMA bytes landed
     uint64_t* scaled = full + kStages;                                // K rows normalised (128 arrivals)
     uint64_t* empty = scaled + kStages;                               // UMMAs of the stage retired
-    uint64_t* accum = empty + kStages;                                // whole accumulation retired
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+    uint64_t* accum = empty + kStages;                                // [2] whole accumulation of an item retired
+    uint64_t* acc_free = accum + 2;                                   // [2] accumulator read out (128 arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_free + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int p = blockIdx.x % P, bh = blockIdx.x / P;
+    // Work items.  With P > 1 a CTA serves one (b,h, split).  With P == 1 (many heads, few tokens) a CTA
+    // serves items_per_cta consecutive (b,h) one after another, so that barrier set-up, TMEM allocation
+    // and the first load latency are paid once and the loads of the next (b,h) overlap the current one.
     const int total_tiles = (N + kTile - 1) / kTile;
+    const int p = (P > 1) ? blockIdx.x % P : 0;
+    const int bh0 = (P > 1) ? blockIdx.x / P : blockIdx.x * items_per_cta;
+    const int n_items = (P > 1) ? 1 : min(items_per_cta, BH - bh0);
     const int t_begin = p * tiles_per_cta;
-    const int n_tiles = min(total_tiles, t_begin + tiles_per_cta) - t_begin;
-    float* out = dst + ((size_t)bh * P + p) * (kD * kD + kD);
-    if (n_tiles <= 0) {  // the host never makes such a split; keep the partial well defined anyway
-        for (int i = tid; i < kD * kD + kD; i += kThreads) out[i] = 0.f;
+    const int n_tiles = min(total_tiles, t_begin + tiles_per_cta) - t_begin;  // per item
+    const int bh = bh0;  // the (b,h) of the split reduction below (P > 1: the only item)
+    if (n_tiles <= 0 || n_items <= 0) {  // the host never makes such a CTA; keep the partial well defined anyway
+        if (P > 1) {
+            float* out = dst + ((size_t)bh * P + p) * (kD * kD + kD);
+            for (int i = tid; i < kD * kD + kD; i += kThreads) out[i] = 0.f;
+        }
         return;
     }
 
@@ -63,7 +72,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             mbar_init(&scaled[s], kTile);
             mbar_init(&empty[s], 1);
         }
-        mbar_init(accum, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&accum[b], 1); mbar_init(&acc_free[b], kTile); }
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmK);
@@ -90,14 +99,16 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             int issued = 0;
             // K is read once; V is read again by the apply kernel: keep it in L2 as long as possible
             const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_last();
-            for (int it = 0; it < n_tiles; ++it) {
-                const int s = it % kStages, use = it / kStages;
-                if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, status, kStatusStateTimeout)) break;
-                uint8_t* ks = smem + s * kStageBytes;
-                mbar_expect_tx(&full[s], kStageBytes);
-                tma_load_3d_hint(ks, &tmK, &full[s], 0, (t_begin + it) * kTile, bh, pol_k);
-                tma_load_3d_hint(ks + kTileBytes, &tmV, &full[s], 0, (t_begin + it) * kTile, bh, pol_v);
-                ++issued;
+            bool ok = true;
+            for (int item = 0; item < n_items && ok; ++item) {
+                for (int it = 0; it < n_tiles; ++it, ++issued) {
+                    const int s = issued % kStages, use = issued / kStages;
+                    if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, status, kStatusStateTimeout)) { ok = false; break; }
+                    uint8_t* ks = smem + s * kStageBytes;
+                    mbar_expect_tx(&full[s], kStageBytes);
+                    tma_load_3d_hint(ks, &tmK, &full[s], 0, (t_begin + it) * kTile, bh0 + item, pol_k);
+                    tma_load_3d_hint(ks + kTileBytes, &tmV, &full[s], 0, (t_begin + it) * kTile, bh0 + item, pol_v);
+                }
             }
             if (*abort_flag) {
                 // giving up: let copies already in flight land before the CTA's shared memory goes away
@@ -110,77 +121,46 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             constexpr uint32_t idesc = umma_idesc_bf16(128, kD, true, true);
             const uint32_t ones_addr = smem_u32(ones);
             bool ok = true;
-            for (int it = 0; it < n_tiles && ok; ++it) {
-                const int s = it % kStages, use = it / kStages;
-                ok = mbar_wait(&scaled[s], use & 1, abort_flag, status, kStatusStateTimeout);
-                if (!ok) break;
-                tcgen05_fence_after_sync();
-                const uint32_t ka = smem_u32(smem + s * kStageBytes), va = ka + kTileBytes;
+            int gt = 0;  // tiles issued so far, over all items
+            for (int item = 0; item < n_items && ok; ++item) {
+                const int buf = item & 1;
+                if (item >= 2) ok = mbar_wait(&acc_free[buf], ((item >> 1) - 1) & 1, abort_flag, status, kStatusStateTimeout);
+                for (int it = 0; it < n_tiles && ok; ++it, ++gt) {
+                    const int s = gt % kStages, use = gt / kStages;
+                    ok = mbar_wait(&scaled[s], use & 1, abort_flag, status, kStatusStateTimeout);
+                    if (!ok) break;
+                    tcgen05_fence_after_sync();
+                    const uint32_t ka = smem_u32(smem + s * kStageBytes), va = ka + kTileBytes;
 #pragma unroll
-                for (int j = 0; j < kTile / 16; ++j) {  // one UMMA per 16 tokens (K = 16)
-                    const uint32_t a0 = ka + j * 2048, b0 = va + j * 2048;
-                    const uint64_t a = umma_desc_sw128(a0, ones_addr - a0, 1024);
-                    const uint64_t b = umma_desc_sw128(b0, 0, 1024);
-                    umma_bf16(tmem, a, b, idesc, (it | j) != 0);
+                    for (int j = 0; j < kTile / 16; ++j) {  // one UMMA per 16 tokens (K = 16)
+                        const uint32_t a0 = ka + j * 2048, b0 = va + j * 2048;
+                        const uint64_t a = umma_desc_sw128(a0, ones_addr - a0, 1024);
+                        const uint64_t b = umma_desc_sw128(b0, 0, 1024);
+                        umma_bf16(tmem + buf * kD, a, b, idesc, (it | j) != 0);
+                    }
+                    umma_commit(&empty[s]);
                 }
-                umma_commit(&empty[s]);
+                if (ok) umma_commit(&accum[buf]);
             }
-            if (ok) umma_commit(accum);
         }
     } else {
         const int t = tid - 64;  // token row of the stage handled by this thread
-        bool ok = true;
-        for (int it = 0; it < n_tiles; ++it) {
-            const int s = it % kStages, use = it / kStages;
-            ok = mbar_wait(&full[s], use & 1, abort_flag, status, kStatusStateTimeout);
-            if (!ok) break;
-            uint8_t* row = smem + s * kStageBytes + t * 128;
-            uint4 c[8];
-            float ssa = 0.f, ssb = 0.f;  // first / second half of the row (two tokens when PAIR)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                c[j] = *reinterpret_cast<const uint4*>(row + ((j ^ (t & 7)) << 4));
-                const uint32_t w[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
-                float part = 0.f;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float lo = bf16lo(w[e]), hi = bf16hi(w[e]);
-                    part = fmaf(lo, lo, part);
-                    part = fmaf(hi, hi, part);
-                }
-                if (j < 4) ssa += part; else ssb += part;
-            }
-            float rka, rkb;
-            if (PAIR) {
-                rka = 1.0f / sqrtf(fmaxf(ssa, eps2));
-                rkb = 1.0f / sqrtf(fmaxf(ssb, eps2));
-            } else {
-                rka = rkb = 1.0f / sqrtf(fmaxf(ssa + ssb, eps2));
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float rk = j < 4 ? rka : rkb;
-                uint4 o;
-                o.x = pack_bf16x2(bf16lo(c[j].x) * rk, bf16hi(c[j].x) * rk);
-                o.y = pack_bf16x2(bf16lo(c[j].y) * rk, bf16hi(c[j].y) * rk);
-                o.z = pack_bf16x2(bf16lo(c[j].z) * rk, bf16hi(c[j].z) * rk);
-                o.w = pack_bf16x2(bf16lo(c[j].w) * rk, bf16hi(c[j].w) * rk);
-                *reinterpret_cast<uint4*>(row + ((j ^ (t & 7)) << 4)) = o;
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(&scaled[s]);
-        }
-        // epilogue: accumulator rows 0..63 are S, row 64 is s; a warp reads TMEM lanes 32*(warp%4)..+31
         const int quarter = warp & 3;
-        if (ok && quarter < 3) {
-            ok = mbar_wait(accum, 0, abort_flag, status, kStatusStateTimeout);
-            if (ok) {
-                tcgen05_fence_after_sync();
+        bool ok = true;
+        // read the finished accumulator of `item` out of TMEM: rows 0..63 are S, row 64 is s; a warp reads
+        // TMEM lanes 32*(warp%4)..+31.  Runs one item late, so that the UMMAs of an item overlap the
+        // normalisation of the next item's tiles.
+        auto flush = [&](int item) -> bool {
+            const int buf = item & 1;
+            if (!mbar_wait(&accum[buf], (item >> 1) & 1, abort_flag, status, kStatusStateTimeout)) return false;
+            tcgen05_fence_after_sync();
+            if (quarter < 3) {
+                float* out = dst + ((size_t)(bh0 + item) * P + p) * (kD * kD + kD);
                 const int row = quarter * 32 + lane;
 #pragma unroll
                 for (int cc = 0; cc < kD / 16; ++cc) {
                     float v[16];
-                    tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + cc * 16, v);
+                    tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + buf * kD + cc * 16, v);
                     tmem_ld_wait();
                     if (row <= kD) {
                         float4* o4 = reinterpret_cast<float4*>(out + row * kD + cc * 16);  // row 64 lands on s
@@ -189,7 +169,55 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                 }
             }
+            tcgen05_fence_before_sync();
+            mbar_arrive(&acc_free[buf]);
+            return true;
+        };
+        int gt = 0;  // tiles handled so far, over all items
+        for (int item = 0; item < n_items && ok; ++item) {
+            for (int it = 0; it < n_tiles; ++it, ++gt) {
+                const int s = gt % kStages, use = gt / kStages;
+                ok = mbar_wait(&full[s], use & 1, abort_flag, status, kStatusStateTimeout);
+                if (!ok) break;
+                uint8_t* row = smem + s * kStageBytes + t * 128;
+                uint4 c[8];
+                float ssa = 0.f, ssb = 0.f;  // first / second half of the row (two tokens when PAIR)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    c[j] = *reinterpret_cast<const uint4*>(row + ((j ^ (t & 7)) << 4));
+                    const uint32_t w[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
+                    float part = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float lo = bf16lo(w[e]), hi = bf16hi(w[e]);
+                        part = fmaf(lo, lo, part);
+                        part = fmaf(hi, hi, part);
+                    }
+                    if (j < 4) ssa += part; else ssb += part;
+                }
+                float rka, rkb;
+                if (PAIR) {
+                    rka = 1.0f / sqrtf(fmaxf(ssa, eps2));
+                    rkb = 1.0f / sqrtf(fmaxf(ssb, eps2));
+                } else {
+                    rka = rkb = 1.0f / sqrtf(fmaxf(ssa + ssb, eps2));
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float rk = j < 4 ? rka : rkb;
+                    uint4 o;
+                    o.x = pack_bf16x2(bf16lo(c[j].x) * rk, bf16hi(c[j].x) * rk);
+                    o.y = pack_bf16x2(bf16lo(c[j].y) * rk, bf16hi(c[j].y) * rk);
+                    o.z = pack_bf16x2(bf16lo(c[j].z) * rk, bf16hi(c[j].z) * rk);
+                    o.w = pack_bf16x2(bf16lo(c[j].w) * rk, bf16hi(c[j].w) * rk);
+                    *reinterpret_cast<uint4*>(row + ((j ^ (t & 7)) << 4)) = o;
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(&scaled[s]);
+            }
+            if (ok && item > 0) ok = flush(item - 1);
         }
+        if (ok) ok = flush(n_items - 1);
     }
     tcgen05_fence_before_sync();
     __threadfence();  // this split's partial state is visible device-wide before the arrival below
@@ -291,12 +319,18 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
         attr_set = true;
     }
     float* dst = P > 1 ? partial : final_state;
+    // P == 1: a CTA serves several consecutive (b,h); at most 296 CTAs (two per SM) so all are resident
+    int grid = p.BH * P, items = 1;
+    if (P == 1 && p.BH > 296) {
+        items = (p.BH + 295) / 296;
+        grid = (p.BH + items - 1) / items;
+    }
     if (pair)
-        tc_state_kernel<true><<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(
-            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.eps2, status);
+        tc_state_kernel<true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(
+            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, items, p.eps2, status);
     else
-        tc_state_kernel<false><<<(unsigned)(p.BH * P), kThreads, kSmemBytes, st>>>(
-            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.eps2, status);
+        tc_state_kernel<false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(
+            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, items, p.eps2, status);
     return cudaGetLastError();
 }
 
