@@ -116,8 +116,11 @@ CASTLING_API int castling_attn_forward(castling_attn_t* handle,
  * castling_attn_forward_host: the same computation with every tensor in HOST memory.
  * Copies q, k, v, dw_weight and dw_bias to handle-owned device staging buffers on
  * `stream`, runs the forward pass, copies `out` back and synchronises the stream
- * before returning, so on return `out` holds the result.  Pinned host memory makes the
- * copies asynchronous to each other; pageable memory also works.  Shapes, dtype and
+ * before returning, so on return `out` holds the result.  Large problems are cut into chunks
+ * of whole (b,h) planes whose uploads, kernels and downloads overlap on two internal copy streams
+ * (created on first use); that needs pinned host memory to be effective, pageable memory also
+ * works.  Because a chunk is a smaller problem, its token splits and hence the fp32 summation
+ * order may differ from one castling_attn_forward call on the whole batch (same tolerance).  Shapes, dtype and
  * errors as for castling_attn_forward (alignment is not required of host pointers).
  */
 CASTLING_API int castling_attn_forward_host(castling_attn_t* handle,

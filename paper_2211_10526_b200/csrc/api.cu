@@ -18,6 +18,10 @@ struct castling_attn {
     size_t counters_cap = 0;
     char* stage = nullptr;      // device staging for castling_attn_forward_host
     size_t stage_bytes = 0;
+    // castling_attn_forward_host pipelines batch chunks: copies in, kernels and copies out overlap
+    static constexpr int kMaxChunks = 8;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_end = nullptr, ev_in[kMaxChunks] = {}, ev_done[kMaxChunks] = {};
     int last_cuda_error = 0;
     int last_path = 0;
     int last_launches = 0;
@@ -130,6 +134,12 @@ int castling_attn_destroy(castling_attn_t* h) {
     if (h->ws) cudaFree(h->ws);
     if (h->stage) cudaFree(h->stage);
     if (h->counters) cudaFree(h->counters);
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
+    if (h->ev_start) cudaEventDestroy(h->ev_start);
+    if (h->ev_end) cudaEventDestroy(h->ev_end);
+    for (auto& e : h->ev_in) if (e) cudaEventDestroy(e);
+    for (auto& e : h->ev_done) if (e) cudaEventDestroy(e);
     for (auto& e : h->timer.ev)
         if (e) cudaEventDestroy(e);
     delete h;
@@ -203,7 +213,7 @@ Problem make_problem(const castling_attn* h, const void* q, const void* k, const
     Problem p;
     p.q = q; p.k = k; p.v = v; p.w = w; p.bias = bias; p.out = out;
     p.B = B; p.H = H; p.gridH = gridH; p.gridW = gridW; p.d = d; p.ksize = h->cfg.ksize;
-    p.N = gridH * gridW; p.BH = B * H;
+    p.N = gridH * gridW; p.BH = B * H; p.head0 = 0;
     p.bf16 = (dtype == CASTLING_BF16);
     p.eps2 = (float)(h->cfg.eps * h->cfg.eps);
     return p;
@@ -260,18 +270,74 @@ int castling_attn_forward_host(castling_attn_t* h, const void* q, const void* k,
     char* dw = dout + tb; char* db = dw + wb;
     const size_t t_exact = (size_t)B * H * gridH * gridW * d * eb;
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(dq, q, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
-    if ((e = cudaMemcpyAsync(dk, k, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
-    if ((e = cudaMemcpyAsync(dv, v, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
     if ((e = cudaMemcpyAsync(dw, dw_weight, (size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb,
                              cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
     if (dw_bias &&
         (e = cudaMemcpyAsync(db, dw_bias, (size_t)H * d * eb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
         return fail_cuda(h, e);
-    const Problem p = make_problem(h, dq, dk, dv, dw, dw_bias ? db : nullptr, dout, B, H, gridH, gridW, d, dtype);
-    rc = run_device(h, p, st);
-    if (rc != CASTLING_OK) return rc;
-    if ((e = cudaMemcpyAsync(out, dout, t_exact, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_cuda(h, e);
+
+    // Chunks of whole (b,h) planes, at least 8 MB of one tensor each: small problems go through in one piece.
+    const int BH = B * H;
+    const size_t plane_bytes = t_exact / BH;
+    int chunks = BH < castling_attn::kMaxChunks ? BH : castling_attn::kMaxChunks;
+    while (chunks > 1 && t_exact / chunks < ((size_t)8 << 20)) --chunks;
+    if (chunks <= 1) {
+        if ((e = cudaMemcpyAsync(dq, q, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaMemcpyAsync(dk, k, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaMemcpyAsync(dv, v, t_exact, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);
+        const Problem p = make_problem(h, dq, dk, dv, dw, dw_bias ? db : nullptr, dout, B, H, gridH, gridW, d, dtype);
+        rc = run_device(h, p, st);
+        if (rc != CASTLING_OK) return rc;
+        if ((e = cudaMemcpyAsync(out, dout, t_exact, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(h, e);
+        return CASTLING_OK;
+    }
+
+    // Pipeline: all chunk uploads queue on a copy stream; the kernels of chunk c wait for its upload on the
+    // caller's stream; its download runs on a second copy stream while later chunks upload and compute
+    // (PCIe is full duplex).  Streams and events are created on first use and kept in the handle.
+    if (!h->copy_in) {
+        if ((e = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaEventCreateWithFlags(&h->ev_end, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(h, e);
+        for (int c = 0; c < castling_attn::kMaxChunks; ++c) {
+            if ((e = cudaEventCreateWithFlags(&h->ev_in[c], cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(h, e);
+            if ((e = cudaEventCreateWithFlags(&h->ev_done[c], cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(h, e);
+        }
+    }
+    // the copy streams start after everything already queued on the caller's stream (filters included)
+    if ((e = cudaEventRecord(h->ev_start, st)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaStreamWaitEvent(h->copy_in, h->ev_start, 0)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaStreamWaitEvent(h->copy_out, h->ev_start, 0)) != cudaSuccess) return fail_cuda(h, e);
+    int b0[castling_attn::kMaxChunks + 1];
+    for (int c = 0; c <= chunks; ++c) b0[c] = (int)((long long)BH * c / chunks);
+    for (int c = 0; c < chunks; ++c) {
+        const size_t off = (size_t)b0[c] * plane_bytes, len = (size_t)(b0[c + 1] - b0[c]) * plane_bytes;
+        const char* hq = static_cast<const char*>(q); const char* hk = static_cast<const char*>(k);
+        const char* hv = static_cast<const char*>(v);
+        // K and V first: the state kernel needs them before the apply kernel needs Q
+        if ((e = cudaMemcpyAsync(dk + off, hk + off, len, cudaMemcpyHostToDevice, h->copy_in)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaMemcpyAsync(dv + off, hv + off, len, cudaMemcpyHostToDevice, h->copy_in)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaMemcpyAsync(dq + off, hq + off, len, cudaMemcpyHostToDevice, h->copy_in)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaEventRecord(h->ev_in[c], h->copy_in)) != cudaSuccess) return fail_cuda(h, e);
+    }
+    for (int c = 0; c < chunks; ++c) {
+        const size_t off = (size_t)b0[c] * plane_bytes, len = (size_t)(b0[c + 1] - b0[c]) * plane_bytes;
+        if ((e = cudaStreamWaitEvent(st, h->ev_in[c], 0)) != cudaSuccess) return fail_cuda(h, e);
+        Problem p = make_problem(h, dq + off, dk + off, dv + off, dw, dw_bias ? db : nullptr, dout + off,
+                                 1, H, gridH, gridW, d, dtype);
+        p.BH = b0[c + 1] - b0[c];   // a run of planes that may start and end inside a batch
+        p.head0 = b0[c] % H;
+        rc = run_device(h, p, st);
+        if (rc != CASTLING_OK) return rc;
+        if ((e = cudaEventRecord(h->ev_done[c], st)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaStreamWaitEvent(h->copy_out, h->ev_done[c], 0)) != cudaSuccess) return fail_cuda(h, e);
+        if ((e = cudaMemcpyAsync(static_cast<char*>(out) + off, dout + off, len, cudaMemcpyDeviceToHost, h->copy_out)) != cudaSuccess)
+            return fail_cuda(h, e);
+    }
+    if ((e = cudaEventRecord(h->ev_end, h->copy_out)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaStreamWaitEvent(st, h->ev_end, 0)) != cudaSuccess) return fail_cuda(h, e);
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(h, e);
     return CASTLING_OK;
 }

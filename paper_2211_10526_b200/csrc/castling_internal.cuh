@@ -21,7 +21,8 @@ struct Problem {
     void* out;
     int B, H, gridH, gridW, d, ksize;
     int N;             // gridH * gridW
-    int BH;            // B * H
+    int BH;            // B * H (the (b,h) planes of this call)
+    int head0;         // head index of plane 0: plane i uses the filters of head (head0 + i) % H
     bool bf16;
     float eps2;        // eps^2: the floor under the sum of squares
 };

@@ -165,7 +165,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __restrict__ w,
                   const T* __restrict__ bias, const float* __restrict__ state, T* __restrict__ out,
-                  int H, int gridH, int gridW, int ksize, float eps2) {
+                  int H, int head0, int gridH, int gridW, int ksize, float eps2) {
     constexpr int R = D / 16;
     constexpr int LDQ = D + 1;
     extern __shared__ __align__(16) float smem[];
@@ -178,7 +178,7 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
 
     const int N = gridH * gridW;
     const int tiles = (N + kApplyTile - 1) / kApplyTile;
-    const int bh = blockIdx.x / tiles, h = bh % H;
+    const int bh = blockIdx.x / tiles, h = (head0 + bh) % H;
     const int t0 = (blockIdx.x % tiles) * kApplyTile;
     const int valid = min(kApplyTile, N - t0);
     const float* st = state + (size_t)bh * (D * D + D);
@@ -283,7 +283,7 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     const unsigned grid = (unsigned)(p.BH * ((p.N + kApplyTile - 1) / kApplyTile));
     simt_apply_kernel<T, D><<<grid, kThreads, smem, stream>>>(
         static_cast<const T*>(p.q), static_cast<const T*>(p.v), static_cast<const T*>(p.w),
-        static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.gridH, p.gridW, p.ksize, p.eps2);
+        static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     timer->mark(stream, "simt_apply");

@@ -64,7 +64,7 @@ struct ApplyParams {
     int P;
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
-    int H, bh0, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
+    int H, head0, bh0, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
 };
@@ -287,7 +287,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 // for the token of parity lane >> 4
                 const int gbh = prm.bh0 + bh;
                 const int cp2 = PAIR ? 2 * (lane & 15) : 2 * lane;
-                const int ch = (gbh % prm.H) * (PAIR ? 32 : kD) + cp2;
+                const int ch = ((prm.head0 + gbh) % prm.H) * (PAIR ? 32 : kD) + cp2;
                 const float* sv = prm.state + (size_t)gbh * prm.P * (kD * kD + kD) + kD * kD;
                 float s0, s1;
                 if (PAIR) {  // token sum = sum of the two halves of the paired sums
@@ -375,7 +375,7 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.P = P;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
-    prm.H = p.H; prm.bh0 = 0;
+    prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
     prm.eps2 = p.eps2; prm.status = status;

@@ -174,3 +174,23 @@ def test_create_destroy_cycles():
     for _ in range(50):
         h = b.castling_attn_create(5)
         assert b.castling_attn_destroy(h) == b.OK
+
+
+def test_host_entry_point_pipelines_batch_chunks():
+    """Large host-side problems are uploaded, computed and downloaded in overlapping batch chunks."""
+    from paper_2211_10526_b200 import CastlingAttn
+    c = workloads.custom_call(4, 8, 128, 64, 64, 3, "bf16", seed=440)   # 33.5 MB per tensor -> four chunks
+    s = c.shape
+    pinned = [t.pin_memory() for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)]
+    out_h = torch.full_like(c.q, float("nan")).pin_memory()
+    with CastlingAttn(ksize=3) as attn:
+        for _ in range(2):
+            attn.forward_host(*pinned, s.gridH, s.gridW, out=out_h)
+        out_d = attn.forward(*_dev(c), s.gridH, s.gridW)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+    assert torch.isfinite(out_h.float()).all()
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, 3, threads=8)
+    for got in (out_h, out_d.cpu()):
+        err = np.max(np.abs(got.double().numpy() - ref)) / np.max(np.abs(ref))
+        assert err <= 2e-2
