@@ -26,14 +26,18 @@ constexpr int kTile = kTY * kTX;
 constexpr int kQBytes = kTile * kD * 2;     // 16 KiB
 constexpr int kStgStride = kD * 4 + 16;     // fp32 row + 16 B pad: conflict-free row-per-thread reads
 constexpr int kStgBytes = kTile * kStgStride;
-constexpr int kEpiWarps = 8, kConvWarps = 8;   // two warps per TMEM lane quarter / per pair of patch rows
-constexpr int kEpiThreads = kEpiWarps * 32, kConvThreads = kConvWarps * 32;
-constexpr int kThreads = 64 + kEpiThreads + kConvThreads;
+constexpr int kEpiWarps = 8;                   // two warps per TMEM lane quarter
+constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kTmemCols = 128;              // two 64-column accumulators
 
 // PAIR = true serves head width 32: a 128-byte row holds two horizontally adjacent tokens, so a
 // "column" of the patch is a token pair and the 8 x 16-column patch covers 8 x 32 tokens.
 template <int KS, bool PAIR> struct Geo {
+    // conv warps: each takes kConvRows patch rows x 8 columns.  3x3: 8 warps of 2 rows; 5x5: 4 warps of
+    // 4 rows (fewer redundant window loads, and the larger window fits the registers of 448 threads)
+    static constexpr int kConvRows = (KS == 3) ? 2 : 4;
+    static constexpr int kConvWarps = 2 * kTY / kConvRows, kConvThreads = kConvWarps * 32;
+    static constexpr int kThreads = 64 + kEpiThreads + kConvThreads;
     static constexpr int R = KS / 2;
     static constexpr int HC = PAIR ? (R + 1) / 2 : R;   // halo columns on each side
     static constexpr int HY = kTY + 2 * R, HX = kTX + 2 * HC;
@@ -70,7 +74,7 @@ struct ApplyParams {
 };
 
 template <int KS, bool PAIR>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__((Geo<KS, PAIR>::kThreads), 1)
 tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmO, const ApplyParams prm) {
     using G = Geo<KS, PAIR>;
@@ -99,8 +103,8 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int my_tiles = g_end - g_begin;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConvThreads + kEpiThreads + 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], kConvThreads); mbar_init(&buf_free[b], kEpiThreads); }
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], G::kConvThreads + kEpiThreads + 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], G::kConvThreads); mbar_init(&buf_free[b], kEpiThreads); }
         mbar_init(s_ready, kEpiThreads);
         *abort_flag = 0;
         mbar_fence_init();
@@ -273,7 +277,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ------- depthwise convolution: lane = channel pair, warp = two patch rows x eight columns -------
         const int cw = (warp - 2 - kEpiWarps) >> 1, xh = (warp - 2 - kEpiWarps) & 1;
         constexpr int kCX = kTX / 2;
-        constexpr int R = G::R, ROWS = 2 + 2 * R;
+        constexpr int R = G::R, RO = G::kConvRows, ROWS = RO + 2 * R;
         float2 wreg[KS][KS];
         float2 cinit = make_float2(0.f, 0.f);
         int prev_bh = -1;
@@ -317,9 +321,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             // its parity).  Slot of token t in the rotating window: t % KS (t is a compile-time value).
             constexpr int U = PAIR ? 64 : 128, STEP = PAIR ? 2 : 1;
             const int tok0 = PAIR ? 2 * (xh * kCX + G::HC) + (lane >> 4) - R : xh * kCX;
-            const uint8_t* vh = stages + s * G::kStage + kQBytes + (2 * cw) * G::HX * 128 + tok0 * U +
+            const uint8_t* vh = stages + s * G::kStage + kQBytes + (RO * cw) * G::HX * 128 + tok0 * U +
                                 (PAIR ? (lane & 15) * 4 : lane * 4);
-            uint8_t* so = stg + b * kStgBytes + ((2 * cw) * kTX + xh * kCX) * kStgStride + lane * 8;
+            uint8_t* so = stg + b * kStgBytes + ((RO * cw) * kTX + xh * kCX) * kStgStride + lane * 8;
             float2 win[ROWS][KS];
 #pragma unroll
             for (int t = 0; t < KS - STEP; ++t)
@@ -339,16 +343,18 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         win[r][t % KS] = make_float2(bf16lo(wv), bf16hi(wv));
                     }
                 }
-                float2 a0 = cinit, a1 = cinit;
+                float2 acc[RO];
+#pragma unroll
+                for (int r = 0; r < RO; ++r) acc[r] = cinit;
 #pragma unroll
                 for (int dy = 0; dy < KS; ++dy)
 #pragma unroll
-                    for (int dx = 0; dx < KS; ++dx) {
-                        a0 = ffma2(wreg[dy][dx], win[dy][(STEP * x + dx) % KS], a0);
-                        a1 = ffma2(wreg[dy][dx], win[dy + 1][(STEP * x + dx) % KS], a1);
-                    }
-                *reinterpret_cast<float2*>(so + x * kStgStride) = a0;
-                *reinterpret_cast<float2*>(so + (kTX + x) * kStgStride) = a1;
+                    for (int dx = 0; dx < KS; ++dx)
+#pragma unroll
+                        for (int r = 0; r < RO; ++r)
+                            acc[r] = ffma2(wreg[dy][dx], win[dy + r][(STEP * x + dx) % KS], acc[r]);
+#pragma unroll
+                for (int r = 0; r < RO; ++r) *reinterpret_cast<float2*>(so + (r * kTX + x) * kStgStride) = acc[r];
             }
             mbar_arrive(&empty[s]);      // the V patch of this stage is no longer needed
             mbar_arrive(&conv_full[b]);
@@ -389,7 +395,7 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     // programmatic dependent launch: this grid's prologue and first Q / V loads overlap the tail of
     // the state kernel; the warps that read its results wait for it (griddepcontrol.wait) first
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = G::kSmem; cfg.stream = st;
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(G::kThreads); cfg.dynamicSmemBytes = G::kSmem; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
