@@ -312,12 +312,13 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16 operands, fp32 accumulate" if s.dtype == "bf16" else "f32",
+            "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32",
             "data": "synthetic",
             "config": {"workload": f"{args.workload} {s.label()}", "tokens_per_step": s.image_tokens,
                        "head_tokens_per_step": s.head_tokens, "algorithmic_bytes_per_step": s.algorithmic_bytes,
                        "l2": "inputs exceed L2, no flush" if s.algorithmic_bytes > 2 * 126e6 else "L2-resident: hot timing",
                        "parallelism": "independent replicas" if world > 1 else "single GPU",
+                       "arithmetic": "bf16 tensor-core operands, fp32 accumulation" if s.dtype == "bf16" else "fp32",
                        "kernel_path": {1: "cuda-core", 2: "tensor-core"}.get(path, str(path))},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu,
