@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <atomic>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -55,6 +56,22 @@ struct KernelTimer {
         cudaEventRecord(ev[++n], st);
     }
 };
+
+// Opt-in to more than 48 KiB of dynamic shared memory.  The attribute belongs to a kernel on one
+// device, so it is set once per (kernel, device): `flags` is a static of the call site, one per kernel.
+constexpr int kMaxDevices = 64;
+struct PerDevice { std::atomic<bool> done[kMaxDevices]; };
+template <typename Kernel>
+inline cudaError_t opt_in_smem(Kernel kernel, size_t bytes, PerDevice& flags) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool tracked = dev >= 0 && dev < kMaxDevices;
+    if (tracked && flags.done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && tracked) flags.done[dev].store(true, std::memory_order_release);
+    return e;
+}
 
 // CUDA-core path.  simt_forward returns the cudaError_t of its launches.
 cudaError_t simt_forward(const Problem& p, float* ws_state, float* ws_partial, int P,

@@ -7,6 +7,8 @@
 //                   S += k^^T v (d x d), s += v           (Eq. 9, K^T V and the 1/2 term)
 //   reduce kernel : sums the token splits in a fixed order (only when P > 1)
 //   apply kernel  : out_t = (1/pi) q^_t S + 1/2 s + bias + DWConv(V)_t    (Eq. 9)
+//   fused kernel  : all three steps in one CTA per (b,h) when a whole plane (at most 256 tokens)
+//                   fits in shared memory: one launch, no workspace
 #include "castling_internal.cuh"
 #include "tc_host.cuh"
 
@@ -61,6 +63,33 @@ __device__ __forceinline__ void stage_rows(const T* __restrict__ g, float* __res
         }
 #pragma unroll
         for (int i = 0; i < V; ++i) s[r * LD + col + i] = f[i];
+    }
+}
+
+// The same copy for a whole plane of `rows` valid rows, four 16-byte loads in flight per thread.
+template <typename T, int D, int LD>
+__device__ __forceinline__ void stage_plane(const T* __restrict__ g, float* __restrict__ s, int rows) {
+    constexpr int V = Elem<T>::kVec;
+    constexpr int kChunksPerRow = D / V;
+    constexpr int U = 4;
+    const int total = rows * kChunksPerRow;
+    for (int c0 = threadIdx.x; c0 < total; c0 += U * kThreads) {
+        float f[U][V];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int c = c0 + u * kThreads;
+            if (c < total) Elem<T>::load16(g + (size_t)c * V, f[u]);  // rows are contiguous: chunk c starts at element c * V
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int c = c0 + u * kThreads;
+            if (c < total) {
+                const int r = c / kChunksPerRow, col = (c % kChunksPerRow) * V;
+#pragma unroll
+                for (int i = 0; i < V; i += 4)
+                    *reinterpret_cast<float4*>(s + r * LD + col + i) = make_float4(f[u][i], f[u][i + 1], f[u][i + 2], f[u][i + 3]);
+            }
+        }
     }
 }
 
@@ -258,9 +287,174 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
     }
 }
 
+// ---------------------------------------------------------------------------
+// fused kernel for short sequences: grid (BH), one CTA per (b,h).  K, V and Q of the plane sit in
+// shared memory as fp32 for the whole pass, so the state never leaves the SM, V is read from
+// memory once for both the state and the convolution, and the forward is a single launch with
+// no workspace.  The arithmetic order per element is that of the three-kernel path with P = 1.
+// ---------------------------------------------------------------------------
+// It is taken when at least two such CTAs fit on an SM and there are enough planes to occupy the
+// device (measured: 64 x 8 planes of 7 x 7 tokens 22.7 -> 17.8 us, 64 x 12 of 4 x 4 20.6 -> 15.1 us;
+// 8 planes of 14 x 14 are faster on the three-kernel path, which spreads a plane over several CTAs).
+constexpr int kFusedMaxTokens = 256;
+constexpr int kFusedMinPlanes = 64;
+constexpr size_t kFusedSmemLimit = 100 * 1024;
+
+template <int D> constexpr size_t simt_fused_smem(int N, int ksize) {
+    return sizeof(float) * (3 * (size_t)N * (D + 4) + 2 * (size_t)N + (size_t)D * D + D + (size_t)ksize * ksize * D);
+}
+
+// 1 / max(||row||, eps) for `rows` rows of a shared tile, one warp per row at a time.
+template <int D, int LD>
+__device__ __forceinline__ void row_rnorm_warp(const float* __restrict__ s, float* __restrict__ rn, int rows, float eps2) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r < rows; r += kThreads / 32) {
+        float ss = 0.f;
+        for (int i = lane; i < D; i += 32) { const float x = s[r * LD + i]; ss = fmaf(x, x, ss); }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) rn[r] = 1.0f / sqrtf(fmaxf(ss, eps2));
+    }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                  const T* __restrict__ w, const T* __restrict__ bias, T* __restrict__ out,
+                  int H, int head0, int gridH, int gridW, int ksize, float eps2) {
+    constexpr int R = D / 16;
+    constexpr int LD = D + 4;
+    extern __shared__ __align__(16) float smem[];
+    const int N = gridH * gridW;
+    const int KK = ksize * ksize, rad = (ksize - 1) / 2;
+    float* ks = smem;               // [N][LD]
+    float* vs = ks + N * LD;        // [N][LD]
+    float* qs = vs + N * LD;        // [N][LD]
+    float* rk = qs + N * LD;        // [N]
+    float* rq = rk + N;             // [N]
+    float* S_sm = rq + N;           // [D][D], scaled by 1/pi
+    float* c_sm = S_sm + D * D;     // [D]    1/2 s + bias
+    float* w_sm = c_sm + D;         // [KK][D] filters of this head, tap-major
+
+    const int bh = blockIdx.x, h = (head0 + bh) % H;
+    const size_t plane = (size_t)bh * N * D;
+    stage_plane<T, D, LD>(k + plane, ks, N);
+    stage_plane<T, D, LD>(v + plane, vs, N);
+    stage_plane<T, D, LD>(q + plane, qs, N);
+    for (int i = threadIdx.x; i < KK * D; i += kThreads) {
+        const int tap = i / D, ch = i % D;
+        w_sm[i] = Elem<T>::load1(w + ((size_t)(h * D + ch)) * KK + tap);
+    }
+    __syncthreads();
+    row_rnorm_warp<D, LD>(ks, rk, N, eps2);
+    row_rnorm_warp<D, LD>(qs, rq, N, eps2);
+    __syncthreads();
+
+    const int ti = threadIdx.x / 16, tj = threadIdx.x % 16;
+    {   // state: thread (ti, tj) owns an R x R block of S
+        float acc[R][R];
+        float vsum[R];
+#pragma unroll
+        for (int a = 0; a < R; ++a) {
+            vsum[a] = 0.f;
+#pragma unroll
+            for (int b = 0; b < R; ++b) acc[a][b] = 0.f;
+        }
+#pragma unroll 4
+        for (int n = 0; n < N; ++n) {
+            const float r = rk[n];
+            float a[R], b[R];
+#pragma unroll
+            for (int x = 0; x < R; ++x) { a[x] = ks[n * LD + ti * R + x] * r; b[x] = vs[n * LD + tj * R + x]; }
+#pragma unroll
+            for (int x = 0; x < R; ++x) {
+                vsum[x] += b[x];
+#pragma unroll
+                for (int y = 0; y < R; ++y) acc[x][y] = fmaf(a[x], b[y], acc[x][y]);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < R; ++x)
+#pragma unroll
+            for (int y = 0; y < R; ++y) S_sm[(ti * R + x) * D + tj * R + y] = acc[x][y] * kInvPi;
+        if (ti == 0) {
+#pragma unroll
+            for (int y = 0; y < R; ++y) {
+                const int ch = tj * R + y;
+                c_sm[ch] = 0.5f * vsum[y] + (bias ? Elem<T>::load1(bias + h * D + ch) : 0.f);
+            }
+        }
+    }
+    __syncthreads();
+
+    // apply: thread (tq, tj) owns tokens t0 + tq + 16 r (r = 0..3) and channels tj*R .. tj*R + R - 1
+    const int tq = ti;
+    T* ob = out + plane;
+    for (int t0 = 0; t0 < N; t0 += kApplyTile) {
+        float acc[4][R];
+        int row[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            row[r] = min(t0 + tq + 16 * r, N - 1);  // clamped rows are computed and dropped
+#pragma unroll
+            for (int c = 0; c < R; ++c) acc[r][c] = 0.f;
+        }
+#pragma unroll 4
+        for (int i = 0; i < D; ++i) {
+            float a[4], b[R];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) a[r] = qs[row[r] * LD + i];
+#pragma unroll
+            for (int c = 0; c < R; ++c) b[c] = S_sm[i * D + tj * R + c];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < R; ++c) acc[r][c] = fmaf(a[r], b[c], acc[r][c]);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int t = t0 + tq + 16 * r;
+            if (t >= N) continue;
+            const int y = t / gridW, x = t % gridW;
+            const float scale = rq[t];
+            float o[R];
+#pragma unroll
+            for (int c = 0; c < R; ++c) o[c] = fmaf(acc[r][c], scale, c_sm[tj * R + c]);
+            for (int dy = -rad; dy <= rad; ++dy) {
+                const int yy = y + dy;
+                if (yy < 0 || yy >= gridH) continue;
+                for (int dx = -rad; dx <= rad; ++dx) {
+                    const int xx = x + dx;
+                    if (xx < 0 || xx >= gridW) continue;
+                    const float* vp = vs + (yy * gridW + xx) * LD + tj * R;
+                    const float* wp = w_sm + ((dy + rad) * ksize + (dx + rad)) * D + tj * R;
+#pragma unroll
+                    for (int c = 0; c < R; ++c) o[c] = fmaf(wp[c], vp[c], o[c]);
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < R; ++c) Elem<T>::store1(ob + (size_t)t * D + tj * R + c, o[c]);
+        }
+    }
+}
+
 template <typename T, int D>
 cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, int P,
                         cudaStream_t stream, int* launches, KernelTimer* timer) {
+    if (p.N <= kFusedMaxTokens && p.BH >= kFusedMinPlanes && simt_fused_smem<D>(p.N, p.ksize) <= kFusedSmemLimit) {
+        const size_t smem = simt_fused_smem<D>(p.N, p.ksize);
+        static PerDevice fused_opt_in;
+        cudaError_t e = opt_in_smem(simt_fused_kernel<T, D>, kFusedSmemLimit, fused_opt_in);
+        if (e != cudaSuccess) return e;
+        simt_fused_kernel<T, D><<<(unsigned)p.BH, kThreads, smem, stream>>>(
+            static_cast<const T*>(p.q), static_cast<const T*>(p.k), static_cast<const T*>(p.v),
+            static_cast<const T*>(p.w), static_cast<const T*>(p.bias), static_cast<T*>(p.out),
+            p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2);
+        e = cudaGetLastError();
+        if (e == cudaSuccess) *launches = 1;
+        timer->mark(stream, "simt_fused");
+        return e;
+    }
     const int tiles = (p.N + kStateTile - 1) / kStateTile;
     const int chunk = ((tiles + P - 1) / P) * kStateTile;
     float* dst = (P > 1) ? ws_partial : ws_state;
@@ -278,7 +472,8 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
         timer->mark(stream, "simt_reduce");
     }
     const size_t smem = simt_apply_smem<D>(p.ksize);
-    e = cudaFuncSetAttribute(simt_apply_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static PerDevice apply_opt_in;
+    e = opt_in_smem(simt_apply_kernel<T, D>, simt_apply_smem<D>(7), apply_opt_in);  // 7 x 7: the largest filter
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(p.BH * ((p.N + kApplyTile - 1) / kApplyTile));
     simt_apply_kernel<T, D><<<grid, kThreads, smem, stream>>>(

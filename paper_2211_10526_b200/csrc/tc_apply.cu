@@ -385,11 +385,10 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
     prm.eps2 = p.eps2; prm.status = status;
-    static bool attr_set = false;  // one flag per instantiation
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_apply_kernel<KS, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmem);
+    static PerDevice opt_in;  // one per instantiation
+    {
+        const cudaError_t e = opt_in_smem(tc_apply_kernel<KS, PAIR>, G::kSmem, opt_in);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     const int grid = prm.n_tiles < 148 ? prm.n_tiles : 148;
     // programmatic dependent launch: this grid's prologue and first Q / V loads overlap the tail of

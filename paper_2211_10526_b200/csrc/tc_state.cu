@@ -310,13 +310,11 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
     const uint32_t box[3] = {kD, kTile, 1};
     if (!make_tensor_map_bf16(&tmK, p.k, 3, dims, box, true) || !make_tensor_map_bf16(&tmV, p.v, 3, dims, box, true))
         return cudaErrorNotSupported;
-    static bool attr_set = false;  // per process; the attribute belongs to the function, not to a call
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc_state_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc_state_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    static PerDevice opt_in[2];
+    {
+        const cudaError_t e = pair ? opt_in_smem(tc_state_kernel<true>, kSmemBytes, opt_in[1])
+                                   : opt_in_smem(tc_state_kernel<false>, kSmemBytes, opt_in[0]);
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     float* dst = P > 1 ? partial : final_state;
     // P == 1: a CTA serves several consecutive (b,h); at most 296 CTAs (two per SM) so all are resident

@@ -188,6 +188,50 @@ def test_split_state_path_fp32():
     check(c)
 
 
+# Many planes of few tokens: the CUDA-core path runs its single-launch kernel (one CTA per (b,h),
+# the whole plane in shared memory).  B, H, gridH, gridW, d, ksize
+FUSED_SHAPES = [(16, 4, 1, 1, 32, 3), (8, 8, 1, 1, 16, 7), (32, 2, 4, 4, 32, 5), (16, 4, 2, 2, 64, 7),
+                (64, 1, 3, 17, 32, 3), (8, 8, 13, 5, 64, 3), (64, 2, 8, 8, 16, 1), (4, 16, 5, 13, 48, 5),
+                (16, 4, 7, 9, 80, 3), (64, 1, 4, 8, 96, 3), (8, 8, 3, 5, 112, 3), (16, 4, 4, 4, 128, 3),
+                (8, 8, 14, 14, 32, 3), (8, 8, 16, 16, 16, 5)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", FUSED_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_single_launch_kernel_parity(shape, dtype):
+    pkg = _lib()
+    c = workloads.custom_call(*shape, dtype, seed=330 + sum(shape))
+    s = c.shape
+    ref = run_oracle(c)
+    dev = torch.device("cuda:0")
+    q, k, v, w, b = (t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias))
+    with pkg.CastlingAttn(ksize=s.ksize, force_path=pkg.binding.PATH_SIMT) as attn:
+        out = attn.forward(q, k, v, w, b, s.gridH, s.gridW)
+        torch.cuda.synchronize()
+        assert attn.last_path() == (pkg.binding.PATH_SIMT, 1), "expected the one-launch kernel"
+        out_nb = attn.forward(q, k, v, w, None, s.gridH, s.gridW)
+        torch.cuda.synchronize()
+    assert rel_err(out, ref) <= TOL[dtype]
+    ref_nb = run_oracle(c, bias=False)
+    assert rel_err(out_nb, ref_nb) <= TOL[dtype]
+
+
+def test_single_launch_kernel_zero_rows_and_few_planes():
+    """Zero q/k rows in the one-launch kernel; and with few planes the three-kernel path is kept."""
+    pkg = _lib()
+    c = workloads.custom_call(16, 4, 5, 5, 32, 3, "f32", seed=331)
+    c.q[0, 0, 3] = 0
+    c.k[3, 1, 7] = 0
+    c.k[15, 3, 24] = 0
+    check(c)
+    few = workloads.custom_call(2, 4, 14, 14, 32, 3, "f32", seed=332)
+    dev = torch.device("cuda:0")
+    with pkg.CastlingAttn(ksize=3) as attn:
+        attn.forward(*(t.to(dev) for t in (few.q, few.k, few.v, few.dw_weight, few.dw_bias)), 14, 14)
+        torch.cuda.synchronize()
+        assert attn.last_path() == (pkg.binding.PATH_SIMT, 2)
+
+
 # ---------------------------------------------------------------------------
 # kernel families: the tensor-core path must be the one that runs where it applies
 # ---------------------------------------------------------------------------
