@@ -16,6 +16,14 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"unsupported dtype {t.dtype}: the attention core takes float32 or bfloat16")
 
 
+def _current_raw_stream(device: torch.device) -> int:
+    """Handle of torch's current stream on ``device`` (the short route when torch offers it)."""
+    raw = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+    if raw is not None and device.index is not None:
+        return raw(device.index)
+    return torch.cuda.current_stream(device).cuda_stream
+
+
 class CastlingAttn:
     """Owns one library handle (one stream at a time).
 
@@ -50,22 +58,29 @@ class CastlingAttn:
         return self._h
 
     def _check(self, q, k, v, w, bias, out, gridH, gridW, device_type):
-        if q.dim() != 4 or q.shape != k.shape or q.shape != v.shape or q.shape != out.shape:
+        # straight-line on purpose: this runs on every call and small shapes are bound by host time
+        shape = q.shape
+        if len(shape) != 4 or k.shape != shape or v.shape != shape or out.shape != shape:
             raise ValueError("q, k, v, out must share one [B, H, N, d] shape")
-        B, H, N, d = q.shape
+        B, H, N, d = shape
         if N != gridH * gridW:
             raise ValueError("N != gridH * gridW")
-        if tuple(w.shape) != (H * d, self.ksize, self.ksize):
+        ks = self.ksize
+        if w.shape != (H * d, ks, ks):
             raise ValueError("dw_weight must be [H*d, ksize, ksize]")
-        if bias is not None and tuple(bias.shape) != (H * d,):
-            raise ValueError("dw_bias must be [H*d]")
-        for t in (q, k, v, w, out) + ((bias,) if bias is not None else ()):
-            if t.device.type != device_type:
-                raise ValueError(f"expected {device_type} tensors")
-            if not t.is_contiguous():
-                raise ValueError("tensors must be contiguous")
-            if t.dtype != q.dtype:
-                raise TypeError("all tensors must share one dtype")
+        dt = q.dtype
+        if bias is not None:
+            if bias.shape != (H * d,):
+                raise ValueError("dw_bias must be [H*d]")
+            if bias.device.type != device_type or not bias.is_contiguous() or bias.dtype != dt:
+                raise ValueError(f"dw_bias must be a contiguous {device_type} tensor of the tensors' dtype")
+        if not (q.device.type == k.device.type == v.device.type == w.device.type == out.device.type == device_type):
+            raise ValueError(f"expected {device_type} tensors")
+        if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and w.is_contiguous()
+                and out.is_contiguous()):
+            raise ValueError("tensors must be contiguous")
+        if not (k.dtype == dt and v.dtype == dt and w.dtype == dt and out.dtype == dt):
+            raise TypeError("all tensors must share one dtype")
         return B, H, N, d
 
     def forward(self, q, k, v, dw_weight, dw_bias: Optional[torch.Tensor], gridH: int, gridW: int,
@@ -73,7 +88,7 @@ class CastlingAttn:
         if out is None:
             out = torch.empty_like(q)
         B, H, N, d = self._check(q, k, v, dw_weight, dw_bias, out, gridH, gridW, "cuda")
-        stream = torch.cuda.current_stream(q.device).cuda_stream
+        stream = _current_raw_stream(q.device)
         rc = _b.castling_attn_forward(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), dw_weight.data_ptr(),
                                       None if dw_bias is None else dw_bias.data_ptr(), out.data_ptr(),
                                       B, H, gridH, gridW, d, _dtype_code(q), stream)
