@@ -38,6 +38,13 @@ int choose_splits(int BH, int N) {
 cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
+    if (fused_supports(p)) {  // a whole (b,h) fits in shared memory: one kernel, no workspace
+        const cudaError_t e = launch_fused(p, status, stream);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        timer->mark(stream, "tc_fused");
+        return cudaSuccess;
+    }
     const int tiles = (rows_per_head(p.N, p.d) + kStateTile - 1) / kStateTile;
     const int per = (tiles + P - 1) / P;
     cudaError_t e = launch_state(p, ws_partial, ws_state, counters, P, per, status, stream);

@@ -40,6 +40,10 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
                          int tiles_per_cta, unsigned* status, cudaStream_t st);
 cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st);
 
+// Single-kernel forward for short sequences (bf16, d = 64, N <= 256, 3x3 or 5x5 filters): no workspace.
+bool fused_supports(const Problem& p);
+cudaError_t launch_fused(const Problem& p, unsigned* status, cudaStream_t st);
+
 }  // namespace tc
 
 // Shared with the CUDA-core path: sums P partial states per (b,h) in index order.

@@ -294,6 +294,62 @@ def test_tensor_path_term_isolation():
     check(c, force_path=binding.PATH_TENSOR)
 
 
+# Short sequences of width-64 heads (N <= 256): one tensor-core kernel does the whole pass.
+# B, H, gridH, gridW, d, ksize
+ONE_KERNEL_SHAPES = [(1, 1, 1, 1, 64, 3), (2, 3, 14, 14, 64, 3), (1, 2, 16, 16, 64, 3), (3, 2, 1, 129, 64, 3),
+                     (2, 2, 3, 70, 64, 5), (1, 1, 128, 1, 64, 3), (1, 3, 9, 14, 64, 5), (5, 70, 8, 8, 64, 3),
+                     (1, 1, 2, 128, 64, 5), (2, 1, 127, 1, 64, 5), (37, 9, 5, 7, 64, 3)]
+
+
+@pytest.mark.parametrize("shape", ONE_KERNEL_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_tensor_one_kernel_parity(shape):
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    c = workloads.custom_call(*shape, "bf16", seed=700 + sum(shape))
+    s = c.shape
+    dev = torch.device("cuda:0")
+    q, k, v, w, b = (t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias))
+    with CastlingAttn(ksize=s.ksize, force_path=binding.PATH_TENSOR) as attn:
+        guard = torch.full((s.B * s.H * s.N * s.d + 4096,), 7.0, dtype=torch.bfloat16, device=dev)
+        out = guard[2048:2048 + s.B * s.H * s.N * s.d].view(s.B, s.H, s.N, s.d)
+        attn.forward(q, k, v, w, b, s.gridH, s.gridW, out=out)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+        assert attn.last_path() == (binding.PATH_TENSOR, 1), "expected the single-kernel forward"
+        assert bool((guard[:2048] == 7.0).all()) and bool((guard[-2048:] == 7.0).all()), "wrote outside the output"
+        out_nb = attn.forward(q, k, v, w, None, s.gridH, s.gridW)
+        out_again = attn.forward(q, k, v, w, b, s.gridH, s.gridW)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+    assert rel_err(out, run_oracle(c)) <= TOL["bf16"]
+    assert rel_err(out_nb, run_oracle(c, bias=False)) <= TOL["bf16"]
+    assert torch.equal(out, out_again), "two runs differ bitwise"
+
+
+def test_tensor_one_kernel_term_isolation():
+    """Each term of Eq. 9 alone, on the single-kernel forward (240 tokens: two tiles, the second ragged)."""
+    from paper_2211_10526_b200 import binding
+    for ks in (3, 5):
+        base = lambda seed: workloads.custom_call(3, 2, 12, 20, 64, ks, "bf16", seed=seed)
+        c = base(621)  # linear term alone
+        v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+        c.dw_weight.zero_(); c.dw_bias.zero_()
+        check(c, force_path=binding.PATH_TENSOR)
+        c = base(622)  # 1/2 sum (constant V)
+        c.v[:] = c.v[:, :, :1, :].clone()
+        c.dw_weight.zero_(); c.dw_bias.zero_()
+        check(c, force_path=binding.PATH_TENSOR)
+        c = base(623)  # convolution alone
+        v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+        c.dw_weight = (c.dw_weight.float() * 30).to(torch.bfloat16)
+        c.k.zero_()
+        check(c, force_path=binding.PATH_TENSOR)
+        c = base(624)  # zero rows
+        c.q[0, 0, 5] = 0; c.k[1, 1, 17] = 0; c.k[2, 0, 239] = 0
+        check(c, force_path=binding.PATH_TENSOR)
+        c = workloads.custom_call(2, 2, 10, 10, 64, ks, "bf16", seed=625, qk_lognormal_sigma=3.0)  # row scales
+        check(c, force_path=binding.PATH_TENSOR)
+
+
 def test_tensor_path_term_isolation_head_width_32():
     from paper_2211_10526_b200 import binding
     base = lambda seed, ks: workloads.custom_call(2, 2, 24, 20, 32, ks, "bf16", seed=seed)
