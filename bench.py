@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, help="workload name[:call index]")
     ap.add_argument("--force-path", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
+    ap.add_argument("--layout", default="head_major", choices=["head_major", "token_major"],
+                    help="memory layout of q, k, v, out: [B,H,N,d] contiguous, or [B,N,H,d] passed as strided views")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -238,6 +240,8 @@ def main():
     host = [t.pin_memory() for t in (call.q, call.k, call.v, call.dw_weight, call.dw_bias)]
     q, k, v, w, b = (t.to(dev, non_blocking=True) for t in host)
     out = torch.empty_like(q)
+    if args.layout == "token_major":  # same values, stored [B,N,H,d]; the library reads them through strides
+        q, k, v, out = (t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for t in (q, k, v, out))
     attn = CastlingAttn(ksize=s.ksize, force_path=args.force_path)
     stream = torch.cuda.current_stream(dev)
     # A workload that fits in L2 is timed "cold" over a rotating ring of copies of its tensors whose
@@ -342,6 +346,7 @@ def main():
                        "l2": "inputs exceed L2, no flush" if n_sets == 1 else
                              f"cold: ring of {n_sets} copies of q, k, v, out ({n_sets * s.algorithmic_bytes / 1e6:.0f} MB) cycled",
                        "hot_ms_per_step": hot_ms,
+                       "layout": "[B,H,N,d]" if args.layout == "head_major" else "[B,N,H,d] (strided views)",
                        "parallelism": "independent replicas" if world > 1 else "single GPU",
                        "arithmetic": "bf16 tensor-core operands, fp32 accumulation" if s.dtype == "bf16" else "fp32",
                        "kernel_path": {1: "cuda-core", 2: "tensor-core"}.get(path, str(path))},

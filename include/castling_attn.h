@@ -113,6 +113,42 @@ CASTLING_API int castling_attn_forward(castling_attn_t* handle,
                           castling_dtype_t dtype, void* stream);
 
 /*
+ * Element strides of q, k, v and out for castling_attn_forward_strided.  Element (b, h, n, j)
+ * of a tensor sits at  base + b*batch + h*head + n*token + j  (the d elements of a token are
+ * always contiguous).  [B,H,N,d] contiguous is {H*N*d, N*d, d}; token-major [B,N,H,d], which is what a
+ * projection layer produces without a transpose, is {N*H*d, d, H*d}; q taken out of a fused
+ * [B,N,3,H,d] projection is {N*3*H*d, d, 3*H*d} with base = qkv + 0, H*d or 2*H*d.
+ */
+typedef struct {
+    long long q_batch, q_head, q_token;
+    long long k_batch, k_head, k_token;
+    long long v_batch, v_head, v_token;
+    long long out_batch, out_head, out_token;
+} castling_attn_layout_t;
+
+/*
+ * castling_attn_forward_strided: castling_attn_forward for tensors that are not [B,H,N,d]
+ * contiguous (same Eq. 8-9 computation; the paper does not prescribe a memory layout).
+ *
+ *   layout      HOST pointer, read during the call.  Every stride is in elements, >= 0, a multiple of
+ *               16 bytes; token strides are >= d; batch (head) strides are > 0 when B (H) > 1.
+ *   q,k,v,out   DEVICE base pointers (element (0,0,0,0)), 16-byte aligned.  The ranges spanned by
+ *               `out` and by each input must not overlap, and distinct (b,h,n) of `out` must not
+ *               share memory (not checked).
+ *   everything else as for castling_attn_forward.
+ *
+ * The tensor-core kernels read such layouts directly through strided TMA descriptors (width-64
+ * heads; width-32 heads need contiguous tokens, because two tokens share one 128-byte row there);
+ * everything else, and any layout a descriptor cannot express, runs on the CUDA-core kernels.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, OOM, CUDA.
+ */
+CASTLING_API int castling_attn_forward_strided(castling_attn_t* handle,
+                          const void* q, const void* k, const void* v,
+                          const void* dw_weight, const void* dw_bias, void* out,
+                          int B, int H, int gridH, int gridW, int d,
+                          castling_dtype_t dtype, const castling_attn_layout_t* layout, void* stream);
+
+/*
  * castling_attn_forward_host: the same computation with every tensor in HOST memory.
  * Copies q, k, v, dw_weight and dw_bias to handle-owned device staging buffers on
  * `stream`, runs the forward pass, copies `out` back and synchronises the stream

@@ -27,8 +27,9 @@ def _current_raw_stream(device: torch.device) -> int:
 class CastlingAttn:
     """Owns one library handle (one stream at a time).
 
-    ``forward`` takes device tensors ``[B, H, N, d]`` and enqueues on the current torch
-    stream; ``forward_host`` takes CPU tensors (pinned for best speed) and returns after
+    ``forward`` takes device tensors of shape ``[B, H, N, d]`` (contiguous, or any view whose
+    last dimension has stride 1, e.g. ``x.view(B, N, H, d).permute(0, 2, 1, 3)``) and enqueues on
+    the current torch stream; ``forward_host`` takes CPU tensors (pinned for best speed) and returns after
     the result has been copied back.
     """
 
@@ -76,9 +77,14 @@ class CastlingAttn:
                 raise ValueError(f"dw_bias must be a contiguous {device_type} tensor of the tensors' dtype")
         if not (q.device.type == k.device.type == v.device.type == w.device.type == out.device.type == device_type):
             raise ValueError(f"expected {device_type} tensors")
-        if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and w.is_contiguous()
-                and out.is_contiguous()):
-            raise ValueError("tensors must be contiguous")
+        if not w.is_contiguous():
+            raise ValueError("dw_weight must be contiguous")
+        if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and out.is_contiguous()):
+            if device_type != "cuda":
+                raise ValueError("host tensors must be contiguous")
+            for t in (q, k, v, out):
+                if t.stride(3) != 1:
+                    raise ValueError("the d elements of a token must be contiguous (stride 1 in the last dimension)")
         if not (k.dtype == dt and v.dtype == dt and w.dtype == dt and out.dtype == dt):
             raise TypeError("all tensors must share one dtype")
         return B, H, N, d
@@ -89,9 +95,15 @@ class CastlingAttn:
             out = torch.empty_like(q)
         B, H, N, d = self._check(q, k, v, dw_weight, dw_bias, out, gridH, gridW, "cuda")
         stream = _current_raw_stream(q.device)
-        rc = _b.castling_attn_forward(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), dw_weight.data_ptr(),
-                                      None if dw_bias is None else dw_bias.data_ptr(), out.data_ptr(),
-                                      B, H, gridH, gridW, d, _dtype_code(q), stream)
+        bias_ptr = None if dw_bias is None else dw_bias.data_ptr()
+        if q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and out.is_contiguous():
+            rc = _b.castling_attn_forward(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), dw_weight.data_ptr(),
+                                          bias_ptr, out.data_ptr(), B, H, gridH, gridW, d, _dtype_code(q), stream)
+        else:  # views of token-major or fused-projection buffers: pass their strides through
+            strides = [s for t in (q, k, v, out) for s in t.stride()[:3]]
+            rc = _b.castling_attn_forward_strided(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                                  dw_weight.data_ptr(), bias_ptr, out.data_ptr(), B, H, gridH, gridW,
+                                                  d, _dtype_code(q), strides, stream)
         if rc != _b.OK:
             raise _b.CastlingError(rc, "castling_attn_forward")
         return out

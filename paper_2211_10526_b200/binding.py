@@ -26,6 +26,10 @@ class castling_attn_config_t(ctypes.Structure):
                 ("max_workspace", ctypes.c_size_t)]
 
 
+class castling_attn_layout_t(ctypes.Structure):
+    _fields_ = [(f"{t}_{s}", ctypes.c_longlong) for t in ("q", "k", "v", "out") for s in ("batch", "head", "token")]
+
+
 class CastlingError(RuntimeError):
     def __init__(self, code: int, what: str):
         super().__init__(f"{what}: {error_string(code)} (code {code})")
@@ -45,6 +49,8 @@ def _load() -> ctypes.CDLL:
     lib.castling_attn_forward.argtypes = fwd_args
     lib.castling_attn_forward_host.restype = i
     lib.castling_attn_forward_host.argtypes = fwd_args
+    lib.castling_attn_forward_strided.restype = i
+    lib.castling_attn_forward_strided.argtypes = [vp] * 7 + [i] * 5 + [i, ctypes.POINTER(castling_attn_layout_t), vp]
     lib.castling_attn_destroy.restype = i
     lib.castling_attn_destroy.argtypes = [vp]
     lib.castling_attn_workspace_bytes.restype = sz
@@ -89,6 +95,16 @@ def castling_attn_forward(handle, q: int, k: int, v: int, dw_weight: int, dw_bia
     """Raw call on device addresses; returns the C return code."""
     return lib.castling_attn_forward(handle, q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, dtype,
                                      stream or None)
+
+
+def castling_attn_forward_strided(handle, q: int, k: int, v: int, dw_weight: int, dw_bias: Optional[int], out: int,
+                                  B: int, H: int, gridH: int, gridW: int, d: int, dtype: int, strides,
+                                  stream: int = 0) -> int:
+    """Raw call on device base addresses; ``strides`` holds the twelve element strides
+    (q, k, v, out) x (batch, head, token) in that order.  Returns the C return code."""
+    layout = castling_attn_layout_t(*[int(x) for x in strides])
+    return lib.castling_attn_forward_strided(handle, q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, dtype,
+                                             ctypes.byref(layout), stream or None)
 
 
 def castling_attn_forward_host(handle, q: int, k: int, v: int, dw_weight: int, dw_bias: Optional[int], out: int,

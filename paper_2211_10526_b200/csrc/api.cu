@@ -185,7 +185,7 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     if (rc != CASTLING_OK) return rc;
     const bool tensor_ok = castling::tc::supports(p);
     if (h->cfg.force_path == CASTLING_PATH_TENSOR && !tensor_ok) return CASTLING_ERR_UNSUPPORTED;
-    const bool use_tensor = h->cfg.force_path == CASTLING_PATH_TENSOR ||
+    bool use_tensor = h->cfg.force_path == CASTLING_PATH_TENSOR ||
                             (h->cfg.force_path == CASTLING_PATH_AUTO && castling::tc::preferred(p));
     float* state = h->ws + castling::kHeaderWords;
     float* partial = state + (size_t)p.BH * (use_tensor ? (size_t)castling::tc::kStateWords : castling::state_words(p.d));
@@ -200,6 +200,14 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     } else {
         e = castling::simt_forward(p, state, partial, castling::simt_choose_splits(p.BH, p.N), stream, &launches,
                                    &h->timer);
+    }
+    if (use_tensor && e == cudaErrorNotSupported && h->cfg.force_path == CASTLING_PATH_AUTO) {
+        // the TMA descriptor could not be encoded for these strides: the CUDA-core kernels take any layout
+        (void)cudaGetLastError();
+        use_tensor = false;
+        partial = state + (size_t)p.BH * castling::state_words(p.d);
+        h->timer.begin(stream);
+        e = castling::simt_forward(p, state, partial, castling::simt_choose_splits(p.BH, p.N), stream, &launches, &h->timer);
     }
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->last_path = use_tensor ? CASTLING_PATH_TENSOR : CASTLING_PATH_SIMT;
@@ -216,7 +224,13 @@ Problem make_problem(const castling_attn* h, const void* q, const void* k, const
     p.N = gridH * gridW; p.BH = B * H; p.head0 = 0;
     p.bf16 = (dtype == CASTLING_BF16);
     p.eps2 = (float)(h->cfg.eps * h->cfg.eps);
+    p.set_contiguous();
     return p;
+}
+
+// Elements spanned by a [B, H, N, d] tensor laid out with the given strides.
+long long extent(long long batch, long long head, long long token, int B, int H, long long N, int d) {
+    return (B - 1) * batch + (H - 1) * head + (N - 1) * token + d;
 }
 
 }  // namespace
@@ -241,6 +255,43 @@ int castling_attn_forward(castling_attn_t* h, const void* q, const void* k, cons
         (dw_bias && overlaps(out, tensor_bytes, dw_bias, b_bytes)))
         return CASTLING_ERR_INVALID_ARG;
     const Problem p = make_problem(h, q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, dtype);
+    return run_device(h, p, static_cast<cudaStream_t>(stream));
+}
+
+int castling_attn_forward_strided(castling_attn_t* h, const void* q, const void* k, const void* v,
+                                  const void* dw_weight, const void* dw_bias, void* out,
+                                  int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype,
+                                  const castling_attn_layout_t* layout, void* stream) {
+    int rc = check_shape(h, B, H, gridH, gridW, d, dtype);
+    if (rc != CASTLING_OK) return rc;
+    if (!q || !k || !v || !dw_weight || !out || !layout) return CASTLING_ERR_INVALID_ARG;
+    const long long eb = (long long)elem_bytes(dtype), N = (long long)gridH * gridW;
+    const long long* s = &layout->q_batch;  // twelve strides: q, k, v, out x (batch, head, token)
+    long long ext[4];
+    for (int t = 0; t < 4; ++t) {
+        const long long sb = s[3 * t], sh = s[3 * t + 1], st = s[3 * t + 2];
+        if (sb < 0 || sh < 0 || st < d) return CASTLING_ERR_INVALID_ARG;
+        if ((B > 1 && sb == 0) || (H > 1 && sh == 0)) return CASTLING_ERR_INVALID_ARG;
+        if ((sb * eb) % 16 || (sh * eb) % 16 || (st * eb) % 16) return CASTLING_ERR_ALIGNMENT;
+        if (sb > (1LL << 40) || sh > (1LL << 40) || st > (1LL << 32)) return CASTLING_ERR_UNSUPPORTED;
+        ext[t] = extent(sb, sh, st, B, H, N, d);
+        if (ext[t] > (1LL << 42)) return CASTLING_ERR_UNSUPPORTED;
+    }
+    const void* ptrs[4] = {q, k, v, out};
+    for (const void* ptr : ptrs)
+        if ((uintptr_t)ptr & 15) return CASTLING_ERR_ALIGNMENT;
+    const size_t w_bytes = (size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb, b_bytes = (size_t)H * d * eb;
+    const size_t out_bytes = (size_t)(ext[3] * eb);
+    if (overlaps(out, out_bytes, q, (size_t)(ext[0] * eb)) || overlaps(out, out_bytes, k, (size_t)(ext[1] * eb)) ||
+        overlaps(out, out_bytes, v, (size_t)(ext[2] * eb)) || overlaps(out, out_bytes, dw_weight, w_bytes) ||
+        (dw_bias && overlaps(out, out_bytes, dw_bias, b_bytes)))
+        return CASTLING_ERR_INVALID_ARG;
+    Problem p = make_problem(h, q, k, v, dw_weight, dw_bias, out, B, H, gridH, gridW, d, dtype);
+    p.lq = {layout->q_batch, layout->q_head, layout->q_token};
+    p.lk = {layout->k_batch, layout->k_head, layout->k_token};
+    p.lv = {layout->v_batch, layout->v_head, layout->v_token};
+    p.lo = {layout->out_batch, layout->out_head, layout->out_token};
+    p.hdiv = H;
     return run_device(h, p, static_cast<cudaStream_t>(stream));
 }
 

@@ -12,6 +12,17 @@ namespace castling {
 
 constexpr float kInvPi = 0.31830988618379067154f;
 
+// Element strides of one [B, H, N, d] tensor whose d elements are contiguous.
+struct Layout {
+    long long batch, head, token;
+};
+
+// Offset (in elements) of (b,h) plane i: planes are numbered b * hdiv + h with hdiv planes per batch step.
+__host__ __device__ inline long long plane_offset(const Layout& l, int i, int hdiv) {
+    const int b = i / hdiv;
+    return (long long)b * l.batch + (long long)(i - b * hdiv) * l.head;
+}
+
 // One forward call, as the kernels see it.
 struct Problem {
     const void* q;
@@ -26,6 +37,16 @@ struct Problem {
     int head0;         // head index of plane 0: plane i uses the filters of head (head0 + i) % H
     bool bf16;
     float eps2;        // eps^2: the floor under the sum of squares
+    Layout lq, lk, lv, lo;  // where token n of plane i of q, k, v, out starts: plane_offset(l, i, hdiv) + n * l.token
+    int hdiv;          // planes per batch step of the layouts: H for a caller's strided tensors, BH for a
+                       // run of contiguous planes (one uniform plane stride)
+    // Contiguous [planes][N][d] tensors; needs N, d and BH.
+    void set_contiguous() {
+        const Layout c = {0, (long long)N * d, (long long)d};
+        lq = lk = lv = lo = c;
+        hdiv = BH;
+    }
+    bool contiguous_tokens() const { return lq.token == d && lk.token == d && lv.token == d && lo.token == d; }
 };
 
 // Workspace layout (fp32 words):

@@ -46,17 +46,17 @@ template <> struct Elem<__nv_bfloat16> {
     static __device__ __forceinline__ void store1(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
 };
 
-// Copy `rows` token rows of width D (contiguous in memory) into a padded fp32
+// Copy `rows` token rows of width D (row r starts r * tok elements after g) into a padded fp32
 // shared tile; rows at or beyond `valid` are zero-filled.
 template <typename T, int D, int LD>
-__device__ __forceinline__ void stage_rows(const T* __restrict__ g, float* __restrict__ s, int rows, int valid) {
+__device__ __forceinline__ void stage_rows(const T* __restrict__ g, long long tok, float* __restrict__ s, int rows, int valid) {
     constexpr int V = Elem<T>::kVec;
     constexpr int kChunksPerRow = D / V;
     for (int c = threadIdx.x; c < rows * kChunksPerRow; c += kThreads) {
         const int r = c / kChunksPerRow, col = (c % kChunksPerRow) * V;
         float f[V];
         if (r < valid) {
-            Elem<T>::load16(g + (size_t)r * D + col, f);
+            Elem<T>::load16(g + r * tok + col, f);
         } else {
 #pragma unroll
             for (int i = 0; i < V; ++i) f[i] = 0.f;
@@ -68,7 +68,7 @@ __device__ __forceinline__ void stage_rows(const T* __restrict__ g, float* __res
 
 // The same copy for a whole plane of `rows` valid rows, four 16-byte loads in flight per thread.
 template <typename T, int D, int LD>
-__device__ __forceinline__ void stage_plane(const T* __restrict__ g, float* __restrict__ s, int rows) {
+__device__ __forceinline__ void stage_plane(const T* __restrict__ g, long long tok, float* __restrict__ s, int rows) {
     constexpr int V = Elem<T>::kVec;
     constexpr int kChunksPerRow = D / V;
     constexpr int U = 4;
@@ -78,7 +78,7 @@ __device__ __forceinline__ void stage_plane(const T* __restrict__ g, float* __re
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int c = c0 + u * kThreads;
-            if (c < total) Elem<T>::load16(g + (size_t)c * V, f[u]);  // rows are contiguous: chunk c starts at element c * V
+            if (c < total) Elem<T>::load16(g + (c / kChunksPerRow) * tok + (c % kChunksPerRow) * V, f[u]);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -113,7 +113,7 @@ __device__ __forceinline__ void row_rnorm(const float* __restrict__ s, float* __
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 simt_state_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __restrict__ dst,
-                  int N, int chunk, int P, float eps2) {
+                  int N, int chunk, int P, float eps2, Layout lk, Layout lv, int hdiv) {
     constexpr int R = D / 16;
     constexpr int LD = D + 4;  // padded row, keeps 16-byte alignment
     __shared__ __align__(16) float ks[kStateTile * LD];
@@ -122,8 +122,8 @@ simt_state_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __res
 
     const int p = blockIdx.x % P, bh = blockIdx.x / P;
     const int n_begin = p * chunk, n_end = min(N, n_begin + chunk);
-    const T* kb = k + (size_t)bh * N * D;
-    const T* vb = v + (size_t)bh * N * D;
+    const T* kb = k + plane_offset(lk, bh, hdiv);
+    const T* vb = v + plane_offset(lv, bh, hdiv);
     const int ti = threadIdx.x / 16, tj = threadIdx.x % 16;
 
     float acc[R][R];
@@ -138,8 +138,8 @@ simt_state_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __res
     for (int n0 = n_begin; n0 < n_end; n0 += kStateTile) {
         const int valid = min(kStateTile, n_end - n0);
         __syncthreads();  // previous tile fully consumed
-        stage_rows<T, D, LD>(kb + (size_t)n0 * D, ks, kStateTile, valid);
-        stage_rows<T, D, LD>(vb + (size_t)n0 * D, vs, kStateTile, valid);
+        stage_rows<T, D, LD>(kb + n0 * lk.token, lk.token, ks, kStateTile, valid);
+        stage_rows<T, D, LD>(vb + n0 * lv.token, lv.token, vs, kStateTile, valid);
         __syncthreads();
         row_rnorm<D, LD, kStateTile>(ks, rk, eps2);
         __syncthreads();
@@ -194,7 +194,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __restrict__ w,
                   const T* __restrict__ bias, const float* __restrict__ state, T* __restrict__ out,
-                  int H, int head0, int gridH, int gridW, int ksize, float eps2) {
+                  int H, int head0, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lv, Layout lo,
+                  int hdiv) {
     constexpr int R = D / 16;
     constexpr int LDQ = D + 1;
     extern __shared__ __align__(16) float smem[];
@@ -221,12 +222,12 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
     }
     {   // Q tile; rows are padded by one float, so staged with scalar stores
         constexpr int V = Elem<T>::kVec;
-        const T* qb = q + ((size_t)bh * N + t0) * D;
+        const T* qb = q + plane_offset(lq, bh, hdiv) + t0 * lq.token;
         for (int c = threadIdx.x; c < kApplyTile * (D / V); c += kThreads) {
             const int r = c / (D / V), col = (c % (D / V)) * V;
             float f[V];
             if (r < valid) {
-                Elem<T>::load16(qb + (size_t)r * D + col, f);
+                Elem<T>::load16(qb + r * lq.token + col, f);
             } else {
 #pragma unroll
                 for (int i = 0; i < V; ++i) f[i] = 0.f;
@@ -259,8 +260,8 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
             for (int c = 0; c < R; ++c) acc[r][c] = fmaf(a[r], b[c], acc[r][c]);
     }
 
-    const T* vb = v + (size_t)bh * N * D;
-    T* ob = out + (size_t)bh * N * D;
+    const T* vb = v + plane_offset(lv, bh, hdiv);
+    T* ob = out + plane_offset(lo, bh, hdiv);
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         const int tl = tq + 16 * r;
@@ -276,14 +277,14 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
             for (int dx = -rad; dx <= rad; ++dx) {
                 const int xx = x + dx;
                 if (xx < 0 || xx >= gridW) continue;
-                const T* vp = vb + ((size_t)yy * gridW + xx) * D + tj * R;
+                const T* vp = vb + (yy * gridW + xx) * lv.token + tj * R;
                 const float* wp = w_sm + ((dy + rad) * ksize + (dx + rad)) * D + tj * R;
 #pragma unroll
                 for (int c = 0; c < R; ++c) o[c] = fmaf(wp[c], Elem<T>::load1(vp + c), o[c]);
             }
         }
 #pragma unroll
-        for (int c = 0; c < R; ++c) Elem<T>::store1(ob + (size_t)t * D + tj * R + c, o[c]);
+        for (int c = 0; c < R; ++c) Elem<T>::store1(ob + t * lo.token + tj * R + c, o[c]);
     }
 }
 
@@ -321,7 +322,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                   const T* __restrict__ w, const T* __restrict__ bias, T* __restrict__ out,
-                  int H, int head0, int gridH, int gridW, int ksize, float eps2) {
+                  int H, int head0, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lk, Layout lv,
+                  Layout lo, int hdiv) {
     constexpr int R = D / 16;
     constexpr int LD = D + 4;
     extern __shared__ __align__(16) float smem[];
@@ -337,10 +339,9 @@ simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
     float* w_sm = c_sm + D;         // [KK][D] filters of this head, tap-major
 
     const int bh = blockIdx.x, h = (head0 + bh) % H;
-    const size_t plane = (size_t)bh * N * D;
-    stage_plane<T, D, LD>(k + plane, ks, N);
-    stage_plane<T, D, LD>(v + plane, vs, N);
-    stage_plane<T, D, LD>(q + plane, qs, N);
+    stage_plane<T, D, LD>(k + plane_offset(lk, bh, hdiv), lk.token, ks, N);
+    stage_plane<T, D, LD>(v + plane_offset(lv, bh, hdiv), lv.token, vs, N);
+    stage_plane<T, D, LD>(q + plane_offset(lq, bh, hdiv), lq.token, qs, N);
     for (int i = threadIdx.x; i < KK * D; i += kThreads) {
         const int tap = i / D, ch = i % D;
         w_sm[i] = Elem<T>::load1(w + ((size_t)(h * D + ch)) * KK + tap);
@@ -389,7 +390,7 @@ simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
 
     // apply: thread (tq, tj) owns tokens t0 + tq + 16 r (r = 0..3) and channels tj*R .. tj*R + R - 1
     const int tq = ti;
-    T* ob = out + plane;
+    T* ob = out + plane_offset(lo, bh, hdiv);
     for (int t0 = 0; t0 < N; t0 += kApplyTile) {
         float acc[4][R];
         int row[4];
@@ -433,7 +434,7 @@ simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
                 }
             }
 #pragma unroll
-            for (int c = 0; c < R; ++c) Elem<T>::store1(ob + (size_t)t * D + tj * R + c, o[c]);
+            for (int c = 0; c < R; ++c) Elem<T>::store1(ob + t * lo.token + tj * R + c, o[c]);
         }
     }
 }
@@ -449,7 +450,7 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
         simt_fused_kernel<T, D><<<(unsigned)p.BH, kThreads, smem, stream>>>(
             static_cast<const T*>(p.q), static_cast<const T*>(p.k), static_cast<const T*>(p.v),
             static_cast<const T*>(p.w), static_cast<const T*>(p.bias), static_cast<T*>(p.out),
-            p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2);
+            p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2, p.lq, p.lk, p.lv, p.lo, p.hdiv);
         e = cudaGetLastError();
         if (e == cudaSuccess) *launches = 1;
         timer->mark(stream, "simt_fused");
@@ -459,7 +460,7 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     const int chunk = ((tiles + P - 1) / P) * kStateTile;
     float* dst = (P > 1) ? ws_partial : ws_state;
     simt_state_kernel<T, D><<<(unsigned)(p.BH * P), kThreads, 0, stream>>>(
-        static_cast<const T*>(p.k), static_cast<const T*>(p.v), dst, p.N, chunk, P, p.eps2);
+        static_cast<const T*>(p.k), static_cast<const T*>(p.v), dst, p.N, chunk, P, p.eps2, p.lk, p.lv, p.hdiv);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     *launches = 1;
@@ -478,7 +479,8 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     const unsigned grid = (unsigned)(p.BH * ((p.N + kApplyTile - 1) / kApplyTile));
     simt_apply_kernel<T, D><<<grid, kThreads, smem, stream>>>(
         static_cast<const T*>(p.q), static_cast<const T*>(p.v), static_cast<const T*>(p.w),
-        static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2);
+        static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2,
+        p.lq, p.lv, p.lo, p.hdiv);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     timer->mark(stream, "simt_apply");

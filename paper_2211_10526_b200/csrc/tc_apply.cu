@@ -57,7 +57,7 @@ struct ApplyParams {
     int P;
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
-    int H, head0, bh0, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
+    int H, head0, bh0, hdiv, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
 };
@@ -117,8 +117,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
                 uint8_t* qs = stages + s * G::kStage;
                 mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
-                tma_load_4d_hint(qs, &tmQ, &full[s], 0, x0, y0, bh, pol_q);
-                tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, bh);
+                const int pb = bh / prm.hdiv, ph = bh - pb * prm.hdiv;
+                tma_load_5d_hint(qs, &tmQ, &full[s], 0, x0, y0, ph, pb, pol_q);
+                tma_load_5d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, ph, pb);
                 ++issued;
             }
             if (*abort_flag) {
@@ -257,7 +258,8 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             fence_proxy_async_smem();
             named_barrier_sync(1, kEpiThreads);
             if (leader) {
-                tma_store_4d_hint(&tmO, out_s, 0, x0, y0, bh, pol_o);
+                const int pb = bh / prm.hdiv;
+                tma_store_5d_hint(&tmO, out_s, 0, x0, y0, bh - pb * prm.hdiv, pb, pol_o);
                 tma_store_commit();
             }
         }
@@ -359,18 +361,28 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     using G = Geo<KS, PAIR>;
     CUtensorMap tmQ, tmV, tmO;
     const int cols = PAIR ? p.gridW / 2 : p.gridW;  // 128-byte columns per grid row
-    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)cols, (uint64_t)p.gridH, (uint64_t)p.BH};
-    const uint32_t box[4] = {kD, kTX, kTY, 1};
-    const uint32_t boxv[4] = {kD, (uint32_t)G::HX, (uint32_t)G::HY, 1};
-    if (!make_tensor_map_bf16(&tmQ, p.q, 4, dims, box, true) || !make_tensor_map_bf16(&tmO, p.out, 4, dims, box, true) ||
-        !make_tensor_map_bf16(&tmV, p.v, 4, dims, boxv, false))
+    // [64, columns, grid rows, planes per batch step, batch steps]
+    const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
+    const uint64_t dims[5] = {(uint64_t)kD, (uint64_t)cols, (uint64_t)p.gridH, (uint64_t)p.hdiv, nb};
+    const uint32_t box[5] = {kD, kTX, kTY, 1, 1};
+    const uint32_t boxv[5] = {kD, (uint32_t)G::HX, (uint32_t)G::HY, 1, 1};
+    auto strides = [&](const Layout& l, uint64_t (&s)[4]) {
+        s[0] = (uint64_t)(PAIR ? kD : l.token);          // next column: one token, or (PAIR) two
+        s[1] = (uint64_t)(l.token * p.gridW);            // next grid row
+        s[2] = (uint64_t)l.head;
+        s[3] = (uint64_t)(nb > 1 ? l.batch : l.head * p.hdiv);
+    };
+    uint64_t sq[4], sv[4], so[4];
+    strides(p.lq, sq); strides(p.lv, sv); strides(p.lo, so);
+    if (!make_tensor_map_bf16(&tmQ, p.q, 5, dims, sq, box, true) || !make_tensor_map_bf16(&tmO, p.out, 5, dims, so, box, true) ||
+        !make_tensor_map_bf16(&tmV, p.v, 5, dims, sv, boxv, false))
         return cudaErrorNotSupported;
     ApplyParams prm;
     prm.state = state;
     prm.P = P;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
-    prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0;
+    prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0; prm.hdiv = p.hdiv;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
     prm.eps2 = p.eps2; prm.status = status;

@@ -13,7 +13,8 @@ constexpr int kStateTile = 128;  // tokens per UMMA stage of the state kernel
 // 128-byte row there); 3x3 or 5x5 filters.
 bool supports(const Problem& p) {
     if (!p.bf16 || (p.ksize != 3 && p.ksize != 5)) return false;
-    return p.d == 64 || (p.d == 32 && p.gridW % 2 == 0);
+    // width-32 heads pair two adjacent tokens in one 128-byte row: the tokens must be contiguous
+    return p.d == 64 || (p.d == 32 && p.gridW % 2 == 0 && p.contiguous_tokens());
 }
 
 int rows_per_head(int N, int d) { return d == 32 ? N / 2 : N; }

@@ -48,13 +48,16 @@ constexpr size_t kSmemBytes = 1024 + kOffBar + 128;
 struct FusedParams {
     const __nv_bfloat16* w;     // [H*64][KS][KS]
     const __nv_bfloat16* bias;  // [H*64] or nullptr
-    __nv_bfloat16* out;         // [BH][N][64]
-    int H, head0, BH, N, gridH, gridW;
+    __nv_bfloat16* out;         // token n of plane i at plane_offset(lo, i, hdiv) + n * lo.token
+    Layout lo;
+    int H, head0, BH, hdiv, N, gridH, gridW;
     float eps2;
     unsigned* status;
 };
 
-template <int KS>
+// OUT_PACKED: the output's token rows are contiguous (stride 64), which keeps the row addresses of the
+// store loop compile-time offsets.
+template <int KS, bool OUT_PACKED>
 __global__ void __launch_bounds__(kThreads, (KS == 3) ? 2 : 1)
 tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmVplain,
@@ -118,19 +121,19 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const uint64_t pol = l2_policy_evict_first();  // K and Q are read once
             int issued = 0, issued_vp = 0;
             for (int it = 0; it < n_planes; ++it) {
-                const int bh = blockIdx.x + it * gridDim.x;
+                const int bh = blockIdx.x + it * gridDim.x, pb = bh / prm.hdiv, ph = bh - pb * prm.hdiv;
                 if (it > 0 && !mbar_wait(plane_free, (it - 1) & 1, abort_flag, prm.status, kBit)) break;
                 mbar_expect_tx(k_full, tiles * kTileBytes);
-                for (int t = 0; t < tiles; ++t) tma_load_3d_hint(K_s + t * kTileBytes, &tmK, k_full, 0, t * kTile, bh, pol);
+                for (int t = 0; t < tiles; ++t) tma_load_4d_hint(K_s + t * kTileBytes, &tmK, k_full, 0, t * kTile, ph, pb, pol);
                 mbar_expect_tx(v_full, tiles * kTileBytes);
-                for (int t = 0; t < tiles; ++t) tma_load_3d(V_s + t * kTileBytes, &tmV, v_full, 0, t * kTile, bh);
+                for (int t = 0; t < tiles; ++t) tma_load_4d(V_s + t * kTileBytes, &tmV, v_full, 0, t * kTile, ph, pb);
                 mbar_expect_tx(q_full, tiles * kTileBytes);
-                for (int t = 0; t < tiles; ++t) tma_load_3d_hint(Q_s + t * kTileBytes, &tmQ, q_full, 0, t * kTile, bh, pol);
+                for (int t = 0; t < tiles; ++t) tma_load_4d_hint(Q_s + t * kTileBytes, &tmQ, q_full, 0, t * kTile, ph, pb, pol);
                 ++issued;
                 // the K tiles are dead once the state UMMAs have retired: bring V in again, unswizzled
                 if (!mbar_wait(s_done, it & 1, abort_flag, prm.status, kBit)) break;
                 mbar_expect_tx(vp_full, tiles * kTileBytes);
-                for (int t = 0; t < tiles; ++t) tma_load_3d(K_s + t * kTileBytes, &tmVplain, vp_full, 0, t * kTile, bh);
+                for (int t = 0; t < tiles; ++t) tma_load_4d(K_s + t * kTileBytes, &tmVplain, vp_full, 0, t * kTile, ph, pb);
                 ++issued_vp;
             }
             if (*abort_flag) {
@@ -325,7 +328,8 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                                __uint_as_float((uint32_t)wraw[1][dy * KS + dx] << 16));
             const float2 c2 = make_float2(fmaf(0.5f, sum_s[2 * lane], __uint_as_float((uint32_t)braw[0] << 16)),
                                           fmaf(0.5f, sum_s[2 * lane + 1], __uint_as_float((uint32_t)braw[1] << 16)));
-            uint32_t* out_plane = reinterpret_cast<uint32_t*>(prm.out + (size_t)bh * N * kD) + lane;
+            uint32_t* out_plane = reinterpret_cast<uint32_t*>(prm.out + plane_offset(prm.lo, bh, prm.hdiv)) + lane;
+            const long long out_tok = OUT_PACKED ? kD / 2 : prm.lo.token / 2;  // 32-bit words per token step
             const int sc = lane >> 1, sw = (lane & 1) * 8;  // chunk and offset of the lane's pair in an fp32 row
             // Branch-free inside a unit: a neighbour outside the grid is read from a row of zeros, the
             // columns of a ragged last unit are computed (from in-bounds shared memory) and not stored.
@@ -370,7 +374,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         const float2 a2 = *reinterpret_cast<const float2*>(srow + ((sc ^ (tr & 7)) << 4) + sw);
                         const float rq = rq_s[t];
                         const float2 o = ffma2(a2, make_float2(rq, rq), acc);
-                        if (j < nx) out_plane[(size_t)t * (kD / 2)] = pack_bf16x2(o.x, o.y);
+                        if (j < nx) out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
                     }
                 }
             }
@@ -386,22 +390,35 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 template <int KS>
 cudaError_t launch_fused_ks(const Problem& p, unsigned* status, cudaStream_t st) {
     CUtensorMap tmK, tmV, tmQ, tmVplain;
-    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)p.N, (uint64_t)p.BH};
-    const uint32_t box[3] = {kD, kTile, 1};
-    if (!make_tensor_map_bf16(&tmK, p.k, 3, dims, box, true) || !make_tensor_map_bf16(&tmV, p.v, 3, dims, box, true) ||
-        !make_tensor_map_bf16(&tmQ, p.q, 3, dims, box, true) || !make_tensor_map_bf16(&tmVplain, p.v, 3, dims, box, false))
+    // [64, tokens, planes per batch step, batch steps]
+    const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
+    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)p.N, (uint64_t)p.hdiv, nb};
+    const uint32_t box[4] = {kD, kTile, 1, 1};
+    auto strides = [&](const Layout& l, uint64_t (&s)[3]) {
+        s[0] = (uint64_t)l.token; s[1] = (uint64_t)l.head; s[2] = (uint64_t)(nb > 1 ? l.batch : l.head * p.hdiv);
+    };
+    uint64_t sq[3], sk[3], sv[3];
+    strides(p.lq, sq); strides(p.lk, sk); strides(p.lv, sv);
+    if (!make_tensor_map_bf16(&tmK, p.k, 4, dims, sk, box, true) || !make_tensor_map_bf16(&tmV, p.v, 4, dims, sv, box, true) ||
+        !make_tensor_map_bf16(&tmQ, p.q, 4, dims, sq, box, true) || !make_tensor_map_bf16(&tmVplain, p.v, 4, dims, sv, box, false))
         return cudaErrorNotSupported;
     FusedParams prm;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.out = static_cast<__nv_bfloat16*>(p.out);
-    prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.N = p.N; prm.gridH = p.gridH; prm.gridW = p.gridW;
+    prm.lo = p.lo;
+    prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv; prm.N = p.N; prm.gridH = p.gridH; prm.gridW = p.gridW;
     prm.eps2 = p.eps2; prm.status = status;
-    static PerDevice opt_in;  // one per instantiation
-    const cudaError_t e = opt_in_smem(tc_fused_kernel<KS>, kSmemBytes, opt_in);
+    static PerDevice opt_in[2];  // per instantiation
+    const bool packed = (p.lo.token == kD);
+    const cudaError_t e = packed ? opt_in_smem(tc_fused_kernel<KS, true>, kSmemBytes, opt_in[1])
+                                 : opt_in_smem(tc_fused_kernel<KS, false>, kSmemBytes, opt_in[0]);
     if (e != cudaSuccess) return e;
     const int grid = p.BH < 2 * 148 ? p.BH : 2 * 148;  // two CTAs per SM
-    tc_fused_kernel<KS><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
+    if (packed)
+        tc_fused_kernel<KS, true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
+    else
+        tc_fused_kernel<KS, false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
     return cudaGetLastError();
 }
 

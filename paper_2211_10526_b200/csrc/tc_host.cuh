@@ -11,7 +11,7 @@ namespace tc {
 constexpr int kCountersPerHead = 17;
 
 bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
-                          const uint32_t* box, bool swizzle128);
+                          const uint64_t* strides, const uint32_t* box, bool swizzle128);
 
 // True when the tensor-core kernels can take this problem (bf16; d = 64, or d = 32 with even gridW;
 // 3x3 or 5x5 filters).

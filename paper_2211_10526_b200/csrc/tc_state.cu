@@ -34,7 +34,7 @@ template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 2)
 tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 float* __restrict__ dst, float* __restrict__ final_state, unsigned* __restrict__ counters,
-                int N, int tiles_per_cta, int P, int BH, int items_per_cta, float eps2, unsigned* status) {
+                int N, int tiles_per_cta, int P, int BH, int hdiv, int items_per_cta, float eps2, unsigned* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* ones = smem + kStages * kStageBytes;
@@ -106,8 +106,9 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, status, kStatusStateTimeout)) { ok = false; break; }
                     uint8_t* ks = smem + s * kStageBytes;
                     mbar_expect_tx(&full[s], kStageBytes);
-                    tma_load_3d_hint(ks, &tmK, &full[s], 0, (t_begin + it) * kTile, bh0 + item, pol_k);
-                    tma_load_3d_hint(ks + kTileBytes, &tmV, &full[s], 0, (t_begin + it) * kTile, bh0 + item, pol_v);
+                    const int plane = bh0 + item, pb = plane / hdiv, ph = plane - pb * hdiv;
+                    tma_load_4d_hint(ks, &tmK, &full[s], 0, (t_begin + it) * kTile, ph, pb, pol_k);
+                    tma_load_4d_hint(ks + kTileBytes, &tmV, &full[s], 0, (t_begin + it) * kTile, ph, pb, pol_v);
                 }
             }
             if (*abort_flag) {
@@ -306,9 +307,15 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
     const bool pair = (p.d == 32);
     const int rows = pair ? p.N / 2 : p.N;  // 128-byte rows per (b,h)
     CUtensorMap tmK, tmV;
-    const uint64_t dims[3] = {(uint64_t)kD, (uint64_t)rows, (uint64_t)p.BH};
-    const uint32_t box[3] = {kD, kTile, 1};
-    if (!make_tensor_map_bf16(&tmK, p.k, 3, dims, box, true) || !make_tensor_map_bf16(&tmV, p.v, 3, dims, box, true))
+    // [64, rows, planes per batch step, batch steps]; a 128-byte row is one token, or two adjacent ones
+    const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
+    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)rows, (uint64_t)p.hdiv, nb};
+    const uint32_t box[4] = {kD, kTile, 1, 1};
+    const uint64_t sk[3] = {(uint64_t)(pair ? kD : p.lk.token), (uint64_t)p.lk.head,
+                            (uint64_t)(nb > 1 ? p.lk.batch : p.lk.head * p.hdiv)};
+    const uint64_t sv[3] = {(uint64_t)(pair ? kD : p.lv.token), (uint64_t)p.lv.head,
+                            (uint64_t)(nb > 1 ? p.lv.batch : p.lv.head * p.hdiv)};
+    if (!make_tensor_map_bf16(&tmK, p.k, 4, dims, sk, box, true) || !make_tensor_map_bf16(&tmV, p.v, 4, dims, sv, box, true))
         return cudaErrorNotSupported;
     static PerDevice opt_in[2];
     {
@@ -325,10 +332,10 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
     }
     if (pair)
         tc_state_kernel<true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(
-            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, items, p.eps2, status);
+            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, p.hdiv, items, p.eps2, status);
     else
         tc_state_kernel<false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(
-            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, items, p.eps2, status);
+            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, p.hdiv, items, p.eps2, status);
     return cudaGetLastError();
 }
 

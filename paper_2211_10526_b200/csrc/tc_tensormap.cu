@@ -27,6 +27,7 @@ struct CacheEntry {
     const void* base = nullptr;
     int rank = 0;
     uint64_t dims[5] = {};
+    uint64_t strides[4] = {};
     uint32_t box[5] = {};
     bool swizzle = false;
     CUtensorMap map;
@@ -36,49 +37,58 @@ CacheEntry g_cache[kCacheSize];
 int g_cache_next = 0;
 std::mutex g_cache_mutex;
 
-bool same_key(const CacheEntry& e, const void* base, int rank, const uint64_t* dims, const uint32_t* box, bool sw) {
+bool same_key(const CacheEntry& e, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+              const uint32_t* box, bool sw) {
     if (!e.valid || e.base != base || e.rank != rank || e.swizzle != sw) return false;
     for (int i = 0; i < rank; ++i)
         if (e.dims[i] != dims[i] || e.box[i] != box[i]) return false;
+    for (int i = 0; i + 1 < rank; ++i)
+        if (e.strides[i] != strides[i]) return false;
     return true;
 }
 }  // namespace
 
 namespace {
 bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
-                            const uint32_t* box, bool swizzle128);
+                            const uint64_t* strides, const uint32_t* box, bool swizzle128);
 }
 
-// dims/box are innermost-first, in elements; the innermost dimension is contiguous.
+// dims/box are innermost-first, in elements; the innermost dimension is contiguous; strides[i] is the
+// distance in elements between consecutive indices of dimension i + 1 (rank - 1 entries).
 bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
-                          const uint32_t* box, bool swizzle128) {
+                          const uint64_t* strides, const uint32_t* box, bool swizzle128) {
     if (rank < 2 || rank > 5) return false;
+    uint64_t fixed[4];
+    for (int i = 0; i + 1 < rank; ++i) {
+        fixed[i] = (dims[i + 1] == 1 && strides[i] == 0) ? 8 : strides[i];  // never stepped over: any legal value
+        if (fixed[i] == 0 || (fixed[i] * 2) % 16 != 0 || fixed[i] * 2 >= (1ull << 40)) return false;
+    }
+    strides = fixed;
     std::lock_guard<std::mutex> lock(g_cache_mutex);
     for (const CacheEntry& e : g_cache)
-        if (same_key(e, base, rank, dims, box, swizzle128)) { *out = e.map; return true; }
-    if (!encode_tensor_map_bf16(out, base, rank, dims, box, swizzle128)) return false;
+        if (same_key(e, base, rank, dims, strides, box, swizzle128)) { *out = e.map; return true; }
+    if (!encode_tensor_map_bf16(out, base, rank, dims, strides, box, swizzle128)) return false;
     CacheEntry& e = g_cache[g_cache_next];
     g_cache_next = (g_cache_next + 1) % kCacheSize;
     e.valid = true; e.base = base; e.rank = rank; e.swizzle = swizzle128; e.map = *out;
     for (int i = 0; i < rank; ++i) { e.dims[i] = dims[i]; e.box[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) e.strides[i] = strides[i];
     return true;
 }
 
 namespace {
 bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
-                            const uint32_t* box, bool swizzle128) {
+                            const uint64_t* strides, const uint32_t* box, bool swizzle128) {
     std::call_once(g_once, lookup);
     if (!g_encode) return false;
     cuuint64_t gdim[5];
     cuuint64_t gstride[4];
     cuuint32_t bdim[5], estride[5];
-    uint64_t stride = 2;  // bytes per element
     for (int i = 0; i < rank; ++i) {
         gdim[i] = dims[i];
         bdim[i] = box[i];
         estride[i] = 1;
-        stride *= dims[i];
-        if (i + 1 < rank) gstride[i] = stride;
+        if (i + 1 < rank) gstride[i] = strides[i] * 2;  // bytes
     }
     const CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim,
                                 gstride, bdim, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,

@@ -233,6 +233,95 @@ def test_single_launch_kernel_zero_rows_and_few_planes():
 
 
 # ---------------------------------------------------------------------------
+# strided layouts: token-major [B,N,H,d], a fused [B,N,3,H,d] projection buffer, padded token rows
+# ---------------------------------------------------------------------------
+def _strided_views(call, layout, dev):
+    """q, k, v, out as [B,H,N,d] views of differently laid out device buffers, plus the buffer that holds out."""
+    s = call.shape
+    B, H, N, d = s.B, s.H, s.N, s.d
+    dt = s.torch_dtype()
+    if layout == "token_major":
+        mk = lambda t: t.permute(0, 2, 1, 3).contiguous().to(dev).permute(0, 2, 1, 3)
+        q, k, v = mk(call.q), mk(call.k), mk(call.v)
+        obuf = torch.full((B, N, H, d), 7.0, dtype=dt, device=dev)
+        out = obuf.permute(0, 2, 1, 3)
+    elif layout == "fused_qkv":
+        qkv = torch.stack([t.permute(0, 2, 1, 3) for t in (call.q, call.k, call.v)], dim=2).contiguous().to(dev)  # [B,N,3,H,d]
+        q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+        obuf = torch.full((B, N, H, d), 7.0, dtype=dt, device=dev)
+        out = obuf.permute(0, 2, 1, 3)
+    else:  # "padded": head-major with token rows twice as long as d
+        def mk(t):
+            buf = torch.full((B, H, N, 2 * d), 7.0, dtype=dt, device=dev)
+            buf[..., :d] = t.to(dev)
+            return buf[..., :d]
+        q, k, v = mk(call.q), mk(call.k), mk(call.v)
+        obuf = torch.full((B, H, N, 2 * d), 7.0, dtype=dt, device=dev)
+        out = obuf[..., :d]
+    return q, k, v, out, obuf
+
+
+# B, H, gridH, gridW, d, ksize, dtype, kernel family expected for the token-major layout
+LAYOUT_CASES = [(2, 3, 9, 11, 32, 3, "f32", 1), (2, 4, 14, 14, 64, 3, "bf16", 2), (2, 3, 24, 20, 64, 3, "bf16", 2),
+                (1, 2, 37, 53, 64, 5, "bf16", 2), (2, 4, 14, 14, 32, 3, "bf16", 1), (64, 2, 7, 7, 32, 3, "bf16", 1),
+                (1, 1, 7, 8, 64, 3, "bf16", 2), (3, 1, 8, 16, 64, 3, "bf16", 2), (2, 2, 40, 66, 32, 5, "bf16", 1)]
+
+
+@pytest.mark.parametrize("layout", ["token_major", "fused_qkv", "padded"])
+@pytest.mark.parametrize("case", LAYOUT_CASES, ids=lambda c: "x".join(map(str, c[:7])))
+def test_strided_layouts(case, layout):
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    *shape, dtype, family = case
+    c = workloads.custom_call(*shape, dtype, seed=800 + sum(shape))
+    s = c.shape
+    dev = torch.device("cuda:0")
+    q, k, v, out, obuf = _strided_views(c, layout, dev)
+    assert not out.is_contiguous() or s.H == 1 or s.N == 1
+    w, b = c.dw_weight.to(dev), c.dw_bias.to(dev)
+    with CastlingAttn(ksize=s.ksize) as attn:
+        attn.forward(q, k, v, w, b, s.gridH, s.gridW, out=out)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+        used, _ = attn.last_path()
+    if layout == "padded":
+        assert bool((obuf[..., s.d:] == 7.0).all()), "wrote into the padding between token rows"
+        if s.d == 32 and dtype == "bf16" and s.N >= 96 and s.gridW % 2 == 0:
+            family = 1  # padded rows break the two-tokens-per-row view of width-32 heads too
+    elif s.d == 32 and dtype == "bf16":
+        family = 1
+    assert used == family, f"kernel family {used}, expected {family}"
+    assert rel_err(out, run_oracle(c)) <= TOL[dtype]
+
+
+def test_strided_entry_point_rejects_bad_strides():
+    from paper_2211_10526_b200 import binding
+    c = workloads.custom_call(2, 2, 4, 4, 32, 3, "f32", seed=801)
+    dev = torch.device("cuda:0")
+    q, k, v, w, b = (t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias))
+    out = torch.empty_like(q)
+    h = binding.castling_attn_create(3)
+    good = [2 * 16 * 32, 16 * 32, 32] * 4
+    call = lambda st, o=out: binding.castling_attn_forward_strided(
+        h, q.data_ptr(), k.data_ptr(), v.data_ptr(), w.data_ptr(), b.data_ptr(), o.data_ptr(), 2, 2, 4, 4, 32,
+        binding.CASTLING_F32, st)
+    try:
+        assert call(good) == binding.OK
+        torch.cuda.synchronize()
+        assert rel_err(out, run_oracle(c)) <= TOL["f32"]
+        bad = list(good); bad[2] = 16          # token stride shorter than d
+        assert call(bad) == binding.ERR_INVALID_ARG
+        bad = list(good); bad[5] = 34          # not a multiple of 16 bytes
+        assert call(bad) == binding.ERR_ALIGNMENT
+        bad = list(good); bad[6] = 0           # B > 1 with batch stride 0
+        assert call(bad) == binding.ERR_INVALID_ARG
+        bad = list(good); bad[9] = -1024
+        assert call(bad) == binding.ERR_INVALID_ARG
+        assert call(good, q) == binding.ERR_INVALID_ARG  # out aliases an input
+    finally:
+        binding.castling_attn_destroy(h)
+
+
+# ---------------------------------------------------------------------------
 # kernel families: the tensor-core path must be the one that runs where it applies
 # ---------------------------------------------------------------------------
 TENSOR_SHAPES = [(2, 8, 32, 32, 64, 3), (1, 2, 8, 16, 64, 3), (1, 1, 1, 1, 64, 3), (2, 3, 14, 14, 64, 3),
