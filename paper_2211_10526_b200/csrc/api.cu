@@ -41,7 +41,13 @@ size_t workspace_words(int BH, int N, int d, bool bf16) {
         if (Pt > P) P = Pt;
         words = castling::tc::kStateWords;
     }
-    return castling::kHeaderWords + (size_t)BH * words * (1 + (P > 1 ? P : 0));
+    size_t slots = (size_t)BH * (P > 1 ? P : 0);  // partial states behind the BH final ones
+    if (bf16 && d == 32 && BH % 2 == 0) {
+        // two width-32 heads side by side (token-major layouts): BH / 2 planes of N rows each
+        const int Pp = castling::tc::choose_splits(BH / 2, N);
+        if (Pp > 1 && (size_t)(BH / 2) * Pp > slots) slots = (size_t)(BH / 2) * Pp;
+    }
+    return castling::kHeaderWords + ((size_t)BH + slots) * words;
 }
 
 int fail_cuda(castling_attn* h, cudaError_t e, int code = CASTLING_ERR_CUDA) {

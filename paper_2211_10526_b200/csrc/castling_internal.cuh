@@ -38,6 +38,9 @@ struct Problem {
     bool bf16;
     float eps2;        // eps^2: the floor under the sum of squares
     Layout lq, lk, lv, lo;  // where token n of plane i of q, k, v, out starts: plane_offset(l, i, hdiv) + n * l.token
+    bool blockdiag = false;  // tensor-core path only: a width-64 plane holds two independent width-32 heads side by
+                             // side (heads h, h+1 of a layout whose head stride is 32): rows are normalised per
+                             // half and only the two diagonal 32 x 32 blocks of the state are used
     int hdiv;          // planes per batch step of the layouts: H for a caller's strided tensors, BH for a
                        // run of contiguous planes (one uniform plane stride)
     // Contiguous [planes][N][d] tensors; needs N, d and BH.

@@ -57,6 +57,7 @@ struct ApplyParams {
     int P;
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
+    int blockdiag;                 // the plane is two width-32 heads side by side (one-token-per-row geometry only)
     int H, head0, bh0, hdiv, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
@@ -182,6 +183,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                             lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
                             hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
                         }
+                        if (prm.blockdiag && ((i < 32) != (part < 2))) {  // off-diagonal block: the other head's keys
+                            lo = make_float4(0.f, 0.f, 0.f, 0.f); hi = lo;
+                        }
                     } else {
                         // operand = blockdiag(S32, S32) with S32 = block(0,0) + block(1,1) of the paired sums
                         const int col = part * 16 + c * 8;  // first of 8 columns
@@ -238,8 +242,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             // barrier makes both halves of every row's sum of squares visible
             if (it > 0 && leader) tma_store_wait_read();
             named_barrier_sync(1, kEpiThreads);
-            const float rq = PAIR ? rsqrtf(fmaxf(rq_s[half * kTile + row], prm.eps2))   // half row = one token
-                                  : rsqrtf(fmaxf(rq_s[row] + rq_s[kTile + row], prm.eps2));
+            const float rq = (PAIR || prm.blockdiag)
+                                 ? rsqrtf(fmaxf(rq_s[half * kTile + row], prm.eps2))   // half row = one token / one head
+                                 : rsqrtf(fmaxf(rq_s[row] + rq_s[kTile + row], prm.eps2));
             const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
             uint8_t* orow = out_s + row * 128;
 #pragma unroll
@@ -383,6 +388,7 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0; prm.hdiv = p.hdiv;
+    prm.blockdiag = (!PAIR && p.blockdiag) ? 1 : 0;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
     prm.eps2 = p.eps2; prm.status = status;

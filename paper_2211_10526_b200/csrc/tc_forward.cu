@@ -9,19 +9,32 @@ namespace {
 constexpr int kStateTile = 128;  // tokens per UMMA stage of the state kernel
 }
 
-// bf16 with head width 64, or head width 32 on a grid of even width (two tokens share one
-// 128-byte row there); 3x3 or 5x5 filters.
+namespace {
+// Width-32 heads fill a 128-byte row in one of two ways: two adjacent tokens of one head (tokens
+// contiguous, even grid width), or the same token of two adjacent heads (head stride 32, as in a
+// token-major [B,N,H,32] tensor with an even number of heads).
+bool token_pairs(const Problem& p) { return p.d == 32 && p.gridW % 2 == 0 && p.contiguous_tokens(); }
+bool head_pairs(const Problem& p) {
+    return p.d == 32 && p.H % 2 == 0 && p.hdiv == p.H && p.head0 == 0 && p.lq.head == 32 && p.lk.head == 32 &&
+           p.lv.head == 32 && p.lo.head == 32;
+}
+}  // namespace
+
+// bf16, 3x3 or 5x5 filters, head width 64 or one of the two width-32 arrangements above.
 bool supports(const Problem& p) {
     if (!p.bf16 || (p.ksize != 3 && p.ksize != 5)) return false;
-    // width-32 heads pair two adjacent tokens in one 128-byte row: the tokens must be contiguous
-    return p.d == 64 || (p.d == 32 && p.gridW % 2 == 0 && p.contiguous_tokens());
+    return p.d == 64 || token_pairs(p) || head_pairs(p);
 }
 
 int rows_per_head(int N, int d) { return d == 32 ? N / 2 : N; }
 
 // With fewer than 48 rows per (b,h) the 128-row tiles of the tensor-core kernels are mostly padding
 // and the CUDA-core kernels are faster (measured: 4x4 grids of width-32 heads, 20 us against 33 us).
-bool preferred(const Problem& p) { return supports(p) && rows_per_head(p.N, p.d) >= 48; }
+bool preferred(const Problem& p) {
+    if (!supports(p)) return false;
+    const int rows = (p.d == 32 && !token_pairs(p)) ? p.N : rows_per_head(p.N, p.d);
+    return rows >= 48;
+}
 
 // Two state CTAs fit on an SM: as many splits as keep all CTAs of the launch resident at once
 // (2 x 148), every split non-empty, at most 64 splits.
@@ -36,9 +49,16 @@ int choose_splits(int BH, int N) {
     return (tiles + per - 1) / per;
 }
 
-cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsigned* counters, int P,
+cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
+    Problem p = p_in;
+    if (p.d == 32 && !token_pairs(p)) {
+        // heads (2m, 2m+1) side by side = one width-64 plane whose state is block diagonal
+        p.d = 64; p.H /= 2; p.BH /= 2; p.hdiv = p.H; p.blockdiag = true;
+        p.lq.head = p.lk.head = p.lv.head = p.lo.head = 64;
+        P = choose_splits(p.BH, p.N);
+    }
     if (fused_supports(p)) {  // a whole (b,h) fits in shared memory: one kernel, no workspace
         const cudaError_t e = launch_fused(p, status, stream);
         if (e != cudaSuccess) return e;

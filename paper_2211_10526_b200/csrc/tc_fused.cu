@@ -39,8 +39,9 @@ constexpr int kSeg = 8;                          // tokens of one grid row per c
 constexpr int kOffK = 0, kOffV = kBufBytes, kOffQ = 2 * kBufBytes;
 constexpr int kOffS = 3 * kBufBytes;            // S' 64 x 64 bf16
 constexpr int kOffOnes = kOffS + 8192;          // constant block of the A operand (after K: positive offset)
-constexpr int kOffRq = kOffOnes + 2048;         // [256] 1 / max(||q||, eps)
-constexpr int kOffSum = kOffRq + 256 * 4;       // [64] token sum of V (directly after rq: ragged units read up to 7 floats past rq)
+constexpr int kRqStride = 256 + kSeg;           // ragged units read up to kSeg - 1 entries past token N - 1
+constexpr int kOffRq = kOffOnes + 2048;         // [2][kRqStride] 1 / max(||q||, eps); second row: second half (blockdiag)
+constexpr int kOffSum = kOffRq + 2 * kRqStride * 4;  // [64] token sum of V
 constexpr int kOffZero = kOffSum + kD * 4;      // 128 B of zeros: the convolution's padding
 constexpr int kOffBar = kOffZero + 128;
 constexpr size_t kSmemBytes = 1024 + kOffBar + 128;
@@ -50,6 +51,7 @@ struct FusedParams {
     const __nv_bfloat16* bias;  // [H*64] or nullptr
     __nv_bfloat16* out;         // token n of plane i at plane_offset(lo, i, hdiv) + n * lo.token
     Layout lo;
+    int blockdiag;              // the plane is two width-32 heads side by side
     int H, head0, BH, hdiv, N, gridH, gridW;
     float eps2;
     unsigned* status;
@@ -210,7 +212,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             if (wt < N) {
                 uint8_t* row = K_s + wt * 128;
                 uint4 c[8];
-                float2 ss[4] = {zero2, zero2, zero2, zero2};  // four independent chains
+                float2 ss[4] = {zero2, zero2, zero2, zero2};  // two chains for each half of the row
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     c[j] = *reinterpret_cast<const uint4*>(row + ((j ^ (wt & 7)) << 4));
@@ -218,14 +220,16 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 p = make_float2(bf16lo(w4[e]), bf16hi(w4[e]));
-                        ss[e] = ffma2(p, p, ss[e]);
+                        ss[2 * (j >> 2) + (e & 1)] = ffma2(p, p, ss[2 * (j >> 2) + (e & 1)]);
                     }
                 }
-                const float rk = 1.0f / sqrtf(fmaxf(((ss[0].x + ss[0].y) + (ss[1].x + ss[1].y)) + ((ss[2].x + ss[2].y) + (ss[3].x + ss[3].y)), prm.eps2));
-                const float2 rk2 = make_float2(rk, rk);
+                const float sa = (ss[0].x + ss[0].y) + (ss[1].x + ss[1].y), sb = (ss[2].x + ss[2].y) + (ss[3].x + ss[3].y);
+                const float rka = 1.0f / sqrtf(fmaxf(prm.blockdiag ? sa : sa + sb, prm.eps2));
+                const float rkb = prm.blockdiag ? 1.0f / sqrtf(fmaxf(sb, prm.eps2)) : rka;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const uint32_t w4[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
+                    const float2 rk2 = (j < 4) ? make_float2(rka, rka) : make_float2(rkb, rkb);
                     uint32_t o4[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -250,10 +254,12 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 p = make_float2(bf16lo(w4[e]), bf16hi(w4[e]));
-                        ss[e] = ffma2(p, p, ss[e]);
+                        ss[2 * (j >> 2) + (e & 1)] = ffma2(p, p, ss[2 * (j >> 2) + (e & 1)]);
                     }
                 }
-                rq_s[wt] = rsqrtf(fmaxf(((ss[0].x + ss[0].y) + (ss[1].x + ss[1].y)) + ((ss[2].x + ss[2].y) + (ss[3].x + ss[3].y)), prm.eps2));
+                const float sa = (ss[0].x + ss[0].y) + (ss[1].x + ss[1].y), sb = (ss[2].x + ss[2].y) + (ss[3].x + ss[3].y);
+                rq_s[wt] = rsqrtf(fmaxf(prm.blockdiag ? sa : sa + sb, prm.eps2));
+                rq_s[kRqStride + wt] = rsqrtf(fmaxf(sb, prm.eps2));  // read only when the halves are separate heads
             }
 
             // ---- S, s out of TMEM -> S' (bf16 operand) and s ----
@@ -270,13 +276,14 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     for (int e = 0; e < 16; ++e) { a[e] = a0[e]; a[16 + e] = a1[e]; }
                 }
                 if (quarter < 2) {  // row r of S (key feature r), 32 value features
+                    const float sp = (prm.blockdiag && quarter != half) ? 0.f : kInvPi;  // other head's block: zero
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         uint4 o;
-                        o.x = pack_bf16x2(a[8 * e + 0] * kInvPi, a[8 * e + 1] * kInvPi);
-                        o.y = pack_bf16x2(a[8 * e + 2] * kInvPi, a[8 * e + 3] * kInvPi);
-                        o.z = pack_bf16x2(a[8 * e + 4] * kInvPi, a[8 * e + 5] * kInvPi);
-                        o.w = pack_bf16x2(a[8 * e + 6] * kInvPi, a[8 * e + 7] * kInvPi);
+                        o.x = pack_bf16x2(a[8 * e + 0] * sp, a[8 * e + 1] * sp);
+                        o.y = pack_bf16x2(a[8 * e + 2] * sp, a[8 * e + 3] * sp);
+                        o.z = pack_bf16x2(a[8 * e + 4] * sp, a[8 * e + 5] * sp);
+                        o.w = pack_bf16x2(a[8 * e + 6] * sp, a[8 * e + 7] * sp);
                         *reinterpret_cast<uint4*>(S_s + r * 128 + (((half * 4 + e) ^ (r & 7)) << 4)) = o;
                     }
                 } else if (lane == 0) {  // accumulator row 64: the token sum of V
@@ -331,6 +338,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             uint32_t* out_plane = reinterpret_cast<uint32_t*>(prm.out + plane_offset(prm.lo, bh, prm.hdiv)) + lane;
             const long long out_tok = OUT_PACKED ? kD / 2 : prm.lo.token / 2;  // 32-bit words per token step
             const int sc = lane >> 1, sw = (lane & 1) * 8;  // chunk and offset of the lane's pair in an fp32 row
+            const float* rq_l = rq_s + ((prm.blockdiag && lane >= 16) ? kRqStride : 0);  // the norm of the lane's head
             // Branch-free inside a unit: a neighbour outside the grid is read from a row of zeros, the
             // columns of a ragged last unit are computed (from in-bounds shared memory) and not stored.
             const uint32_t k_base = smem_u32(K_s) + lane * 4, z_addr = smem_u32(smem + kOffZero) + lane * 4;
@@ -369,10 +377,10 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         float2 acc = part[0];
 #pragma unroll
                         for (int dy = 1; dy < KS; ++dy) { acc.x += part[dy].x; acc.y += part[dy].y; }
-                        const int t = y * W + x0 + j, tr = t & (kTile - 1);  // t < N + kSeg: inside rq_s | sum_s
+                        const int t = y * W + x0 + j, tr = t & (kTile - 1);  // t < N + kSeg: inside a row of rq_s
                         const uint8_t* srow = (t < kTile ? V_s : Q_s) + tr * 256;
                         const float2 a2 = *reinterpret_cast<const float2*>(srow + ((sc ^ (tr & 7)) << 4) + sw);
-                        const float rq = rq_s[t];
+                        const float rq = rq_l[t];
                         const float2 o = ffma2(a2, make_float2(rq, rq), acc);
                         if (j < nx) out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
                     }
@@ -407,6 +415,7 @@ cudaError_t launch_fused_ks(const Problem& p, unsigned* status, cudaStream_t st)
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.out = static_cast<__nv_bfloat16*>(p.out);
     prm.lo = p.lo;
+    prm.blockdiag = p.blockdiag ? 1 : 0;
     prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv; prm.N = p.N; prm.gridH = p.gridH; prm.gridW = p.gridW;
     prm.eps2 = p.eps2; prm.status = status;
     static PerDevice opt_in[2];  // per instantiation

@@ -25,6 +25,8 @@ constexpr int kTmemCols = 128;                // two 64-column accumulators: a C
 constexpr int kGroup = 4;                    // splits per first-level reduction group
 constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
+// PAIR = true also serves two width-32 heads stored side by side in one 128-byte row (same arithmetic,
+// the consumer keeps the two diagonal blocks apart instead of adding them).
 // PAIR = true serves head width 32: the [N][32] tensors are viewed as [N/2][64], one 128-byte row
 // holding two consecutive tokens.  The same contraction then yields the four 32 x 32 blocks
 // [k_even^T v_even, k_even^T v_odd; k_odd^T v_even, k_odd^T v_odd]; the state is the sum of the two
@@ -304,7 +306,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
 cudaError_t launch_state(const Problem& p, float* partial, float* final_state, unsigned* counters, int P,
                          int tiles_per_cta, unsigned* status, cudaStream_t st) {
-    const bool pair = (p.d == 32);
+    const bool pair = (p.d == 32);          // two tokens per 128-byte row
+    const bool halves = pair || p.blockdiag;  // each half of a row has its own norm
     const int rows = pair ? p.N / 2 : p.N;  // 128-byte rows per (b,h)
     CUtensorMap tmK, tmV;
     // [64, rows, planes per batch step, batch steps]; a 128-byte row is one token, or two adjacent ones
@@ -319,8 +322,8 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
         return cudaErrorNotSupported;
     static PerDevice opt_in[2];
     {
-        const cudaError_t e = pair ? opt_in_smem(tc_state_kernel<true>, kSmemBytes, opt_in[1])
-                                   : opt_in_smem(tc_state_kernel<false>, kSmemBytes, opt_in[0]);
+        const cudaError_t e = halves ? opt_in_smem(tc_state_kernel<true>, kSmemBytes, opt_in[1])
+                                     : opt_in_smem(tc_state_kernel<false>, kSmemBytes, opt_in[0]);
         if (e != cudaSuccess) return e;
     }
     float* dst = P > 1 ? partial : final_state;
@@ -330,7 +333,7 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
         items = (p.BH + 295) / 296;
         grid = (p.BH + items - 1) / items;
     }
-    if (pair)
+    if (halves)
         tc_state_kernel<true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(
             tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, p.hdiv, items, p.eps2, status);
     else

@@ -264,7 +264,9 @@ def _strided_views(call, layout, dev):
 # B, H, gridH, gridW, d, ksize, dtype, kernel family expected for the token-major layout
 LAYOUT_CASES = [(2, 3, 9, 11, 32, 3, "f32", 1), (2, 4, 14, 14, 64, 3, "bf16", 2), (2, 3, 24, 20, 64, 3, "bf16", 2),
                 (1, 2, 37, 53, 64, 5, "bf16", 2), (2, 4, 14, 14, 32, 3, "bf16", 1), (64, 2, 7, 7, 32, 3, "bf16", 1),
-                (1, 1, 7, 8, 64, 3, "bf16", 2), (3, 1, 8, 16, 64, 3, "bf16", 2), (2, 2, 40, 66, 32, 5, "bf16", 1)]
+                (1, 1, 7, 8, 64, 3, "bf16", 2), (3, 1, 8, 16, 64, 3, "bf16", 2), (2, 2, 40, 66, 32, 5, "bf16", 1),
+                (2, 6, 33, 21, 32, 3, "bf16", 1), (3, 3, 16, 16, 32, 3, "bf16", 1), (1, 8, 5, 7, 32, 5, "bf16", 1),
+                (8, 8, 64, 64, 32, 5, "bf16", 1)]
 
 
 @pytest.mark.parametrize("layout", ["token_major", "fused_qkv", "padded"])
@@ -285,12 +287,55 @@ def test_strided_layouts(case, layout):
         used, _ = attn.last_path()
     if layout == "padded":
         assert bool((obuf[..., s.d:] == 7.0).all()), "wrote into the padding between token rows"
-        if s.d == 32 and dtype == "bf16" and s.N >= 96 and s.gridW % 2 == 0:
-            family = 1  # padded rows break the two-tokens-per-row view of width-32 heads too
-    elif s.d == 32 and dtype == "bf16":
-        family = 1
+    if s.d == 32 and dtype == "bf16":
+        # token-major width-32 heads: two heads share a 128-byte row on the tensor-core path (even H, at least
+        # 48 tokens); padded rows leave neither two tokens nor two heads side by side
+        family = 2 if (layout != "padded" and s.H % 2 == 0 and s.N >= 48) else 1
     assert used == family, f"kernel family {used}, expected {family}"
     assert rel_err(out, run_oracle(c)) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("grid", [(12, 20), (24, 20)], ids=["one_kernel", "two_kernels"])
+def test_token_major_head_pairs_term_isolation(grid):
+    """Width-32 heads stored [B,N,H,32]: two heads share a 128-byte row on the tensor-core path.  With the
+    other terms removed, any leak between the two heads of a row (the off-diagonal blocks of the paired
+    state, a norm taken over the whole row) is the whole error."""
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    gh, gw = grid
+    dev = torch.device("cuda:0")
+
+    def run(c):
+        s = c.shape
+        q, k, v, out, _ = _strided_views(c, "token_major", dev)
+        with CastlingAttn(ksize=s.ksize) as attn:
+            attn.forward(q, k, v, c.dw_weight.to(dev), c.dw_bias.to(dev), gh, gw, out=out)
+            torch.cuda.synchronize()
+            assert attn.device_status() == (0, 0)
+            assert attn.last_path()[0] == binding.PATH_TENSOR
+        err = rel_err(out, run_oracle(c))
+        assert err <= TOL["bf16"], err
+
+    base = lambda seed: workloads.custom_call(2, 4, gh, gw, 32, 3, "bf16", seed=seed)
+    c = base(631)  # linear term alone, heads of very different scale
+    v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+    c.v[:, 1::2] *= 64
+    c.q[:, 0::2] *= 1e-3; c.k[:, 1::2] *= 1e3
+    c.dw_weight.zero_(); c.dw_bias.zero_()
+    run(c)
+    c = base(632)  # one head of each pair has all-zero keys: its linear term vanishes, its neighbour's does not
+    v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+    c.k[:, 0::2] = 0
+    c.dw_weight.zero_(); c.dw_bias.zero_()
+    run(c)
+    c = base(633)  # 1/2 sum (constant V per head)
+    c.v[:] = c.v[:, :, :1, :].clone()
+    c.dw_weight.zero_(); c.dw_bias.zero_()
+    run(c)
+    c = base(634)  # convolution alone
+    v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(torch.bfloat16)
+    c.dw_weight = (c.dw_weight.float() * 30).to(torch.bfloat16)
+    c.k.zero_()
+    run(c)
 
 
 def test_strided_entry_point_rejects_bad_strides():
