@@ -40,6 +40,8 @@ def _declare(lib: ctypes.CDLL) -> ctypes.CDLL:
     i, dbl = ctypes.c_int, ctypes.c_double
     lib.castling_oracle_forward.restype = i
     lib.castling_oracle_forward.argtypes = [_dp] * 6 + [i] * 6 + [dbl, i, i]
+    lib.castling_oracle_forward_prefix.restype = i
+    lib.castling_oracle_forward_prefix.argtypes = [_dp] * 6 + [i] * 7 + [dbl, i, i]
     lib.castling_oracle_forward_bruteforce.restype = i
     lib.castling_oracle_forward_bruteforce.argtypes = [_dp] * 6 + [i] * 6 + [dbl]
     lib.castling_oracle_similarity.restype = i
@@ -74,12 +76,12 @@ def _ptr(a: Optional[np.ndarray]):
     return None if a is None else a.ctypes.data_as(_dp)
 
 
-def _check_shapes(q, k, v, w, bias, gridH, gridW, ksize):
+def _check_shapes(q, k, v, w, bias, gridH, gridW, ksize, prefix=0):
     if q.ndim != 4 or q.shape != k.shape or q.shape != v.shape:
         raise ValueError("q, k, v must share one [B, H, N, d] shape")
     B, H, N, d = q.shape
-    if N != gridH * gridW:
-        raise ValueError("N != gridH * gridW")
+    if N != prefix + gridH * gridW:
+        raise ValueError("N != prefix + gridH * gridW")
     if w.shape != (H * d, ksize, ksize):
         raise ValueError("dw_weight must be [H*d, ksize, ksize]")
     if bias is not None and bias.shape != (H * d,):
@@ -88,21 +90,27 @@ def _check_shapes(q, k, v, w, bias, gridH, gridW, ksize):
 
 
 def forward(q, k, v, dw_weight, dw_bias, gridH: int, gridW: int, ksize: int,
-            eps: float = DEFAULT_EPS, threads: int = 1, lib: Optional[ctypes.CDLL] = None) -> np.ndarray:
+            eps: float = DEFAULT_EPS, threads: int = 1, lib: Optional[ctypes.CDLL] = None,
+            prefix: int = 0) -> np.ndarray:
     """Linear-angular attention core, re-associated form, float64.  Returns [B,H,N,d].
 
     ``threads`` > 1 splits the independent (b,h) heads over host threads; each
-    thread runs the same single-threaded C routine on its own slice.
+    thread runs the same single-threaded C routine on its own slice.  ``prefix`` > 0:
+    the first ``prefix`` tokens of every sequence are off-grid (class tokens): they take
+    part in the attention terms but not in the depthwise convolution.
     """
     lib = lib or load()
     q, k, v, w = _f64(q), _f64(k), _f64(v), _f64(dw_weight)
     bias = None if dw_bias is None else _f64(dw_bias)
-    B, H, N, d = _check_shapes(q, k, v, w, bias, gridH, gridW, ksize)
+    B, H, N, d = _check_shapes(q, k, v, w, bias, gridH, gridW, ksize, prefix)
     out = np.empty_like(q)
     BH = B * H
     threads = max(1, min(int(threads), BH))
 
     def run(lo: int, hi: int) -> int:
+        if prefix:
+            return lib.castling_oracle_forward_prefix(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(bias), _ptr(out),
+                                                      B, H, int(prefix), gridH, gridW, d, ksize, float(eps), lo, hi)
         return lib.castling_oracle_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(bias), _ptr(out),
                                            B, H, gridH, gridW, d, ksize, float(eps), lo, hi)
 

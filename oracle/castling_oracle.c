@@ -162,6 +162,61 @@ int castling_oracle_forward(const double* q, const double* k, const double* v,
     return 0;
 }
 
+/* ---- leading tokens that are not on the grid (class / distillation tokens) ----
+ * Reading taken where the paper is silent: a sequence may start with `prefix` tokens that
+ * have no grid position.  They attend and are attended to like every other token (they
+ * enter S, the token sum and get an output row from Eq. 9's attention terms), but the
+ * depthwise convolution (and its bias) is defined on the 2-D grid only: it reads and
+ * writes the gridH*gridW tokens that follow the prefix and contributes nothing to the
+ * prefix rows.  prefix = 0 is castling_oracle_forward. */
+int castling_oracle_forward_prefix(const double* q, const double* k, const double* v,
+                                   const double* w, const double* bias, double* out,
+                                   int B, int H, int prefix, int gridH, int gridW, int d, int ksize,
+                                   double eps, int bh_begin, int bh_end)
+{
+    if (!q || !k || !v || !w || !out) return -1;
+    if (B <= 0 || H <= 0 || prefix < 0 || gridH <= 0 || gridW <= 0 || d <= 0) return -1;
+    if (ksize <= 0 || (ksize & 1) == 0) return -1;
+    if (bh_begin < 0 || bh_end > B * H || bh_begin > bh_end) return -1;
+    const int G = gridH * gridW, T = prefix + G;           /* T tokens per sequence */
+    double* state = (double*)malloc(sizeof(double) * d * d);
+    double* tok_sum = (double*)malloc(sizeof(double) * d);
+    double* u = (double*)malloc(sizeof(double) * d);
+    double* grid_conv = (double*)malloc(sizeof(double) * (size_t)G * d);
+    if (!state || !tok_sum || !u || !grid_conv) { free(state); free(tok_sum); free(u); free(grid_conv); return -1; }
+
+    for (int bh = bh_begin; bh < bh_end; ++bh) {
+        const int h = bh % H;
+        const size_t base = (size_t)bh * T * d;
+        const double* qp = q + base; const double* kp = k + base; const double* vp = v + base;
+        double* op = out + base;
+
+        memset(state, 0, sizeof(double) * d * d);
+        memset(tok_sum, 0, sizeof(double) * d);
+        for (int m = 0; m < T; ++m) {                      /* every token, prefix included */
+            unit_row(kp + (size_t)m * d, d, eps, u);
+            for (int a = 0; a < d; ++a)
+                for (int c = 0; c < d; ++c)
+                    state[a * d + c] += u[a] * vp[(size_t)m * d + c];
+            for (int c = 0; c < d; ++c) tok_sum[c] += vp[(size_t)m * d + c];
+        }
+
+        dwconv_head(vp + (size_t)prefix * d, w, bias, h, gridH, gridW, d, ksize, grid_conv);  /* grid tokens only */
+
+        for (int m = 0; m < T; ++m) {
+            unit_row(qp + (size_t)m * d, d, eps, u);
+            for (int c = 0; c < d; ++c) {
+                double dot = 0.0;
+                for (int a = 0; a < d; ++a) dot += u[a] * state[a * d + c];
+                const double on_grid = (m >= prefix) ? grid_conv[(size_t)(m - prefix) * d + c] : 0.0;
+                op[(size_t)m * d + c] = tok_sum[c] / 2.0 + dot / M_PI + on_grid;
+            }
+        }
+    }
+    free(state); free(tok_sum); free(u); free(grid_conv);
+    return 0;
+}
+
 /* ---- the definition written out: explicit N x N similarity matrix -------
  * Sim[t][j] = 1/2 + (q^_t . k^_j)/pi (Eq. 8), A = Sim V (Eq. 9), plus the
  * depthwise convolution.  O(N^2 d); for small N only. */

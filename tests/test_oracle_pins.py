@@ -373,11 +373,42 @@ def pin_threads_agree(lib):
     _close(a, c, 0.0)
 
 
+def pin_prefix_tokens(lib):
+    """Off-grid leading tokens (class tokens): attention terms over all tokens, convolution on the grid only.
+
+    Pinned against the plain forward (itself pinned above) and a library convolution: with the filter bank
+    zeroed the result is the plain forward of the same sequence on a 1 x T grid (the attention terms do not
+    know about the grid); the difference the filters make is scipy's 2-D correlation of the grid tokens of V
+    plus the bias, and exactly zero on the prefix rows."""
+    from scipy.signal import correlate2d
+    B, H, P, gh, gw, d, ks = 2, 2, 2, 3, 4, 5, 3
+    T = P + gh * gw
+    rng = np.random.default_rng(131)
+    q, k, v = (rng.standard_normal((B, H, T, d)) for _ in range(3))
+    w = 0.3 * rng.standard_normal((H * d, ks, ks)); b = 0.3 * rng.standard_normal((H * d,))
+    wz, bz = _zero_filter(H, d, ks)
+    att = oracle.forward(q, k, v, wz, bz, gh, gw, ks, lib=lib, prefix=P)
+    _close(att, oracle.forward(q, k, v, wz, bz, 1, T, ks, lib=lib), 1e-12)
+    full = oracle.forward(q, k, v, w, b, gh, gw, ks, lib=lib, prefix=P)
+    diff = full - att
+    assert float(np.max(np.abs(diff[:, :, :P]))) == 0.0, "the convolution touched a prefix row"
+    for bb in range(B):
+        for h in range(H):
+            for j in range(d):
+                img = v[bb, h, P:, j].reshape(gh, gw)
+                want = correlate2d(img, w[h * d + j], mode="same", boundary="fill", fillvalue=0.0) + b[h * d + j]
+                _close(diff[bb, h, P:, j].reshape(gh, gw), want, 1e-12)
+    # prefix = 0 is the plain forward; threads agree
+    q0, k0, v0, w0, b0 = _problem(1, 2, 3, 3, 4, 3, 132)
+    _close(oracle.forward(q0, k0, v0, w0, b0, 3, 3, 3, lib=lib, prefix=0), oracle.forward(q0, k0, v0, w0, b0, 3, 3, 3, lib=lib), 0.0)
+    _close(oracle.forward(q, k, v, w, b, gh, gw, ks, lib=lib, prefix=P, threads=3), full, 0.0)
+
+
 PINS = [pin_worked_example, pin_series_coefficients, pin_angular_values, pin_series_properties,
         pin_bruteforce_equals_linear, pin_similarity_matrix, pin_constant_v, pin_equal_keys,
         pin_d_equals_one, pin_zero_rows, pin_conv_known_filters, pin_conv_head_channel_mapping,
         pin_conv_matrix_form, pin_conv_library_routine, pin_scale_invariance,
-        pin_linearity_and_symmetry, pin_threads_agree]
+        pin_linearity_and_symmetry, pin_threads_agree, pin_prefix_tokens]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -417,6 +448,14 @@ MISTAKES = [
     ("series_coefficient", "c *= (2.0 * i - 1.0) / (2.0 * i);", "c *= (2.0 * i - 1.0) / (2.0 * i + 1.0);", 1),
     ("series_constant", "double sum = 0.5 + x / M_PI;", "double sum = 0.5 + x / 3.0;", 1),
     ("exact_kernel_sign", "return 1.0 - acos(x) / M_PI;", "return acos(x) / M_PI;", 1),
+    ("prefix_left_out_of_state", "for (int m = 0; m < T; ++m) {                      /* every token, prefix included */",
+     "for (int m = prefix; m < T; ++m) {", 1),
+    ("prefix_conv_reads_from_token_zero", "dwconv_head(vp + (size_t)prefix * d,", "dwconv_head(vp,", 1),
+    ("prefix_rows_get_conv", "(m >= prefix) ? grid_conv[(size_t)(m - prefix) * d + c] : 0.0;",
+     "grid_conv[(size_t)(m >= prefix ? m - prefix : m) * d + c];", 1),
+    ("prefix_conv_row_offset", "grid_conv[(size_t)(m - prefix) * d + c] : 0.0;", "grid_conv[(size_t)(m - prefix + 1 < G ? m - prefix + 1 : 0) * d + c] : 0.0;", 1),
+    ("prefix_half_term", "tok_sum[c] / 2.0 + dot / M_PI + on_grid;", "tok_sum[c] + dot / M_PI + on_grid;", 1),
+    ("prefix_state_transposed", "dot += u[a] * state[a * d + c];", "dot += u[a] * state[c * d + a];", 1),
 ]
 
 
