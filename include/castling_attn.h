@@ -74,11 +74,17 @@ typedef struct {
                           /* row therefore has cosine 0 with everything (similarity 1/2).     */
     int force_path;       /* CASTLING_PATH_*; AUTO picks by dtype, d and N                     */
     size_t max_workspace; /* cap on handle-owned device memory in bytes; 0 = no cap            */
+    int prefix_tokens;    /* 0..16 leading tokens per sequence that have no grid position (class */
+                          /* / distillation tokens).  N becomes prefix_tokens + gridH*gridW in     */
+                          /* every forward call.  The paper does not say how such tokens meet the */
+                          /* convolution; here they enter both attention terms of Eq. 9 like any  */
+                          /* token (they add to K^^T V and to the token sum, and get an output    */
+                          /* row), while DWConv and its bias act on the grid tokens only.         */
 } castling_attn_config_t;
 
 /*
  * castling_attn_create: make a handle bound to the CURRENT CUDA device.
- *   cfg         host pointer, read once; NULL selects {ksize 3, eps 1e-12, AUTO, no cap}.
+ *   cfg         host pointer, read once; NULL selects {ksize 3, eps 1e-12, AUTO, no cap, no prefix}.
  *   out_handle  host pointer receiving the handle; set to NULL on failure.
  * Allocates nothing on the device.  Errors: INVALID_ARG, UNSUPPORTED (ksize), ARCH, CUDA.
  */
@@ -88,8 +94,9 @@ CASTLING_API int castling_attn_create(const castling_attn_config_t* cfg, castlin
  * castling_attn_forward: enqueue one forward pass on `stream` and return without
  * synchronising (Eq. 8-9 as stated at the top of this file).
  *
- *   q, k, v     DEVICE pointers, [B, H, N, d] contiguous, d innermost, N = gridH*gridW,
- *               token t = y*gridW + x.  Read only.  16-byte aligned.
+ *   q, k, v     DEVICE pointers, [B, H, N, d] contiguous, d innermost, N = prefix_tokens +
+ *               gridH*gridW, grid token (y, x) at t = prefix_tokens + y*gridW + x.  Read only.
+ *               16-byte aligned.
  *   dw_weight   DEVICE pointer, [H*d, ksize, ksize], same dtype as q.  Read only.
  *   dw_bias     DEVICE pointer, [H*d], same dtype, or NULL for no bias.
  *   out         DEVICE pointer, [B, H, N, d], same dtype; every element is written exactly
@@ -171,7 +178,9 @@ CASTLING_API int castling_attn_forward_host(castling_attn_t* handle,
  */
 CASTLING_API int castling_attn_destroy(castling_attn_t* handle);
 
-/* Bytes of handle-owned device workspace a forward of this shape needs (0 on bad arguments). */
+/* Bytes of handle-owned device workspace a forward of this shape needs (0 on bad arguments).  The
+ * figure is for sequences of gridH*gridW tokens; a handle with prefix_tokens may need one more
+ * partial-state slot per (b,h). */
 CASTLING_API size_t castling_attn_workspace_bytes(int B, int H, int gridH, int gridW, int d, castling_dtype_t dtype);
 
 /* Static, NUL-terminated description of a return code. */

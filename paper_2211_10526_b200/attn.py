@@ -33,9 +33,11 @@ class CastlingAttn:
     the result has been copied back.
     """
 
-    def __init__(self, ksize: int = 3, eps: float = 0.0, force_path: int = _b.PATH_AUTO, max_workspace: int = 0):
+    def __init__(self, ksize: int = 3, eps: float = 0.0, force_path: int = _b.PATH_AUTO, max_workspace: int = 0,
+                 prefix_tokens: int = 0):
         self.ksize = int(ksize)
-        self._h = _b.castling_attn_create(ksize, eps, force_path, max_workspace)
+        self.prefix_tokens = int(prefix_tokens)  # leading off-grid (class) tokens: N = prefix_tokens + gridH * gridW
+        self._h = _b.castling_attn_create(ksize, eps, force_path, max_workspace, prefix_tokens)
 
     def close(self) -> None:
         if getattr(self, "_h", None):
@@ -64,8 +66,8 @@ class CastlingAttn:
         if len(shape) != 4 or k.shape != shape or v.shape != shape or out.shape != shape:
             raise ValueError("q, k, v, out must share one [B, H, N, d] shape")
         B, H, N, d = shape
-        if N != gridH * gridW:
-            raise ValueError("N != gridH * gridW")
+        if N != self.prefix_tokens + gridH * gridW:
+            raise ValueError("N != prefix_tokens + gridH * gridW")
         ks = self.ksize
         if w.shape != (H * d, ks, ks):
             raise ValueError("dw_weight must be [H*d, ksize, ksize]")

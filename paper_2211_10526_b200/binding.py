@@ -23,7 +23,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 
 class castling_attn_config_t(ctypes.Structure):
     _fields_ = [("ksize", ctypes.c_int), ("eps", ctypes.c_double), ("force_path", ctypes.c_int),
-                ("max_workspace", ctypes.c_size_t)]
+                ("max_workspace", ctypes.c_size_t), ("prefix_tokens", ctypes.c_int)]
 
 
 class castling_attn_layout_t(ctypes.Structure):
@@ -80,9 +80,9 @@ def error_string(code: int) -> str:
 
 
 def castling_attn_create(ksize: int = 3, eps: float = 0.0, force_path: int = PATH_AUTO,
-                         max_workspace: int = 0) -> int:
+                         max_workspace: int = 0, prefix_tokens: int = 0) -> int:
     """Returns the handle (an integer address); raises CastlingError on failure."""
-    cfg = castling_attn_config_t(int(ksize), float(eps), int(force_path), int(max_workspace))
+    cfg = castling_attn_config_t(int(ksize), float(eps), int(force_path), int(max_workspace), int(prefix_tokens))
     h = ctypes.c_void_p()
     rc = lib.castling_attn_create(ctypes.byref(cfg), ctypes.byref(h))
     if rc != OK:

@@ -67,7 +67,7 @@ int check_shape(const castling_attn* h, int B, int H, int gridH, int gridW, int 
     if (B <= 0 || H <= 0 || gridH <= 0 || gridW <= 0 || d <= 0) return CASTLING_ERR_INVALID_ARG;
     if (dtype != CASTLING_F32 && dtype != CASTLING_BF16) return CASTLING_ERR_UNSUPPORTED;
     if (!castling::simt_supports(d, h->cfg.ksize)) return CASTLING_ERR_UNSUPPORTED;
-    const long long N = (long long)gridH * gridW, BH = (long long)B * H;
+    const long long N = (long long)gridH * gridW + h->cfg.prefix_tokens, BH = (long long)B * H;
     if (N > (1 << 24) || BH > (1 << 20) || BH * ((N + 63) / 64) > 0x7fffffffLL) return CASTLING_ERR_UNSUPPORTED;
     if (BH * N * d > (1LL << 40)) return CASTLING_ERR_UNSUPPORTED;
     return CASTLING_OK;
@@ -113,12 +113,14 @@ extern "C" {
 int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** out_handle) {
     if (!out_handle) return CASTLING_ERR_INVALID_ARG;
     *out_handle = nullptr;
-    castling_attn_config_t c = {3, 1e-12, CASTLING_PATH_AUTO, 0};
+    castling_attn_config_t c = {3, 1e-12, CASTLING_PATH_AUTO, 0, 0};
     if (cfg) c = *cfg;
     if (c.eps <= 0.0) c.eps = 1e-12;
     if (c.ksize <= 0 || (c.ksize & 1) == 0) return CASTLING_ERR_INVALID_ARG;
     if (c.ksize > 7) return CASTLING_ERR_UNSUPPORTED;
     if (c.force_path < CASTLING_PATH_AUTO || c.force_path > CASTLING_PATH_TENSOR) return CASTLING_ERR_INVALID_ARG;
+    if (c.prefix_tokens < 0) return CASTLING_ERR_INVALID_ARG;
+    if (c.prefix_tokens > 16) return CASTLING_ERR_UNSUPPORTED;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail_cuda(nullptr, e);
@@ -227,7 +229,8 @@ Problem make_problem(const castling_attn* h, const void* q, const void* k, const
     Problem p;
     p.q = q; p.k = k; p.v = v; p.w = w; p.bias = bias; p.out = out;
     p.B = B; p.H = H; p.gridH = gridH; p.gridW = gridW; p.d = d; p.ksize = h->cfg.ksize;
-    p.N = gridH * gridW; p.BH = B * H; p.head0 = 0;
+    p.prefix = h->cfg.prefix_tokens;
+    p.N = p.prefix + gridH * gridW; p.BH = B * H; p.head0 = 0;
     p.bf16 = (dtype == CASTLING_BF16);
     p.eps2 = (float)(h->cfg.eps * h->cfg.eps);
     p.set_contiguous();
@@ -250,7 +253,7 @@ int castling_attn_forward(castling_attn_t* h, const void* q, const void* k, cons
     if (rc != CASTLING_OK) return rc;
     if (!q || !k || !v || !dw_weight || !out) return CASTLING_ERR_INVALID_ARG;
     const size_t eb = elem_bytes(dtype);
-    const size_t tensor_bytes = (size_t)B * H * gridH * gridW * d * eb;
+    const size_t tensor_bytes = (size_t)B * H * (h->cfg.prefix_tokens + (size_t)gridH * gridW) * d * eb;
     const size_t w_bytes = (size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb;
     const size_t b_bytes = (size_t)H * d * eb;
     const void* ptrs[4] = {q, k, v, out};
@@ -271,7 +274,7 @@ int castling_attn_forward_strided(castling_attn_t* h, const void* q, const void*
     int rc = check_shape(h, B, H, gridH, gridW, d, dtype);
     if (rc != CASTLING_OK) return rc;
     if (!q || !k || !v || !dw_weight || !out || !layout) return CASTLING_ERR_INVALID_ARG;
-    const long long eb = (long long)elem_bytes(dtype), N = (long long)gridH * gridW;
+    const long long eb = (long long)elem_bytes(dtype), N = (long long)gridH * gridW + h->cfg.prefix_tokens;
     const long long* s = &layout->q_batch;  // twelve strides: q, k, v, out x (batch, head, token)
     long long ext[4];
     for (int t = 0; t < 4; ++t) {
@@ -309,7 +312,8 @@ int castling_attn_forward_host(castling_attn_t* h, const void* q, const void* k,
     if (!q || !k || !v || !dw_weight || !out) return CASTLING_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t eb = elem_bytes(dtype);
-    const size_t tb = (((size_t)B * H * gridH * gridW * d * eb) + 255) & ~(size_t)255;
+    const size_t n_tok = h->cfg.prefix_tokens + (size_t)gridH * gridW;
+    const size_t tb = (((size_t)B * H * n_tok * d * eb) + 255) & ~(size_t)255;
     const size_t wb = (((size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb) + 255) & ~(size_t)255;
     const size_t bb = (((size_t)H * d * eb) + 255) & ~(size_t)255;
     const size_t need = 4 * tb + wb + bb;
@@ -325,7 +329,7 @@ int castling_attn_forward_host(castling_attn_t* h, const void* q, const void* k,
     }
     char* dq = h->stage; char* dk = dq + tb; char* dv = dk + tb; char* dout = dv + tb;
     char* dw = dout + tb; char* db = dw + wb;
-    const size_t t_exact = (size_t)B * H * gridH * gridW * d * eb;
+    const size_t t_exact = (size_t)B * H * n_tok * d * eb;
     cudaError_t e;
     if ((e = cudaMemcpyAsync(dw, dw_weight, (size_t)H * d * h->cfg.ksize * h->cfg.ksize * eb,
                              cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail_cuda(h, e);

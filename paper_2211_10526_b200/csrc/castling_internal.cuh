@@ -32,7 +32,8 @@ struct Problem {
     const void* bias;  // [H*d] or nullptr
     void* out;
     int B, H, gridH, gridW, d, ksize;
-    int N;             // gridH * gridW
+    int prefix = 0;    // leading off-grid tokens (class tokens): attended like the rest, not convolved
+    int N;             // tokens per sequence: prefix + gridH * gridW
     int BH;            // B * H (the (b,h) planes of this call)
     int head0;         // head index of plane 0: plane i uses the filters of head (head0 + i) % H
     bool bf16;

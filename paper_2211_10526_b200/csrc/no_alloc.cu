@@ -79,7 +79,7 @@ extern "C" int castling_attn_forward_static(const void* q, const void* k, const 
     castling::Problem p;
     p.q = q; p.k = k; p.v = v; p.w = dw_weight; p.bias = dw_bias; p.out = out;
     p.B = B; p.H = H; p.gridH = gridH; p.gridW = gridW; p.d = d; p.ksize = ksize;
-    p.N = (int)N; p.BH = (int)BH; p.head0 = 0;
+    p.prefix = 0; p.N = (int)N; p.BH = (int)BH; p.head0 = 0;
     p.set_contiguous();
     p.bf16 = (dtype == CASTLING_BF16);
     if (eps <= 0.0) eps = 1e-12;

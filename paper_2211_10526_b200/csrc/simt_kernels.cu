@@ -187,26 +187,27 @@ simt_reduce_kernel(const float* __restrict__ partial, float* __restrict__ state,
 // Thread (tq, tj) owns tokens tq + 16 r (r = 0..3) and channels tj*R .. tj*R + R - 1.
 // ---------------------------------------------------------------------------
 template <int D> constexpr size_t simt_apply_smem(int ksize) {
-    return sizeof(float) * ((size_t)D * D + D + (size_t)ksize * ksize * D + kApplyTile * (D + 1) + kApplyTile);
+    return sizeof(float) * ((size_t)D * D + 2 * D + (size_t)ksize * ksize * D + kApplyTile * (D + 1) + kApplyTile);
 }
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __restrict__ w,
                   const T* __restrict__ bias, const float* __restrict__ state, T* __restrict__ out,
-                  int H, int head0, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lv, Layout lo,
-                  int hdiv) {
+                  int H, int head0, int prefix, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lv,
+                  Layout lo, int hdiv) {
     constexpr int R = D / 16;
     constexpr int LDQ = D + 1;
     extern __shared__ __align__(16) float smem[];
     const int KK = ksize * ksize, rad = (ksize - 1) / 2;
     float* S_sm = smem;                 // [D][D], scaled by 1/pi
-    float* c_sm = S_sm + D * D;         // [D]    1/2 s + bias
-    float* w_sm = c_sm + D;             // [KK][D] filters of this head, tap-major
+    float* c_sm = S_sm + D * D;         // [D]    1/2 s
+    float* b_sm = c_sm + D;             // [D]    bias of the convolution (grid tokens only)
+    float* w_sm = b_sm + D;             // [KK][D] filters of this head, tap-major
     float* qs = w_sm + KK * D;          // [64][D+1]
     float* rq = qs + kApplyTile * LDQ;  // [64]
 
-    const int N = gridH * gridW;
+    const int N = prefix + gridH * gridW;
     const int tiles = (N + kApplyTile - 1) / kApplyTile;
     const int bh = blockIdx.x / tiles, h = (head0 + bh) % H;
     const int t0 = (blockIdx.x % tiles) * kApplyTile;
@@ -214,8 +215,10 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
     const float* st = state + (size_t)bh * (D * D + D);
 
     for (int i = threadIdx.x; i < D * D; i += kThreads) S_sm[i] = st[i] * kInvPi;
-    for (int i = threadIdx.x; i < D; i += kThreads)
-        c_sm[i] = 0.5f * st[D * D + i] + (bias ? Elem<T>::load1(bias + h * D + i) : 0.f);
+    for (int i = threadIdx.x; i < D; i += kThreads) {
+        c_sm[i] = 0.5f * st[D * D + i];
+        b_sm[i] = bias ? Elem<T>::load1(bias + h * D + i) : 0.f;
+    }
     for (int i = threadIdx.x; i < KK * D; i += kThreads) {
         const int tap = i / D, ch = i % D;
         w_sm[i] = Elem<T>::load1(w + ((size_t)(h * D + ch)) * KK + tap);
@@ -266,18 +269,18 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
     for (int r = 0; r < 4; ++r) {
         const int tl = tq + 16 * r;
         if (tl >= valid) continue;
-        const int t = t0 + tl, y = t / gridW, x = t % gridW;
+        const int t = t0 + tl, g = t - prefix, y = g / gridW, x = g % gridW;  // g < 0: an off-grid leading token
         const float scale = rq[tl];
         float o[R];
 #pragma unroll
-        for (int c = 0; c < R; ++c) o[c] = fmaf(acc[r][c], scale, c_sm[tj * R + c]);
-        for (int dy = -rad; dy <= rad; ++dy) {
+        for (int c = 0; c < R; ++c) o[c] = fmaf(acc[r][c], scale, c_sm[tj * R + c] + (g >= 0 ? b_sm[tj * R + c] : 0.f));
+        for (int dy = -rad; dy <= rad && g >= 0; ++dy) {
             const int yy = y + dy;
             if (yy < 0 || yy >= gridH) continue;
             for (int dx = -rad; dx <= rad; ++dx) {
                 const int xx = x + dx;
                 if (xx < 0 || xx >= gridW) continue;
-                const T* vp = vb + (yy * gridW + xx) * lv.token + tj * R;
+                const T* vp = vb + (prefix + yy * gridW + xx) * lv.token + tj * R;
                 const float* wp = w_sm + ((dy + rad) * ksize + (dx + rad)) * D + tj * R;
 #pragma unroll
                 for (int c = 0; c < R; ++c) o[c] = fmaf(wp[c], Elem<T>::load1(vp + c), o[c]);
@@ -302,7 +305,7 @@ constexpr int kFusedMinPlanes = 64;
 constexpr size_t kFusedSmemLimit = 100 * 1024;
 
 template <int D> constexpr size_t simt_fused_smem(int N, int ksize) {
-    return sizeof(float) * (3 * (size_t)N * (D + 4) + 2 * (size_t)N + (size_t)D * D + D + (size_t)ksize * ksize * D);
+    return sizeof(float) * (3 * (size_t)N * (D + 4) + 2 * (size_t)N + (size_t)D * D + 2 * D + (size_t)ksize * ksize * D);
 }
 
 // 1 / max(||row||, eps) for `rows` rows of a shared tile, one warp per row at a time.
@@ -322,12 +325,12 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                   const T* __restrict__ w, const T* __restrict__ bias, T* __restrict__ out,
-                  int H, int head0, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lk, Layout lv,
-                  Layout lo, int hdiv) {
+                  int H, int head0, int prefix, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lk,
+                  Layout lv, Layout lo, int hdiv) {
     constexpr int R = D / 16;
     constexpr int LD = D + 4;
     extern __shared__ __align__(16) float smem[];
-    const int N = gridH * gridW;
+    const int N = prefix + gridH * gridW;
     const int KK = ksize * ksize, rad = (ksize - 1) / 2;
     float* ks = smem;               // [N][LD]
     float* vs = ks + N * LD;        // [N][LD]
@@ -335,8 +338,9 @@ simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
     float* rk = qs + N * LD;        // [N]
     float* rq = rk + N;             // [N]
     float* S_sm = rq + N;           // [D][D], scaled by 1/pi
-    float* c_sm = S_sm + D * D;     // [D]    1/2 s + bias
-    float* w_sm = c_sm + D;         // [KK][D] filters of this head, tap-major
+    float* c_sm = S_sm + D * D;     // [D]    1/2 s
+    float* b_sm = c_sm + D;         // [D]    bias of the convolution (grid tokens only)
+    float* w_sm = b_sm + D;         // [KK][D] filters of this head, tap-major
 
     const int bh = blockIdx.x, h = (head0 + bh) % H;
     stage_plane<T, D, LD>(k + plane_offset(lk, bh, hdiv), lk.token, ks, N);
@@ -382,7 +386,8 @@ simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
 #pragma unroll
             for (int y = 0; y < R; ++y) {
                 const int ch = tj * R + y;
-                c_sm[ch] = 0.5f * vsum[y] + (bias ? Elem<T>::load1(bias + h * D + ch) : 0.f);
+                c_sm[ch] = 0.5f * vsum[y];
+                b_sm[ch] = bias ? Elem<T>::load1(bias + h * D + ch) : 0.f;
             }
         }
     }
@@ -416,18 +421,18 @@ simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
         for (int r = 0; r < 4; ++r) {
             const int t = t0 + tq + 16 * r;
             if (t >= N) continue;
-            const int y = t / gridW, x = t % gridW;
+            const int g = t - prefix, y = g / gridW, x = g % gridW;  // g < 0: an off-grid leading token
             const float scale = rq[t];
             float o[R];
 #pragma unroll
-            for (int c = 0; c < R; ++c) o[c] = fmaf(acc[r][c], scale, c_sm[tj * R + c]);
-            for (int dy = -rad; dy <= rad; ++dy) {
+            for (int c = 0; c < R; ++c) o[c] = fmaf(acc[r][c], scale, c_sm[tj * R + c] + (g >= 0 ? b_sm[tj * R + c] : 0.f));
+            for (int dy = -rad; dy <= rad && g >= 0; ++dy) {
                 const int yy = y + dy;
                 if (yy < 0 || yy >= gridH) continue;
                 for (int dx = -rad; dx <= rad; ++dx) {
                     const int xx = x + dx;
                     if (xx < 0 || xx >= gridW) continue;
-                    const float* vp = vs + (yy * gridW + xx) * LD + tj * R;
+                    const float* vp = vs + (prefix + yy * gridW + xx) * LD + tj * R;
                     const float* wp = w_sm + ((dy + rad) * ksize + (dx + rad)) * D + tj * R;
 #pragma unroll
                     for (int c = 0; c < R; ++c) o[c] = fmaf(wp[c], vp[c], o[c]);
@@ -450,7 +455,7 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
         simt_fused_kernel<T, D><<<(unsigned)p.BH, kThreads, smem, stream>>>(
             static_cast<const T*>(p.q), static_cast<const T*>(p.k), static_cast<const T*>(p.v),
             static_cast<const T*>(p.w), static_cast<const T*>(p.bias), static_cast<T*>(p.out),
-            p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2, p.lq, p.lk, p.lv, p.lo, p.hdiv);
+            p.H, p.head0, p.prefix, p.gridH, p.gridW, p.ksize, p.eps2, p.lq, p.lk, p.lv, p.lo, p.hdiv);
         e = cudaGetLastError();
         if (e == cudaSuccess) *launches = 1;
         timer->mark(stream, "simt_fused");
@@ -479,8 +484,8 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     const unsigned grid = (unsigned)(p.BH * ((p.N + kApplyTile - 1) / kApplyTile));
     simt_apply_kernel<T, D><<<grid, kThreads, smem, stream>>>(
         static_cast<const T*>(p.q), static_cast<const T*>(p.v), static_cast<const T*>(p.w),
-        static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.head0, p.gridH, p.gridW, p.ksize, p.eps2,
-        p.lq, p.lv, p.lo, p.hdiv);
+        static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.head0, p.prefix, p.gridH, p.gridW, p.ksize,
+        p.eps2, p.lq, p.lv, p.lo, p.hdiv);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     timer->mark(stream, "simt_apply");

@@ -379,8 +379,12 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     };
     uint64_t sq[4], sv[4], so[4];
     strides(p.lq, sq); strides(p.lv, sv); strides(p.lo, so);
-    if (!make_tensor_map_bf16(&tmQ, p.q, 5, dims, sq, box, true) || !make_tensor_map_bf16(&tmO, p.out, 5, dims, so, box, true) ||
-        !make_tensor_map_bf16(&tmV, p.v, 5, dims, sv, boxv, false))
+    // the token grid starts after the off-grid leading tokens of every plane
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + p.prefix * p.lq.token;
+    const __nv_bfloat16* vg = static_cast<const __nv_bfloat16*>(p.v) + p.prefix * p.lv.token;
+    __nv_bfloat16* og = static_cast<__nv_bfloat16*>(p.out) + p.prefix * p.lo.token;
+    if (!make_tensor_map_bf16(&tmQ, qg, 5, dims, sq, box, true) || !make_tensor_map_bf16(&tmO, og, 5, dims, so, box, true) ||
+        !make_tensor_map_bf16(&tmV, vg, 5, dims, sv, boxv, false))
         return cudaErrorNotSupported;
     ApplyParams prm;
     prm.state = state;
@@ -409,7 +413,57 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS, PAIR>, tmQ, tmV, tmO, prm);
 }
 
+// Output rows of the off-grid leading tokens: out = q^ S / pi + 1/2 s (no convolution, no bias), from the
+// final state the state kernel left in the workspace.  One block of 64 threads per (plane, token), thread =
+// channel.  mode 0: 64-wide heads; 1: token pairs (width 32, the state is the sum of the two diagonal
+// blocks); 2: two width-32 heads side by side (each half of the row is its own head).
+__global__ void __launch_bounds__(64)
+tc_prefix_rows_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
+                      const float* __restrict__ state, Layout lq, Layout lo, int hdiv, int prefix, int mode,
+                      float eps2) {
+    __shared__ float qs[kD];
+    __shared__ float part[2];
+    const int plane = blockIdx.x / prefix, t = blockIdx.x % prefix, j = threadIdx.x;
+    const int width = (mode == 1) ? 32 : kD;  // elements of this plane's token rows
+    const __nv_bfloat16* qrow = q + plane_offset(lq, plane, hdiv) + t * lq.token;
+    const float x = (j < width) ? __bfloat162float(qrow[j]) : 0.f;
+    qs[j] = x;
+    float ss = x * x;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((j & 31) == 0) part[j >> 5] = ss;
+    __syncthreads();
+    if (j >= width) return;
+    const float* st = state + (size_t)plane * (kD * kD + kD);
+    float nrm2, acc = 0.f, sum;
+    if (mode == 0) {
+        nrm2 = part[0] + part[1];
+        for (int i = 0; i < kD; ++i) acc = fmaf(qs[i], st[i * kD + j], acc);
+        sum = st[kD * kD + j];
+    } else if (mode == 1) {
+        nrm2 = part[0];
+        for (int i = 0; i < 32; ++i) acc = fmaf(qs[i], st[i * kD + j] + st[(32 + i) * kD + 32 + j], acc);
+        sum = st[kD * kD + j] + st[kD * kD + 32 + j];
+    } else {
+        const int h0 = j & 32;  // first channel of this thread's head within the row
+        nrm2 = part[j >> 5];
+        for (int i = 0; i < 32; ++i) acc = fmaf(qs[h0 + i], st[(h0 + i) * kD + j], acc);
+        sum = st[kD * kD + j];
+    }
+    const float o = fmaf(acc * kInvPi, rsqrtf(fmaxf(nrm2, eps2)), 0.5f * sum);
+    out[plane_offset(lo, plane, hdiv) + t * lo.token + j] = __float2bfloat16_rn(o);
+}
+
 }  // namespace
+
+cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_t st) {
+    if (p.prefix <= 0) return cudaSuccess;
+    const int mode = p.d == 32 ? 1 : (p.blockdiag ? 2 : 0);
+    tc_prefix_rows_kernel<<<(unsigned)(p.BH * p.prefix), 64, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(p.q), static_cast<__nv_bfloat16*>(p.out), state, p.lq, p.lo, p.hdiv,
+        p.prefix, mode, p.eps2);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st) {
     if (p.d == 32)

@@ -52,7 +52,7 @@ struct FusedParams {
     __nv_bfloat16* out;         // token n of plane i at plane_offset(lo, i, hdiv) + n * lo.token
     Layout lo;
     int blockdiag;              // the plane is two width-32 heads side by side
-    int H, head0, BH, hdiv, N, gridH, gridW;
+    int H, head0, BH, hdiv, prefix, N, gridH, gridW;  // N = prefix + gridH * gridW
     float eps2;
     unsigned* status;
 };
@@ -333,8 +333,9 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 for (int dx = 0; dx < KS; ++dx)
                     wreg[dy][dx] = make_float2(__uint_as_float((uint32_t)wraw[0][dy * KS + dx] << 16),
                                                __uint_as_float((uint32_t)wraw[1][dy * KS + dx] << 16));
-            const float2 c2 = make_float2(fmaf(0.5f, sum_s[2 * lane], __uint_as_float((uint32_t)braw[0] << 16)),
-                                          fmaf(0.5f, sum_s[2 * lane + 1], __uint_as_float((uint32_t)braw[1] << 16)));
+            const float2 hs2 = make_float2(0.5f * sum_s[2 * lane], 0.5f * sum_s[2 * lane + 1]);  // 1/2 s
+            const float2 c2 = make_float2(hs2.x + __uint_as_float((uint32_t)braw[0] << 16),
+                                          hs2.y + __uint_as_float((uint32_t)braw[1] << 16));  // + bias: grid tokens
             uint32_t* out_plane = reinterpret_cast<uint32_t*>(prm.out + plane_offset(prm.lo, bh, prm.hdiv)) + lane;
             const long long out_tok = OUT_PACKED ? kD / 2 : prm.lo.token / 2;  // 32-bit words per token step
             const int sc = lane >> 1, sw = (lane & 1) * 8;  // chunk and offset of the lane's pair in an fp32 row
@@ -350,7 +351,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 for (int dy = 0; dy < KS; ++dy) {
                     const int yy = y + dy - R;
                     const bool rv = (unsigned)yy < (unsigned)prm.gridH;
-                    ra[dy] = rv ? k_base + (uint32_t)((yy * W + x0) * 128) : z_addr;
+                    ra[dy] = rv ? k_base + (uint32_t)((prm.prefix + yy * W + x0) * 128) : z_addr;
                     rstep[dy] = rv ? 128u : 0u;
                 }
                 float2 win[KS][KS];  // column x0 - R + jj lives in slot jj % KS
@@ -377,7 +378,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         float2 acc = part[0];
 #pragma unroll
                         for (int dy = 1; dy < KS; ++dy) { acc.x += part[dy].x; acc.y += part[dy].y; }
-                        const int t = y * W + x0 + j, tr = t & (kTile - 1);  // t < N + kSeg: inside a row of rq_s
+                        const int t = prm.prefix + y * W + x0 + j, tr = t & (kTile - 1);  // t < N + kSeg: inside a row of rq_s
                         const uint8_t* srow = (t < kTile ? V_s : Q_s) + tr * 256;
                         const float2 a2 = *reinterpret_cast<const float2*>(srow + ((sc ^ (tr & 7)) << 4) + sw);
                         const float rq = rq_l[t];
@@ -385,6 +386,13 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         if (j < nx) out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
                     }
                 }
+            }
+            // off-grid leading tokens: the attention terms only
+            for (int t = ww; t < prm.prefix; t += kWorkers / 32) {
+                const float2 a2 = *reinterpret_cast<const float2*>(V_s + t * 256 + ((sc ^ (t & 7)) << 4) + sw);
+                const float rq = rq_l[t];
+                const float2 o = ffma2(a2, make_float2(rq, rq), hs2);
+                out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
             }
             fence_proxy_async_smem();
             mbar_arrive(plane_free);
@@ -416,7 +424,8 @@ cudaError_t launch_fused_ks(const Problem& p, unsigned* status, cudaStream_t st)
     prm.out = static_cast<__nv_bfloat16*>(p.out);
     prm.lo = p.lo;
     prm.blockdiag = p.blockdiag ? 1 : 0;
-    prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv; prm.N = p.N; prm.gridH = p.gridH; prm.gridW = p.gridW;
+    prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv; prm.prefix = p.prefix; prm.N = p.N;
+    prm.gridH = p.gridH; prm.gridW = p.gridW;
     prm.eps2 = p.eps2; prm.status = status;
     static PerDevice opt_in[2];  // per instantiation
     const bool packed = (p.lo.token == kD);

@@ -39,6 +39,8 @@ cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsign
 cudaError_t launch_state(const Problem& p, float* partial, float* final_state, unsigned* counters, int P,
                          int tiles_per_cta, unsigned* status, cudaStream_t st);
 cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st);
+// Output rows of the off-grid leading tokens (p.prefix of them per plane), from the final state.
+cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_t st);
 
 // Single-kernel forward for short sequences (bf16, d = 64, N <= 256, 3x3 or 5x5 filters): no workspace.
 bool fused_supports(const Problem& p);

@@ -233,6 +233,83 @@ def test_single_launch_kernel_zero_rows_and_few_planes():
 
 
 # ---------------------------------------------------------------------------
+# leading off-grid tokens (class tokens): in the attention terms, not in the convolution
+# ---------------------------------------------------------------------------
+def _prefix_call(B, H, P, gh, gw, d, ks, dtype, seed):
+    """Inputs for sequences of P + gh*gw tokens (drawn as one row of that many tokens)."""
+    c = workloads.custom_call(B, H, 1, P + gh * gw, d, ks, dtype, seed=seed)
+    return c
+
+
+# B, H, prefix, gridH, gridW, d, ksize, dtype, layout, kernel family expected, launches expected
+PREFIX_CASES = [
+    (2, 3, 1, 5, 7, 32, 3, "f32", "head_major", 1, 2),       # CUDA cores, three-kernel path (no split)
+    (1, 2, 2, 40, 33, 48, 5, "f32", "head_major", 1, 3),     # CUDA cores, token range split
+    (16, 4, 1, 7, 7, 32, 3, "bf16", "head_major", 1, 1),     # CUDA cores, single-launch kernel (odd N)
+    (4, 12, 1, 14, 14, 64, 3, "bf16", "head_major", 2, 1),   # DeiT-shaped with a class token: single tensor-core kernel
+    (2, 3, 2, 15, 16, 64, 5, "bf16", "head_major", 2, 1),    # 242 tokens, 5 x 5
+    (2, 2, 1, 24, 20, 64, 3, "bf16", "head_major", 2, 3),    # state + apply + leading rows
+    (1, 2, 3, 37, 53, 64, 5, "bf16", "head_major", 2, 3),
+    (2, 2, 2, 24, 20, 32, 3, "bf16", "head_major", 2, 3),    # width 32, even N: token pairs
+    (2, 2, 1, 24, 20, 32, 3, "bf16", "head_major", 1, 3),    # width 32, odd N: CUDA cores (P = 2 splits)
+    (2, 4, 1, 24, 20, 32, 5, "bf16", "token_major", 2, 3),   # width 32 token-major: head pairs
+    (2, 4, 1, 12, 12, 32, 3, "bf16", "token_major", 2, 1),   # ... in the single-kernel forward
+    (2, 3, 1, 14, 14, 64, 3, "bf16", "token_major", 2, 1),
+    (1, 2, 2, 30, 31, 64, 3, "bf16", "fused_qkv", 2, 3),
+]
+
+
+@pytest.mark.parametrize("case", PREFIX_CASES, ids=lambda c: "x".join(map(str, c[:9])))
+def test_prefix_tokens(case):
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    B, H, P, gh, gw, d, ks, dtype, layout, family, n_launch = case
+    c = _prefix_call(B, H, P, gh, gw, d, ks, dtype, seed=900 + sum(case[:7]))
+    dev = torch.device("cuda:0")
+    if layout == "head_major":
+        q, k, v = (t.to(dev) for t in (c.q, c.k, c.v))
+        guard = torch.full((q.numel() + 4096,), 7.0, dtype=q.dtype, device=dev)
+        out = guard[2048:2048 + q.numel()].view_as(q)
+    else:
+        q, k, v, out, _ = _strided_views(c, layout, dev)
+        guard = None
+    w, b = c.dw_weight.to(dev), c.dw_bias.to(dev)
+    with CastlingAttn(ksize=ks, prefix_tokens=P) as attn:
+        attn.forward(q, k, v, w, b, gh, gw, out=out)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+        assert attn.last_path() == (family, n_launch)
+        out_nb = attn.forward(q, k, v, w, None, gh, gw)
+        torch.cuda.synchronize()
+    if guard is not None:
+        assert bool((guard[:2048] == 7.0).all()) and bool((guard[-2048:] == 7.0).all()), "wrote outside the output"
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, gh, gw, ks, threads=8, prefix=P)
+    assert rel_err(out, ref) <= TOL[dtype]
+    ref_nb = oracle.forward(c.q, c.k, c.v, c.dw_weight, None, gh, gw, ks, threads=8, prefix=P)
+    assert rel_err(out_nb, ref_nb) <= TOL[dtype]
+
+
+def test_prefix_tokens_conv_term_alone():
+    """Only the convolution (with a bias of about 3) left: the leading rows stay near zero (what is left of
+    1/2 sum V after rounding), the grid rows are the filtered grid."""
+    from paper_2211_10526_b200 import CastlingAttn
+    dev = torch.device("cuda:0")
+    for dtype, shape in (("f32", (2, 2, 2, 9, 11, 32, 3)), ("bf16", (2, 2, 1, 24, 20, 64, 3)), ("bf16", (2, 2, 1, 12, 16, 64, 5))):
+        B, H, P, gh, gw, d, ks = shape
+        c = _prefix_call(B, H, P, gh, gw, d, ks, dtype, seed=950 + sum(shape))
+        v = c.v.float(); c.v = (v - v.mean(dim=2, keepdim=True)).to(c.v.dtype)
+        c.k.zero_()
+        c.dw_weight = (c.dw_weight.float() * 30).to(c.v.dtype)
+        c.dw_bias = (c.dw_bias.float() + 3).to(c.v.dtype)   # a bias that would show on a leading row
+        with CastlingAttn(ksize=ks, prefix_tokens=P) as attn:
+            out = attn.forward(*(t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)), gh, gw)
+            torch.cuda.synchronize()
+        ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, gh, gw, ks, threads=8, prefix=P)
+        assert rel_err(out, ref) <= TOL[dtype]
+        lead = out[:, :, :P].float().abs().max().item()
+        assert lead < 0.5, f"leading rows carry {lead}: the convolution or its bias leaked"
+
+
+# ---------------------------------------------------------------------------
 # strided layouts: token-major [B,N,H,d], a fused [B,N,3,H,d] projection buffer, padded token rows
 # ---------------------------------------------------------------------------
 def _strided_views(call, layout, dev):
