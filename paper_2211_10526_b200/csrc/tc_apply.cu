@@ -57,16 +57,18 @@ struct ApplyParams {
     int P;
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
-    int blockdiag;                 // the plane is two width-32 heads side by side (one-token-per-row geometry only)
     int H, head0, bh0, hdiv, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
 };
 
-template <int KS, bool PAIR>
-__global__ void __launch_bounds__((Geo<KS, PAIR>::kThreads), 1)
+// MODE 0: width-64 heads; 1: width-32 heads, two adjacent tokens per 128-byte row (the PAIR geometry);
+// 2: two width-32 heads side by side in the one-token-per-row geometry (block-diagonal state).
+template <int KS, int MODE>
+__global__ void __launch_bounds__((Geo<KS, MODE == 1>::kThreads), 1)
 tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmO, const ApplyParams prm) {
+    constexpr bool PAIR = (MODE == 1), BLOCKDIAG = (MODE == 2);
     using G = Geo<KS, PAIR>;
     constexpr int NS = G::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -183,7 +185,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                             lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
                             hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
                         }
-                        if (prm.blockdiag && ((i < 32) != (part < 2))) {  // off-diagonal block: the other head's keys
+                        if (BLOCKDIAG && ((i < 32) != (part < 2))) {  // off-diagonal block: the other head's keys
                             lo = make_float4(0.f, 0.f, 0.f, 0.f); hi = lo;
                         }
                     } else {
@@ -242,7 +244,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             // barrier makes both halves of every row's sum of squares visible
             if (it > 0 && leader) tma_store_wait_read();
             named_barrier_sync(1, kEpiThreads);
-            const float rq = (PAIR || prm.blockdiag)
+            const float rq = (PAIR || BLOCKDIAG)
                                  ? rsqrtf(fmaxf(rq_s[half * kTile + row], prm.eps2))   // half row = one token / one head
                                  : rsqrtf(fmaxf(rq_s[row] + rq_s[kTile + row], prm.eps2));
             const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
@@ -361,8 +363,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int KS, bool PAIR>
+template <int KS, int MODE>
 cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigned* status, cudaStream_t st) {
+    constexpr bool PAIR = (MODE == 1);
     using G = Geo<KS, PAIR>;
     CUtensorMap tmQ, tmV, tmO;
     const int cols = PAIR ? p.gridW / 2 : p.gridW;  // 128-byte columns per grid row
@@ -392,13 +395,12 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0; prm.hdiv = p.hdiv;
-    prm.blockdiag = (!PAIR && p.blockdiag) ? 1 : 0;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
     prm.eps2 = p.eps2; prm.status = status;
     static PerDevice opt_in;  // one per instantiation
     {
-        const cudaError_t e = opt_in_smem(tc_apply_kernel<KS, PAIR>, G::kSmem, opt_in);
+        const cudaError_t e = opt_in_smem(tc_apply_kernel<KS, MODE>, G::kSmem, opt_in);
         if (e != cudaSuccess) return e;
     }
     const int grid = prm.n_tiles < 148 ? prm.n_tiles : 148;
@@ -410,7 +412,7 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS, PAIR>, tmQ, tmV, tmO, prm);
+    return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS, MODE>, tmQ, tmV, tmO, prm);
 }
 
 // Output rows of the off-grid leading tokens: out = q^ S / pi + 1/2 s (no convolution, no bias), from the
@@ -467,10 +469,13 @@ cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_
 
 cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st) {
     if (p.d == 32)
-        return p.ksize == 3 ? launch_apply_ks<3, true>(p, partial, P, status, st)
-                            : launch_apply_ks<5, true>(p, partial, P, status, st);
-    return p.ksize == 3 ? launch_apply_ks<3, false>(p, partial, P, status, st)
-                        : launch_apply_ks<5, false>(p, partial, P, status, st);
+        return p.ksize == 3 ? launch_apply_ks<3, 1>(p, partial, P, status, st)
+                            : launch_apply_ks<5, 1>(p, partial, P, status, st);
+    if (p.blockdiag)
+        return p.ksize == 3 ? launch_apply_ks<3, 2>(p, partial, P, status, st)
+                            : launch_apply_ks<5, 2>(p, partial, P, status, st);
+    return p.ksize == 3 ? launch_apply_ks<3, 0>(p, partial, P, status, st)
+                        : launch_apply_ks<5, 0>(p, partial, P, status, st);
 }
 
 }  // namespace tc
