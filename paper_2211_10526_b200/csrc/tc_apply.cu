@@ -1,4 +1,5 @@
-// Apply kernel of the tensor-core path (bf16, d = 64):
+// Apply kernel of the tensor-core path (bf16; width-64 heads, or width-32 heads packed two to a 128-byte
+// row: see the modes at the kernel template):
 //     out_t = (1/pi) q^_t S + 1/2 s + bias + DWConv(V)_t                         (Eq. 9)
 // Persistent CTAs walk a contiguous range of 8 x 16-token patches of the token grid.  Per patch
 //   warp 0      TMA: the raw Q patch (128 rows of 128 B, 128-byte swizzle) and the V patch with
