@@ -415,6 +415,47 @@ def test_token_major_head_pairs_term_isolation(grid):
     run(c)
 
 
+def _random_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        dtype = "bf16" if rng.random() < 0.7 else "f32"
+        d = int(rng.choice([32, 64, 32, 64, 16, 48, 96, 128])) if dtype == "bf16" else int(rng.choice([16, 32, 64, 80]))
+        ks = int(rng.choice([3, 5, 3, 5, 1, 7]))
+        big = rng.random() < 0.3
+        gh, gw = (int(rng.integers(1, 60)), int(rng.integers(1, 60))) if big else (int(rng.integers(1, 17)), int(rng.integers(1, 17)))
+        B, H = (int(rng.integers(1, 3)), int(rng.integers(1, 5))) if big else (int(rng.integers(1, 40)), int(rng.integers(1, 7)))
+        prefix = int(rng.choice([0, 0, 1, 2, 3]))
+        layout = str(rng.choice(["head_major", "head_major", "token_major", "fused_qkv", "padded"]))
+        cases.append((B, H, prefix, gh, gw, d, ks, dtype, layout, 1000 + i))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_cases(128, 20221118), ids=lambda c: "x".join(map(str, c[:9])))
+def test_random_shapes_layouts_and_leading_tokens(case):
+    """Seeded random shapes across dtypes, head widths, filter sizes, leading tokens and memory layouts:
+    whatever kernel family the dispatcher picks, the result is the oracle's."""
+    from paper_2211_10526_b200 import CastlingAttn
+    B, H, P, gh, gw, d, ks, dtype, layout, seed = case
+    c = _prefix_call(B, H, P, gh, gw, d, ks, dtype, seed=seed)
+    dev = torch.device("cuda:0")
+    if layout == "head_major":
+        q, k, v = (t.to(dev) for t in (c.q, c.k, c.v))
+        out = torch.empty_like(q)
+    else:
+        q, k, v, out, _ = _strided_views(c, layout, dev)
+    bias = c.dw_bias.to(dev) if seed % 4 else None
+    with CastlingAttn(ksize=ks, prefix_tokens=P) as attn:
+        attn.forward(q, k, v, c.dw_weight.to(dev), bias, gh, gw, out=out)
+        again = torch.empty_like(out)
+        attn.forward(q, k, v, c.dw_weight.to(dev), bias, gh, gw, out=again)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias if bias is not None else None, gh, gw, ks, threads=8, prefix=P)
+    assert rel_err(out, ref) <= TOL[dtype]
+    assert torch.equal(out, again), "two runs differ bitwise"
+
+
 def test_strided_entry_point_rejects_bad_strides():
     from paper_2211_10526_b200 import binding
     c = workloads.custom_call(2, 2, 4, 4, 32, 3, "f32", seed=801)
