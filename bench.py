@@ -257,7 +257,7 @@ def main():
         step(i)
     torch.cuda.synchronize()
     path, launches_per_step = attn.last_path()
-    hot_ms = None
+    hot_ms = graph_ms = None
     if n_sets > 1:  # the same number of steps on one set: every input served from L2
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         h0.record(stream)
@@ -266,6 +266,25 @@ def main():
         h1.record(stream)
         torch.cuda.synchronize()
         hot_ms = h0.elapsed_time(h1) / args.steps
+        # the same, replayed from a CUDA graph of 20 forwards: what is left when the host's launch cost is gone
+        graph_ms = None
+        try:
+            side = torch.cuda.Stream(dev)
+            side.wait_stream(stream)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(20):
+                    step(0)
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            graph.replay()
+            g0.record(stream)
+            for _ in range(max(1, args.steps // 20)):
+                graph.replay()
+            g1.record(stream)
+            torch.cuda.synchronize()
+            graph_ms = g0.elapsed_time(g1) / (20 * max(1, args.steps // 20))
+        except Exception as exc:  # reported, never fatal: the headline does not depend on it
+            graph_ms = f"unavailable: {exc}"
         for i in range(n_sets):  # push that set out of L2 again
             step(i)
         torch.cuda.synchronize()
@@ -347,7 +366,7 @@ def main():
                        "head_tokens_per_step": s.head_tokens, "algorithmic_bytes_per_step": s.algorithmic_bytes,
                        "l2": "inputs exceed L2, no flush" if n_sets == 1 else
                              f"cold: ring of {n_sets} copies of q, k, v, out ({n_sets * s.algorithmic_bytes / 1e6:.0f} MB) cycled",
-                       "hot_ms_per_step": hot_ms,
+                       "hot_ms_per_step": hot_ms, "hot_graph_replay_ms_per_step": graph_ms,
                        "layout": "[B,H,N,d]" if args.layout == "head_major" else "[B,N,H,d] (strided views)",
                        "parallelism": "independent replicas" if world > 1 else "single GPU",
                        "arithmetic": "bf16 tensor-core operands, fp32 accumulation" if s.dtype == "bf16" else "fp32",

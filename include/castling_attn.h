@@ -109,6 +109,9 @@ CASTLING_API int castling_attn_create(const castling_attn_config_t* cfg, castlin
  * d x d states, token sums) that may be (re)allocated with cudaMalloc on the first call
  * for a larger shape -- that call synchronises the device; later calls of the same or a
  * smaller shape allocate nothing.
+ * Such later calls only enqueue kernels on `stream` (no allocation, no synchronisation, no
+ * host-side dependence on device results), so they can be recorded by stream capture and replayed
+ * as a CUDA graph on new data in the same buffers.
  * A handle serves one host thread and one stream at a time; distinct handles are
  * independent.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, OOM, CUDA.  Nothing aborts
  * and no exception crosses this boundary.

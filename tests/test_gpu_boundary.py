@@ -194,3 +194,47 @@ def test_host_entry_point_pipelines_batch_chunks():
     for got in (out_h, out_d.cpu()):
         err = np.max(np.abs(got.double().numpy() - ref)) / np.max(np.abs(ref))
         assert err <= 2e-2
+
+
+GRAPH_SHAPES = [  # B, H, prefix, gridH, gridW, d, ksize, dtype: one per kernel family
+    (2, 4, 0, 14, 14, 32, 3, "f32"),     # CUDA-core state + apply
+    (1, 2, 0, 48, 50, 32, 3, "f32"),     # CUDA-core with the token range split (reduce kernel)
+    (64, 8, 0, 7, 7, 32, 3, "bf16"),     # CUDA-core single-launch kernel
+    (4, 12, 1, 14, 14, 64, 3, "bf16"),   # single tensor-core kernel, one leading token
+    (2, 8, 0, 64, 64, 64, 3, "bf16"),    # tensor-core state + apply (programmatic dependent launch), split state
+    (8, 8, 0, 64, 64, 32, 5, "bf16"),    # width-32 token pairs, 5 x 5
+    (2, 2, 2, 24, 20, 64, 3, "bf16"),    # tensor-core path + leading-rows kernel
+]
+
+
+@pytest.mark.parametrize("shape", GRAPH_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_forward_inside_a_cuda_graph(shape):
+    """A forward only enqueues kernels on the caller's stream once its workspace exists, so it can be
+    captured into a CUDA graph and replayed on new data in the same buffers."""
+    from paper_2211_10526_b200 import CastlingAttn
+    B, H, P, gh, gw, d, ks, dtype = shape
+    c1 = workloads.custom_call(B, H, 1, P + gh * gw, d, ks, dtype, seed=470 + sum(shape[:7]))
+    c2 = workloads.custom_call(B, H, 1, P + gh * gw, d, ks, dtype, seed=471 + sum(shape[:7]))
+    dev = torch.device("cuda:0")
+    q, k, v, w, b = (t.to(dev) for t in (c1.q, c1.k, c1.v, c1.dw_weight, c1.dw_bias))
+    out = torch.empty_like(q)
+    side = torch.cuda.Stream()
+    with CastlingAttn(ksize=ks, prefix_tokens=P) as attn:
+        with torch.cuda.stream(side):
+            attn.forward(q, k, v, w, b, gh, gw, out=out)   # first call: allocates the workspace (not capturable)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            attn.forward(q, k, v, w, b, gh, gw, out=out)
+        for t, src in ((q, c2.q), (k, c2.k), (v, c2.v), (w, c2.dw_weight), (b, c2.dw_bias)):
+            t.copy_(src)
+        out.fill_(float("nan"))
+        graph.replay()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+    ref = oracle.forward(c2.q, c2.k, c2.v, c2.dw_weight, c2.dw_bias, gh, gw, ks, threads=8, prefix=P)
+    g = out.double().cpu().numpy()
+    assert np.all(np.isfinite(g))
+    err = float(np.max(np.abs(g - ref)) / np.max(np.abs(ref)))
+    assert err <= (1e-5 if dtype == "f32" else 2e-2), err
