@@ -58,6 +58,7 @@ struct ApplyParams {
     int P;
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
+    int flat;                      // the planes have one uniform stride: the tensor maps are 4-D, [.., plane]
     int H, head0, bh0, hdiv, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
@@ -121,9 +122,14 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
                 uint8_t* qs = stages + s * G::kStage;
                 mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
-                const int pb = bh / prm.hdiv, ph = bh - pb * prm.hdiv;
-                tma_load_5d_hint(qs, &tmQ, &full[s], 0, x0, y0, ph, pb, pol_q);
-                tma_load_5d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, ph, pb);
+                if (prm.flat) {
+                    tma_load_4d_hint(qs, &tmQ, &full[s], 0, x0, y0, bh, pol_q);
+                    tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, bh);
+                } else {
+                    const int pb = bh / prm.hdiv, ph = bh - pb * prm.hdiv;
+                    tma_load_5d_hint(qs, &tmQ, &full[s], 0, x0, y0, ph, pb, pol_q);
+                    tma_load_5d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, ph, pb);
+                }
                 ++issued;
             }
             if (*abort_flag) {
@@ -266,8 +272,12 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             fence_proxy_async_smem();
             named_barrier_sync(1, kEpiThreads);
             if (leader) {
-                const int pb = bh / prm.hdiv;
-                tma_store_5d_hint(&tmO, out_s, 0, x0, y0, bh - pb * prm.hdiv, pb, pol_o);
+                if (prm.flat) {
+                    tma_store_4d_hint(&tmO, out_s, 0, x0, y0, bh, pol_o);
+                } else {
+                    const int pb = bh / prm.hdiv;
+                    tma_store_5d_hint(&tmO, out_s, 0, x0, y0, bh - pb * prm.hdiv, pb, pol_o);
+                }
                 tma_store_commit();
             }
         }
@@ -370,8 +380,10 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     using G = Geo<KS, PAIR>;
     CUtensorMap tmQ, tmV, tmO;
     const int cols = PAIR ? p.gridW / 2 : p.gridW;  // 128-byte columns per grid row
-    // [64, columns, grid rows, planes per batch step, batch steps]
+    // [64, columns, grid rows, planes per batch step, batch steps]; with a single batch step the last
+    // dimension is dropped (a 4-D copy is a little cheaper for the TMA unit than a 5-D one)
     const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
+    const int rank = nb > 1 ? 5 : 4;
     const uint64_t dims[5] = {(uint64_t)kD, (uint64_t)cols, (uint64_t)p.gridH, (uint64_t)p.hdiv, nb};
     const uint32_t box[5] = {kD, kTX, kTY, 1, 1};
     const uint32_t boxv[5] = {kD, (uint32_t)G::HX, (uint32_t)G::HY, 1, 1};
@@ -387,14 +399,15 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + p.prefix * p.lq.token;
     const __nv_bfloat16* vg = static_cast<const __nv_bfloat16*>(p.v) + p.prefix * p.lv.token;
     __nv_bfloat16* og = static_cast<__nv_bfloat16*>(p.out) + p.prefix * p.lo.token;
-    if (!make_tensor_map_bf16(&tmQ, qg, 5, dims, sq, box, true) || !make_tensor_map_bf16(&tmO, og, 5, dims, so, box, true) ||
-        !make_tensor_map_bf16(&tmV, vg, 5, dims, sv, boxv, false))
+    if (!make_tensor_map_bf16(&tmQ, qg, rank, dims, sq, box, true) || !make_tensor_map_bf16(&tmO, og, rank, dims, so, box, true) ||
+        !make_tensor_map_bf16(&tmV, vg, rank, dims, sv, boxv, false))
         return cudaErrorNotSupported;
     ApplyParams prm;
     prm.state = state;
     prm.P = P;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
+    prm.flat = (rank == 4) ? 1 : 0;
     prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0; prm.hdiv = p.hdiv;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
