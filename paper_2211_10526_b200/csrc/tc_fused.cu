@@ -1,4 +1,5 @@
-// Whole forward pass in one kernel for short sequences (bf16, d = 64, N <= 256 tokens per (b,h)):
+// Whole forward pass in one kernel for short sequences (bf16, N <= 256 tokens per (b,h), head width 64 or
+// two width-32 heads side by side in a 64-wide row):
 //     out_t = (1/pi) q^_t (K^^T V) + 1/2 sum_n v_n + bias + DWConv(V)_t                    (Eq. 9)
 // A plane (one (b,h)) fits in shared memory, so K, V and Q come from memory once, the state never
 // leaves the SM and the forward is a single launch without workspace.  Two CTAs share an SM; each
@@ -16,7 +17,8 @@
 //               V tile and the Q tile, both dead by then); then lane = channel pair, warp = a run of
 //               eight tokens of one grid row: depthwise convolution with the filters in registers and a
 //               sliding window along x, out = acc / max(||q||, eps) + 1/2 s + bias + conv, one rounding
-//               to bf16, 128-byte rows stored straight to memory
+//               to bf16, 128-byte rows stored straight to memory; leading off-grid tokens get the
+//               attention terms only
 #include "tc_common.cuh"
 #include "tc_host.cuh"
 

@@ -25,13 +25,13 @@ constexpr int kTmemCols = 128;                // two 64-column accumulators: a C
 constexpr int kGroup = 4;                    // splits per first-level reduction group
 constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
-// PAIR = true also serves two width-32 heads stored side by side in one 128-byte row (same arithmetic,
-// the consumer keeps the two diagonal blocks apart instead of adding them).
 // PAIR = true serves head width 32: the [N][32] tensors are viewed as [N/2][64], one 128-byte row
 // holding two consecutive tokens.  The same contraction then yields the four 32 x 32 blocks
 // [k_even^T v_even, k_even^T v_odd; k_odd^T v_even, k_odd^T v_odd]; the state is the sum of the two
 // diagonal blocks (and s the sum of the two halves of row 64), which the apply kernel folds when it
 // reads them.  Each half row is normalised by its own token's norm.
+// The same instantiation serves two width-32 heads stored side by side in one 128-byte row (head
+// stride 32): identical arithmetic; there the consumers keep the two diagonal blocks apart, one per head.
 template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 2)
 tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
