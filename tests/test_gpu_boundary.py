@@ -196,6 +196,25 @@ def test_host_entry_point_pipelines_batch_chunks():
         assert err <= 2e-2
 
 
+@pytest.mark.parametrize("shape", [(2, 4, 1, 14, 14, 32, 3, "f32"), (4, 8, 2, 128, 64, 64, 3, "bf16"), (3, 5, 1, 14, 14, 64, 3, "bf16")],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_host_entry_point_with_leading_tokens(shape):
+    """Host-buffer entry point (one piece and pipelined chunks) for sequences that start with off-grid tokens."""
+    from paper_2211_10526_b200 import CastlingAttn
+    B, H, P, gh, gw, d, ks, dtype = shape
+    c = workloads.custom_call(B, H, 1, P + gh * gw, d, ks, dtype, seed=450 + sum(shape[:7]))
+    pinned = [t.pin_memory() for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)]
+    out_h = torch.full_like(c.q, float("nan")).pin_memory()
+    with CastlingAttn(ksize=ks, prefix_tokens=P) as attn:
+        attn.forward_host(*pinned, gh, gw, out=out_h)
+        assert attn.device_status() == (0, 0)
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, gh, gw, ks, threads=8, prefix=P)
+    g = out_h.double().numpy()
+    assert np.all(np.isfinite(g))
+    err = np.max(np.abs(g - ref)) / np.max(np.abs(ref))
+    assert err <= (1e-5 if dtype == "f32" else 2e-2)
+
+
 GRAPH_SHAPES = [  # B, H, prefix, gridH, gridW, d, ksize, dtype: one per kernel family
     (2, 4, 0, 14, 14, 32, 3, "f32"),     # CUDA-core state + apply
     (1, 2, 0, 48, 50, 32, 3, "f32"),     # CUDA-core with the token range split (reduce kernel)
