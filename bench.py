@@ -41,7 +41,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # one ncu capture of this command at full size (profiles/tc_kernels_c5_sweep.md); None for workloads
 # or kernels without a capture of the current code.
-NCU_TRAFFIC_BYTES = {("c5_sweep_bf16:3", "tc_apply"): 252.5e6 + 99.3e6}
+NCU_TRAFFIC_BYTES = {("c5_sweep_bf16:3", "tc_apply"): 252.5e6 + 98.8e6,
+                     ("c3_deit_base_bf16", "tc_fused"): 57.9e6 + 1.8e6}
 
 
 def parse_args():
