@@ -13,9 +13,6 @@ namespace {
 // Width-32 heads fill a 128-byte row in one of two ways: two adjacent tokens of one head (tokens
 // contiguous, even grid width), or the same token of two adjacent heads (head stride 32, as in a
 // token-major [B,N,H,32] tensor with an even number of heads).
-bool token_pairs(const Problem& p) {
-    return p.d == 32 && p.gridW % 2 == 0 && p.N % 2 == 0 && p.contiguous_tokens();
-}
 bool head_pairs(const Problem& p) {
     return p.d == 32 && p.H % 2 == 0 && p.hdiv == p.H && p.head0 == 0 && p.lq.head == 32 && p.lk.head == 32 &&
            p.lv.head == 32 && p.lo.head == 32;

@@ -1,5 +1,5 @@
-// Whole forward pass in one kernel for short sequences (bf16, N <= 256 tokens per (b,h), head width 64 or
-// two width-32 heads side by side in a 64-wide row):
+// Whole forward pass in one kernel for short sequences (bf16, at most 256 128-byte rows per (b,h): head
+// width 64, two width-32 heads side by side, or width-32 heads with two adjacent tokens per row):
 //     out_t = (1/pi) q^_t (K^^T V) + 1/2 sum_n v_n + bias + DWConv(V)_t                    (Eq. 9)
 // A plane (one (b,h)) fits in shared memory, so K, V and Q come from memory once, the state never
 // leaves the SM and the forward is a single launch without workspace.  Two CTAs share an SM; each
@@ -61,7 +61,10 @@ struct FusedParams {
 
 // OUT_PACKED: the output's token rows are contiguous (stride 64), which keeps the row addresses of the
 // store loop compile-time offsets.
-template <int KS, bool OUT_PACKED>
+// TOKPAIR: width-32 heads with two adjacent tokens per 128-byte row (rows = N / 2): each half of a row has
+// its own norm, the state is the sum of the two diagonal 32 x 32 blocks of the accumulator, used for both
+// halves, and a lane of the convolution phase stands for (token parity, channel pair).
+template <int KS, bool OUT_PACKED, bool TOKPAIR>
 __global__ void __launch_bounds__(kThreads, (KS == 3) ? 2 : 1)
 tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmVplain,
@@ -91,7 +94,9 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int N = prm.N, W = prm.gridW;
+    const int W = prm.gridW;
+    const int N = TOKPAIR ? prm.N / 2 : prm.N;  // 128-byte rows per plane
+    const bool halves = TOKPAIR || prm.blockdiag;  // each half of a row is normalised on its own
     const int tiles = (N + kTile - 1) / kTile;  // 1 or 2
     const int n_planes = (prm.BH - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     constexpr unsigned kBit = kStatusFusedTimeout;
@@ -191,7 +196,8 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 are this warp's
         const int half = ww >> 2;                   // thread = token phases: channels half*32 .. half*32 + 31
         const int r = quarter * 32 + lane;          // thread = token phases: row of both tiles
-        const int segs = (W + kSeg - 1) / kSeg, n_units = prm.gridH * segs;
+        const int Wc = TOKPAIR ? W / 2 : W;        // 128-byte columns per grid row
+        const int segs = (Wc + kSeg - 1) / kSeg, n_units = prm.gridH * segs;
         const float2 zero2 = make_float2(0.f, 0.f);
         for (int it = 0; it < n_planes; ++it) {
             const uint32_t ph = it & 1;
@@ -201,11 +207,12 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             // convolution, so that the round trip to L2 hides behind everything in between
             unsigned short wraw[2][KS * KS], braw[2] = {0, 0};
             {
-                const unsigned short* w0 = reinterpret_cast<const unsigned short*>(prm.w) + (size_t)(h * kD + 2 * lane) * (KS * KS);
+                const int ch0 = TOKPAIR ? h * 32 + 2 * (lane & 15) : h * kD + 2 * lane;  // first channel of the lane's pair
+                const unsigned short* w0 = reinterpret_cast<const unsigned short*>(prm.w) + (size_t)ch0 * (KS * KS);
 #pragma unroll
                 for (int i = 0; i < KS * KS; ++i) { wraw[0][i] = __ldg(w0 + i); wraw[1][i] = __ldg(w0 + KS * KS + i); }
                 if (prm.bias) {
-                    const unsigned short* b0 = reinterpret_cast<const unsigned short*>(prm.bias) + h * kD + 2 * lane;
+                    const unsigned short* b0 = reinterpret_cast<const unsigned short*>(prm.bias) + ch0;
                     braw[0] = __ldg(b0); braw[1] = __ldg(b0 + 1);
                 }
             }
@@ -226,8 +233,8 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                 }
                 const float sa = (ss[0].x + ss[0].y) + (ss[1].x + ss[1].y), sb = (ss[2].x + ss[2].y) + (ss[3].x + ss[3].y);
-                const float rka = 1.0f / sqrtf(fmaxf(prm.blockdiag ? sa : sa + sb, prm.eps2));
-                const float rkb = prm.blockdiag ? 1.0f / sqrtf(fmaxf(sb, prm.eps2)) : rka;
+                const float rka = 1.0f / sqrtf(fmaxf(halves ? sa : sa + sb, prm.eps2));
+                const float rkb = halves ? 1.0f / sqrtf(fmaxf(sb, prm.eps2)) : rka;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const uint32_t w4[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
@@ -260,7 +267,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                 }
                 const float sa = (ss[0].x + ss[0].y) + (ss[1].x + ss[1].y), sb = (ss[2].x + ss[2].y) + (ss[3].x + ss[3].y);
-                rq_s[wt] = rsqrtf(fmaxf(prm.blockdiag ? sa : sa + sb, prm.eps2));
+                rq_s[wt] = rsqrtf(fmaxf(halves ? sa : sa + sb, prm.eps2));
                 rq_s[kRqStride + wt] = rsqrtf(fmaxf(sb, prm.eps2));  // read only when the halves are separate heads
             }
 
@@ -277,7 +284,16 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                     for (int e = 0; e < 16; ++e) { a[e] = a0[e]; a[16 + e] = a1[e]; }
                 }
-                if (quarter < 2) {  // row r of S (key feature r), 32 value features
+                if constexpr (TOKPAIR) {
+                    // the two diagonal blocks meet in shared memory (the swizzled V tile is dead by now):
+                    // [2][32 rows][32] fp32, 16-byte chunk c of row i at chunk c ^ (i & 7)
+                    float* scr = reinterpret_cast<float*>(V_s) + quarter * 1024 + lane * 32;
+                    if (quarter < 2 && quarter == half) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            *reinterpret_cast<float4*>(scr + ((e ^ (lane & 7)) << 2)) = make_float4(a[4 * e], a[4 * e + 1], a[4 * e + 2], a[4 * e + 3]);
+                    }
+                } else if (quarter < 2) {  // row r of S (key feature r), 32 value features
                     const float sp = (prm.blockdiag && quarter != half) ? 0.f : kInvPi;  // other head's block: zero
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -288,10 +304,32 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         o.w = pack_bf16x2(a[8 * e + 6] * sp, a[8 * e + 7] * sp);
                         *reinterpret_cast<uint4*>(S_s + r * 128 + (((half * 4 + e) ^ (r & 7)) << 4)) = o;
                     }
-                } else if (lane == 0) {  // accumulator row 64: the token sum of V
+                }
+                if (quarter == 2 && lane == 0) {  // accumulator row 64: the token sum of V
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
                         *reinterpret_cast<float4*>(sum_s + half * 32 + 4 * e) = make_float4(a[4 * e], a[4 * e + 1], a[4 * e + 2], a[4 * e + 3]);
+                }
+            }
+            if constexpr (TOKPAIR) {
+                named_barrier_sync(2, kWorkers);  // both diagonal blocks are in shared memory
+                if (quarter < 2) {  // operand = blockdiag(S32, S32) / pi with S32 = block(0,0) + block(1,1)
+                    const float* s0 = reinterpret_cast<const float*>(V_s) + lane * 32;
+                    const float* s1 = s0 + 1024;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        uint4 o = make_uint4(0, 0, 0, 0);
+                        if (quarter == half) {
+                            const int c0 = ((2 * e) ^ (lane & 7)) << 2, c1 = ((2 * e + 1) ^ (lane & 7)) << 2;
+                            const float4 x0 = *reinterpret_cast<const float4*>(s0 + c0), y0 = *reinterpret_cast<const float4*>(s1 + c0);
+                            const float4 x1 = *reinterpret_cast<const float4*>(s0 + c1), y1 = *reinterpret_cast<const float4*>(s1 + c1);
+                            o.x = pack_bf16x2((x0.x + y0.x) * kInvPi, (x0.y + y0.y) * kInvPi);
+                            o.y = pack_bf16x2((x0.z + y0.z) * kInvPi, (x0.w + y0.w) * kInvPi);
+                            o.z = pack_bf16x2((x1.x + y1.x) * kInvPi, (x1.y + y1.y) * kInvPi);
+                            o.w = pack_bf16x2((x1.z + y1.z) * kInvPi, (x1.w + y1.w) * kInvPi);
+                        }
+                        *reinterpret_cast<uint4*>(S_s + r * 128 + (((half * 4 + e) ^ (r & 7)) << 4)) = o;
+                    }
                 }
             }
             fence_proxy_async_smem();
@@ -335,66 +373,123 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 for (int dx = 0; dx < KS; ++dx)
                     wreg[dy][dx] = make_float2(__uint_as_float((uint32_t)wraw[0][dy * KS + dx] << 16),
                                                __uint_as_float((uint32_t)wraw[1][dy * KS + dx] << 16));
-            const float2 hs2 = make_float2(0.5f * sum_s[2 * lane], 0.5f * sum_s[2 * lane + 1]);  // 1/2 s
-            const float2 c2 = make_float2(hs2.x + __uint_as_float((uint32_t)braw[0] << 16),
-                                          hs2.y + __uint_as_float((uint32_t)braw[1] << 16));  // + bias: grid tokens
-            uint32_t* out_plane = reinterpret_cast<uint32_t*>(prm.out + plane_offset(prm.lo, bh, prm.hdiv)) + lane;
-            const long long out_tok = OUT_PACKED ? kD / 2 : prm.lo.token / 2;  // 32-bit words per token step
-            const int sc = lane >> 1, sw = (lane & 1) * 8;  // chunk and offset of the lane's pair in an fp32 row
-            const float* rq_l = rq_s + ((prm.blockdiag && lane >= 16) ? kRqStride : 0);  // the norm of the lane's head
-            // Branch-free inside a unit: a neighbour outside the grid is read from a row of zeros, the
-            // columns of a ragged last unit are computed (from in-bounds shared memory) and not stored.
-            const uint32_t k_base = smem_u32(K_s) + lane * 4, z_addr = smem_u32(smem + kOffZero) + lane * 4;
-            for (int u = ww; u < n_units; u += kWorkers / 32) {
-                const int y = u / segs, x0 = (u - y * segs) * kSeg, nx = min(kSeg, W - x0);
-                uint32_t ra[KS];  // address of the lane's word of token (y + dy - R, x0); rows outside the grid: the zero row
-                uint32_t rstep[KS];  // bytes per column in that row (0 for the zero row)
-#pragma unroll
-                for (int dy = 0; dy < KS; ++dy) {
-                    const int yy = y + dy - R;
-                    const bool rv = (unsigned)yy < (unsigned)prm.gridH;
-                    ra[dy] = rv ? k_base + (uint32_t)((prm.prefix + yy * W + x0) * 128) : z_addr;
-                    rstep[dy] = rv ? 128u : 0u;
-                }
-                float2 win[KS][KS];  // column x0 - R + jj lives in slot jj % KS
-#pragma unroll
-                for (int jj = 0; jj < KS - 1 + kSeg; ++jj) {
-                    // load column jj of the window (grid column x0 - R + jj), then finish output column jj - (KS - 1)
-                    const bool cv = (unsigned)(x0 + jj - R) < (unsigned)W;
+            if constexpr (TOKPAIR) {
+                // lane = (token parity, channel pair): a 128-byte row of the plain V plane, of the accumulator rows
+                // and of the output holds tokens (2c, 2c+1) of a grid row; tokens are 64 bytes apart
+                const int tp = lane >> 4, cp = lane & 15;
+                const float2 hs2 = make_float2(0.5f * (sum_s[2 * cp] + sum_s[32 + 2 * cp]),
+                                               0.5f * (sum_s[2 * cp + 1] + sum_s[32 + 2 * cp + 1]));  // 1/2 s
+                const float2 c2 = make_float2(hs2.x + __uint_as_float((uint32_t)braw[0] << 16),
+                                              hs2.y + __uint_as_float((uint32_t)braw[1] << 16));
+                uint32_t* out_plane = reinterpret_cast<uint32_t*>(prm.out + plane_offset(prm.lo, bh, prm.hdiv)) + lane;
+                const int sc = lane >> 1, sw = (lane & 1) * 8;
+                const float* rq_l = rq_s + tp * kRqStride;  // the norm of the lane's token
+                const uint32_t k_base = smem_u32(K_s) + cp * 4, z_addr = smem_u32(smem + kOffZero) + cp * 4;
+                for (int u = ww; u < n_units; u += kWorkers / 32) {
+                    const int y = u / segs, c0 = (u - y * segs) * kSeg, nc = min(kSeg, Wc - c0);
+                    uint32_t ra[KS], rstep[KS];  // address of token (y + dy - R, 0) (or the zero row) and bytes per token
 #pragma unroll
                     for (int dy = 0; dy < KS; ++dy) {
-                        const uint32_t a = cv ? ra[dy] + (uint32_t)(jj - R) * rstep[dy] : z_addr;
-                        uint32_t wv;
-                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(a));
-                        win[dy][jj % KS] = make_float2(bf16lo(wv), bf16hi(wv));
+                        const int yy = y + dy - R;
+                        const bool rv = (unsigned)yy < (unsigned)prm.gridH;
+                        ra[dy] = rv ? k_base + (uint32_t)((prm.prefix + yy * W) * 64) : z_addr;
+                        rstep[dy] = rv ? 64u : 0u;
                     }
-                    if (jj >= KS - 1) {  // compile-time
-                        const int j = jj - (KS - 1);
-                        float2 part[KS];  // one chain per filter row
+#pragma unroll
+                    for (int j = 0; j < kSeg; ++j) {
+                        const int x = 2 * (c0 + j) + tp;  // the lane's token in the grid row
+                        float2 part[KS];
 #pragma unroll
                         for (int dy = 0; dy < KS; ++dy) {
                             part[dy] = (dy == 0) ? c2 : zero2;
 #pragma unroll
-                            for (int dx = 0; dx < KS; ++dx) part[dy] = ffma2(wreg[dy][dx], win[dy][(j + dx) % KS], part[dy]);
+                            for (int dx = 0; dx < KS; ++dx) {
+                                const int xt = x + dx - R;
+                                const uint32_t a = ((unsigned)xt < (unsigned)W) ? ra[dy] + (uint32_t)xt * rstep[dy] : z_addr;
+                                uint32_t wv;
+                                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(a));
+                                part[dy] = ffma2(wreg[dy][dx], make_float2(bf16lo(wv), bf16hi(wv)), part[dy]);
+                            }
                         }
                         float2 acc = part[0];
 #pragma unroll
                         for (int dy = 1; dy < KS; ++dy) { acc.x += part[dy].x; acc.y += part[dy].y; }
-                        const int t = prm.prefix + y * W + x0 + j, tr = t & (kTile - 1);  // t < N + kSeg: inside a row of rq_s
-                        const uint8_t* srow = (t < kTile ? V_s : Q_s) + tr * 256;
+                        const int pr = (prm.prefix + y * W) / 2 + c0 + j, tr = pr & (kTile - 1);  // row of the token pair
+                        const uint8_t* srow = (pr < kTile ? V_s : Q_s) + tr * 256;
                         const float2 a2 = *reinterpret_cast<const float2*>(srow + ((sc ^ (tr & 7)) << 4) + sw);
-                        const float rq = rq_l[t];
+                        const float rq = rq_l[pr];
                         const float2 o = ffma2(a2, make_float2(rq, rq), acc);
-                        if (j < nx) out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
+                        if (j < nc) out_plane[pr * (kD / 2)] = pack_bf16x2(o.x, o.y);
                     }
                 }
-            }
-            // off-grid leading tokens: the attention terms only
-            for (int t = ww; t < prm.prefix; t += kWorkers / 32) {
-                const float2 a2 = *reinterpret_cast<const float2*>(V_s + t * 256 + ((sc ^ (t & 7)) << 4) + sw);
-                const float rq = rq_l[t];
-                const float2 o = ffma2(a2, make_float2(rq, rq), hs2);
-                out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
+                for (int pr = ww; pr < prm.prefix / 2; pr += kWorkers / 32) {  // off-grid leading tokens
+                    const float2 a2 = *reinterpret_cast<const float2*>(V_s + pr * 256 + ((sc ^ (pr & 7)) << 4) + sw);
+                    const float rq = rq_l[pr];
+                    const float2 o = ffma2(a2, make_float2(rq, rq), hs2);
+                    out_plane[pr * (kD / 2)] = pack_bf16x2(o.x, o.y);
+                }
+            } else {
+                const float2 hs2 = make_float2(0.5f * sum_s[2 * lane], 0.5f * sum_s[2 * lane + 1]);  // 1/2 s
+                const float2 c2 = make_float2(hs2.x + __uint_as_float((uint32_t)braw[0] << 16),
+                                              hs2.y + __uint_as_float((uint32_t)braw[1] << 16));  // + bias: grid tokens
+                uint32_t* out_plane = reinterpret_cast<uint32_t*>(prm.out + plane_offset(prm.lo, bh, prm.hdiv)) + lane;
+                const long long out_tok = OUT_PACKED ? kD / 2 : prm.lo.token / 2;  // 32-bit words per token step
+                const int sc = lane >> 1, sw = (lane & 1) * 8;  // chunk and offset of the lane's pair in an fp32 row
+                const float* rq_l = rq_s + ((prm.blockdiag && lane >= 16) ? kRqStride : 0);  // the norm of the lane's head
+                // Branch-free inside a unit: a neighbour outside the grid is read from a row of zeros, the
+                // columns of a ragged last unit are computed (from in-bounds shared memory) and not stored.
+                const uint32_t k_base = smem_u32(K_s) + lane * 4, z_addr = smem_u32(smem + kOffZero) + lane * 4;
+                for (int u = ww; u < n_units; u += kWorkers / 32) {
+                    const int y = u / segs, x0 = (u - y * segs) * kSeg, nx = min(kSeg, W - x0);
+                    uint32_t ra[KS];  // address of the lane's word of token (y + dy - R, x0); rows outside the grid: the zero row
+                    uint32_t rstep[KS];  // bytes per column in that row (0 for the zero row)
+    #pragma unroll
+                    for (int dy = 0; dy < KS; ++dy) {
+                        const int yy = y + dy - R;
+                        const bool rv = (unsigned)yy < (unsigned)prm.gridH;
+                        ra[dy] = rv ? k_base + (uint32_t)((prm.prefix + yy * W + x0) * 128) : z_addr;
+                        rstep[dy] = rv ? 128u : 0u;
+                    }
+                    float2 win[KS][KS];  // column x0 - R + jj lives in slot jj % KS
+    #pragma unroll
+                    for (int jj = 0; jj < KS - 1 + kSeg; ++jj) {
+                        // load column jj of the window (grid column x0 - R + jj), then finish output column jj - (KS - 1)
+                        const bool cv = (unsigned)(x0 + jj - R) < (unsigned)W;
+    #pragma unroll
+                        for (int dy = 0; dy < KS; ++dy) {
+                            const uint32_t a = cv ? ra[dy] + (uint32_t)(jj - R) * rstep[dy] : z_addr;
+                            uint32_t wv;
+                            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(a));
+                            win[dy][jj % KS] = make_float2(bf16lo(wv), bf16hi(wv));
+                        }
+                        if (jj >= KS - 1) {  // compile-time
+                            const int j = jj - (KS - 1);
+                            float2 part[KS];  // one chain per filter row
+    #pragma unroll
+                            for (int dy = 0; dy < KS; ++dy) {
+                                part[dy] = (dy == 0) ? c2 : zero2;
+    #pragma unroll
+                                for (int dx = 0; dx < KS; ++dx) part[dy] = ffma2(wreg[dy][dx], win[dy][(j + dx) % KS], part[dy]);
+                            }
+                            float2 acc = part[0];
+    #pragma unroll
+                            for (int dy = 1; dy < KS; ++dy) { acc.x += part[dy].x; acc.y += part[dy].y; }
+                            const int t = prm.prefix + y * W + x0 + j, tr = t & (kTile - 1);  // t < N + kSeg: inside a row of rq_s
+                            const uint8_t* srow = (t < kTile ? V_s : Q_s) + tr * 256;
+                            const float2 a2 = *reinterpret_cast<const float2*>(srow + ((sc ^ (tr & 7)) << 4) + sw);
+                            const float rq = rq_l[t];
+                            const float2 o = ffma2(a2, make_float2(rq, rq), acc);
+                            if (j < nx) out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
+                        }
+                    }
+                }
+                // off-grid leading tokens: the attention terms only
+                for (int t = ww; t < prm.prefix; t += kWorkers / 32) {
+                    const float2 a2 = *reinterpret_cast<const float2*>(V_s + t * 256 + ((sc ^ (t & 7)) << 4) + sw);
+                    const float rq = rq_l[t];
+                    const float2 o = ffma2(a2, make_float2(rq, rq), hs2);
+                    out_plane[t * out_tok] = pack_bf16x2(o.x, o.y);
+                }
             }
             fence_proxy_async_smem();
             mbar_arrive(plane_free);
@@ -410,10 +505,11 @@ cudaError_t launch_fused_ks(const Problem& p, unsigned* status, cudaStream_t st)
     CUtensorMap tmK, tmV, tmQ, tmVplain;
     // [64, tokens, planes per batch step, batch steps]
     const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
-    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)p.N, (uint64_t)p.hdiv, nb};
+    const bool pair = (p.d == 32);  // two tokens per 128-byte row
+    const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)(pair ? p.N / 2 : p.N), (uint64_t)p.hdiv, nb};
     const uint32_t box[4] = {kD, kTile, 1, 1};
     auto strides = [&](const Layout& l, uint64_t (&s)[3]) {
-        s[0] = (uint64_t)l.token; s[1] = (uint64_t)l.head; s[2] = (uint64_t)(nb > 1 ? l.batch : l.head * p.hdiv);
+        s[0] = (uint64_t)(pair ? kD : l.token); s[1] = (uint64_t)l.head; s[2] = (uint64_t)(nb > 1 ? l.batch : l.head * p.hdiv);
     };
     uint64_t sq[3], sk[3], sv[3];
     strides(p.lq, sq); strides(p.lk, sk); strides(p.lv, sv);
@@ -429,23 +525,28 @@ cudaError_t launch_fused_ks(const Problem& p, unsigned* status, cudaStream_t st)
     prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv; prm.prefix = p.prefix; prm.N = p.N;
     prm.gridH = p.gridH; prm.gridW = p.gridW;
     prm.eps2 = p.eps2; prm.status = status;
-    static PerDevice opt_in[2];  // per instantiation
+    static PerDevice opt_in[3];  // per instantiation
     const bool packed = (p.lo.token == kD);
-    const cudaError_t e = packed ? opt_in_smem(tc_fused_kernel<KS, true>, kSmemBytes, opt_in[1])
-                                 : opt_in_smem(tc_fused_kernel<KS, false>, kSmemBytes, opt_in[0]);
+    const cudaError_t e = pair     ? opt_in_smem(tc_fused_kernel<KS, true, true>, kSmemBytes, opt_in[2])
+                          : packed ? opt_in_smem(tc_fused_kernel<KS, true, false>, kSmemBytes, opt_in[1])
+                                   : opt_in_smem(tc_fused_kernel<KS, false, false>, kSmemBytes, opt_in[0]);
     if (e != cudaSuccess) return e;
     const int grid = p.BH < 2 * 148 ? p.BH : 2 * 148;  // two CTAs per SM
-    if (packed)
-        tc_fused_kernel<KS, true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
+    if (pair)
+        tc_fused_kernel<KS, true, true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
+    else if (packed)
+        tc_fused_kernel<KS, true, false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
     else
-        tc_fused_kernel<KS, false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
+        tc_fused_kernel<KS, false, false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 bool fused_supports(const Problem& p) {
-    return p.bf16 && p.d == kD && (p.ksize == 3 || p.ksize == 5) && p.N <= kMaxTiles * kTile;
+    if (!p.bf16 || (p.ksize != 3 && p.ksize != 5)) return false;
+    if (p.d == kD) return p.N <= kMaxTiles * kTile;
+    return token_pairs(p) && p.prefix % 2 == 0 && p.N / 2 <= kMaxTiles * kTile;  // width 32: rows of two tokens
 }
 
 cudaError_t launch_fused(const Problem& p, unsigned* status, cudaStream_t st) {

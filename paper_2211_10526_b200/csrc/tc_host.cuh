@@ -13,6 +13,12 @@ constexpr int kCountersPerHead = 17;
 bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
                           const uint64_t* strides, const uint32_t* box, bool swizzle128);
 
+// Width-32 heads, two adjacent tokens of one head per 128-byte row: contiguous tokens, even grid width,
+// an even number of tokens per plane.
+inline bool token_pairs(const Problem& p) {
+    return p.d == 32 && p.gridW % 2 == 0 && p.N % 2 == 0 && p.contiguous_tokens();
+}
+
 // True when the tensor-core kernels can take this problem (bf16; d = 64, or d = 32 with even gridW;
 // 3x3 or 5x5 filters).
 bool supports(const Problem& p);

@@ -250,7 +250,8 @@ PREFIX_CASES = [
     (2, 3, 2, 15, 16, 64, 5, "bf16", "head_major", 2, 1),    # 242 tokens, 5 x 5
     (2, 2, 1, 24, 20, 64, 3, "bf16", "head_major", 2, 3),    # state + apply + leading rows
     (1, 2, 3, 37, 53, 64, 5, "bf16", "head_major", 2, 3),
-    (2, 2, 2, 24, 20, 32, 3, "bf16", "head_major", 2, 3),    # width 32, even N: token pairs
+    (2, 2, 2, 24, 20, 32, 3, "bf16", "head_major", 2, 1),    # width 32, even N: token pairs, single kernel (241 rows)
+    (2, 2, 2, 40, 30, 32, 5, "bf16", "head_major", 2, 3),    # ... state + apply + leading rows
     (2, 2, 1, 24, 20, 32, 3, "bf16", "head_major", 1, 3),    # width 32, odd N: CUDA cores (P = 2 splits)
     (2, 4, 1, 24, 20, 32, 5, "bf16", "token_major", 2, 3),   # width 32 token-major: head pairs
     (2, 4, 1, 12, 12, 32, 3, "bf16", "token_major", 2, 1),   # ... in the single-kernel forward
@@ -550,7 +551,10 @@ def test_tensor_path_term_isolation():
 # B, H, gridH, gridW, d, ksize
 ONE_KERNEL_SHAPES = [(1, 1, 1, 1, 64, 3), (2, 3, 14, 14, 64, 3), (1, 2, 16, 16, 64, 3), (3, 2, 1, 129, 64, 3),
                      (2, 2, 3, 70, 64, 5), (1, 1, 128, 1, 64, 3), (1, 3, 9, 14, 64, 5), (5, 70, 8, 8, 64, 3),
-                     (1, 1, 2, 128, 64, 5), (2, 1, 127, 1, 64, 5), (37, 9, 5, 7, 64, 3)]
+                     (1, 1, 2, 128, 64, 5), (2, 1, 127, 1, 64, 5), (37, 9, 5, 7, 64, 3),
+                     # width-32 heads, two tokens per row (even grid width, at most 512 tokens)
+                     (2, 4, 14, 14, 32, 3), (1, 2, 16, 32, 32, 3), (3, 2, 1, 130, 32, 3), (2, 2, 3, 70, 32, 5),
+                     (1, 1, 1, 2, 32, 3), (5, 70, 8, 8, 32, 3), (2, 3, 9, 22, 32, 5), (1, 2, 128, 4, 32, 3)]
 
 
 @pytest.mark.parametrize("shape", ONE_KERNEL_SHAPES, ids=lambda s: "x".join(map(str, s)))
