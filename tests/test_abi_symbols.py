@@ -83,3 +83,28 @@ def test_workloads_match_the_configured_shapes():
     import torch
     assert torch.equal(a.q, b.q) and torch.equal(a.dw_weight, b.dw_weight)
     assert a.q.dtype == torch.bfloat16 and tuple(a.q.shape) == (64, 8, 49, 32)
+
+
+def test_binding_structs_match_the_header_layout(tmp_path):
+    """The ctypes mirrors of the two structs in the header have the C compiler's sizes and field offsets."""
+    import subprocess
+    from paper_2211_10526_b200 import binding as b
+    src = tmp_path / "layout.c"
+    src.write_text(
+        '#include <stdio.h>\n#include <stddef.h>\n#include "castling_attn.h"\n'
+        'int main(void) {\n'
+        '  printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(castling_attn_config_t), offsetof(castling_attn_config_t, ksize),\n'
+        '         offsetof(castling_attn_config_t, eps), offsetof(castling_attn_config_t, force_path),\n'
+        '         offsetof(castling_attn_config_t, max_workspace), offsetof(castling_attn_config_t, prefix_tokens));\n'
+        '  printf("%zu %zu %zu %zu\\n", sizeof(castling_attn_layout_t), offsetof(castling_attn_layout_t, q_batch),\n'
+        '         offsetof(castling_attn_layout_t, v_head), offsetof(castling_attn_layout_t, out_token));\n'
+        '  printf("%d %d %d %u\\n", CASTLING_ERR_SCRATCH_LIMIT, CASTLING_PATH_TENSOR, CASTLING_BF16, CASTLING_STATIC_SCRATCH_BYTES);\n'
+        '  return 0;\n}\n')
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c11", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
+    lines = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    cfg, lay = b.castling_attn_config_t, b.castling_attn_layout_t
+    assert [int(x) for x in lines[0].split()] == [ctypes.sizeof(cfg), cfg.ksize.offset, cfg.eps.offset, cfg.force_path.offset,
+                                                 cfg.max_workspace.offset, cfg.prefix_tokens.offset]
+    assert [int(x) for x in lines[1].split()] == [ctypes.sizeof(lay), lay.q_batch.offset, lay.v_head.offset, lay.out_token.offset]
+    assert [int(x) for x in lines[2].split()] == [b.ERR_SCRATCH_LIMIT, b.PATH_TENSOR, b.CASTLING_BF16, b.STATIC_SCRATCH_BYTES]
