@@ -65,7 +65,8 @@ enum {
 enum {
     CASTLING_PATH_AUTO = 0,
     CASTLING_PATH_SIMT = 1,   /* CUDA-core FMA kernels: every dtype, d and ksize supported   */
-    CASTLING_PATH_TENSOR = 2  /* tcgen05/TMEM + TMA kernels: bf16, d = 64                    */
+    CASTLING_PATH_TENSOR = 2  /* tcgen05/TMEM + TMA kernels: bf16, ksize 3 or 5, d = 64, or   */
+                              /* d = 32 packed two tokens or two heads to a 128-byte row      */
 };
 
 typedef struct {
@@ -147,9 +148,11 @@ typedef struct {
  *               share memory (not checked).
  *   everything else as for castling_attn_forward.
  *
- * The tensor-core kernels read such layouts directly through strided TMA descriptors (width-64
- * heads; width-32 heads need contiguous tokens, because two tokens share one 128-byte row there);
- * everything else, and any layout a descriptor cannot express, runs on the CUDA-core kernels.
+ * The tensor-core kernels read such layouts directly through strided TMA descriptors: width-64
+ * heads with any strides; width-32 heads when a 128-byte row holds either two adjacent tokens of one
+ * head (contiguous tokens, even gridW and N) or the same token of two adjacent heads (head stride 32,
+ * even H, as in token-major [B,N,H,32]).  Everything else, and any layout a descriptor cannot express,
+ * runs on the CUDA-core kernels.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, OOM, CUDA.
  */
 CASTLING_API int castling_attn_forward_strided(castling_attn_t* handle,

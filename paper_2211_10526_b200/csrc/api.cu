@@ -11,7 +11,6 @@ using castling::Problem;
 struct castling_attn {
     castling_attn_config_t cfg;
     int device = 0;
-    int sm_count = 0;
     float* ws = nullptr;        // header | state | partial
     size_t ws_bytes = 0;
     unsigned* counters = nullptr;  // arrival counters of the split reduction, zero between calls
@@ -27,6 +26,22 @@ struct castling_attn {
     int last_launches = 0;
     castling::KernelTimer timer;
 };
+
+namespace castling {
+int device_sm_count() {
+    static std::atomic<int> cached[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return 148; }
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    cached[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
+}  // namespace castling
 
 namespace {
 
@@ -132,7 +147,6 @@ int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** ou
     if (!h) return CASTLING_ERR_OOM;
     h->cfg = c;
     h->device = dev;
-    h->sm_count = prop.multiProcessorCount;
     *out_handle = h;
     return CASTLING_OK;
 }
@@ -373,6 +387,14 @@ int castling_attn_forward_host(castling_attn_t* h, const void* q, const void* k,
     if ((e = cudaStreamWaitEvent(h->copy_out, h->ev_start, 0)) != cudaSuccess) return fail_cuda(h, e);
     int b0[castling_attn::kMaxChunks + 1];
     for (int c = 0; c <= chunks; ++c) b0[c] = (int)((long long)BH * c / chunks);
+    // workspace and counters for every run length, before anything is in flight: growing them later
+    // would synchronise the device in the middle of the pipeline (and clear the status word)
+    for (int c = 0; c < chunks; ++c) {
+        rc = ensure_workspace(h, b0[c + 1] - b0[c], (int)n_tok, d, dtype == CASTLING_BF16);
+        if (rc != CASTLING_OK) return rc;
+        rc = ensure_counters(h, b0[c + 1] - b0[c]);
+        if (rc != CASTLING_OK) return rc;
+    }
     for (int c = 0; c < chunks; ++c) {
         const size_t off = (size_t)b0[c] * plane_bytes, len = (size_t)(b0[c + 1] - b0[c]) * plane_bytes;
         const char* hq = static_cast<const char*>(q); const char* hk = static_cast<const char*>(k);
@@ -390,6 +412,7 @@ int castling_attn_forward_host(castling_attn_t* h, const void* q, const void* k,
                                  1, H, gridH, gridW, d, dtype);
         p.BH = b0[c + 1] - b0[c];   // a run of planes that may start and end inside a batch
         p.head0 = b0[c] % H;
+        p.set_contiguous();         // one uniform plane stride over the run (planes per step = the run's length)
         rc = run_device(h, p, st);
         if (rc != CASTLING_OK) return rc;
         if ((e = cudaEventRecord(h->ev_done[c], st)) != cudaSuccess) return fail_cuda(h, e);

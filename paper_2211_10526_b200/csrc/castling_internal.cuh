@@ -98,6 +98,10 @@ inline cudaError_t opt_in_smem(Kernel kernel, size_t bytes, PerDevice& flags) {
     return e;
 }
 
+// Multiprocessors of the current device (queried once per device).  Without a usable device the count
+// of a B200 is returned, so that size queries still answer on a host without a GPU.
+int device_sm_count();
+
 // CUDA-core path.  simt_forward returns the cudaError_t of its launches.
 cudaError_t simt_forward(const Problem& p, float* ws_state, float* ws_partial, int P,
                          cudaStream_t stream, int* launches, KernelTimer* timer);

@@ -60,8 +60,10 @@ extern "C" int castling_attn_forward_static(const void* q, const void* k, const 
     const void* ptrs[4] = {q, k, v, out};
     for (const void* p : ptrs)
         if ((uintptr_t)p & 15) return CASTLING_ERR_ALIGNMENT;
+    const size_t w_bytes = (size_t)H * d * ksize * ksize * eb, b_bytes = (size_t)H * d * eb;
     if (overlaps(out, tensor_bytes, q, tensor_bytes) || overlaps(out, tensor_bytes, k, tensor_bytes) ||
-        overlaps(out, tensor_bytes, v, tensor_bytes))
+        overlaps(out, tensor_bytes, v, tensor_bytes) || overlaps(out, tensor_bytes, dw_weight, w_bytes) ||
+        (dw_bias && overlaps(out, tensor_bytes, dw_bias, b_bytes)))
         return CASTLING_ERR_INVALID_ARG;
 
     // scratch: final state [BH][d*d + d], then (only if the token range is split) P partial states

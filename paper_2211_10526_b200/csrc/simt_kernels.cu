@@ -510,11 +510,11 @@ bool simt_supports(int d, int ksize) {
     return d >= 16 && d <= 128 && d % 16 == 0 && ksize >= 1 && ksize <= 7 && (ksize & 1);
 }
 
-// Token splits of the state kernel: enough CTAs to fill a 148-SM device about twice over,
+// Token splits of the state kernel: enough CTAs to fill the device about twice over,
 // at least four staged tiles per split, capped at 64.
 int simt_choose_splits(int BH, int N) {
     const int tiles = (N + kStateTile - 1) / kStateTile;
-    int P = (2 * 148 + BH - 1) / BH;
+    int P = (2 * device_sm_count() + BH - 1) / BH;
     if (P > tiles / 4) P = tiles / 4;
     if (P > 64) P = 64;
     if (P < 1) P = 1;

@@ -417,7 +417,8 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
         const cudaError_t e = opt_in_smem(tc_apply_kernel<KS, MODE>, G::kSmem, opt_in);
         if (e != cudaSuccess) return e;
     }
-    const int grid = prm.n_tiles < 148 ? prm.n_tiles : 148;
+    const int sms = device_sm_count();  // one persistent CTA per multiprocessor
+    const int grid = prm.n_tiles < sms ? prm.n_tiles : sms;
     // programmatic dependent launch: this grid's prologue and first Q / V loads overlap the tail of
     // the state kernel; the warps that read its results wait for it (griddepcontrol.wait) first
     cudaLaunchConfig_t cfg = {};

@@ -36,11 +36,11 @@ bool preferred(const Problem& p) {
 }
 
 // Two state CTAs fit on an SM: as many splits as keep all CTAs of the launch resident at once
-// (2 x 148), every split non-empty, at most 64 splits.
+// (two per multiprocessor), every split non-empty, at most 64 splits.
 int choose_splits(int BH, int N) {
     const int tiles = (N + kStateTile - 1) / kStateTile;
     if (tiles < 1) return 1;
-    int P = (2 * 148) / BH;
+    int P = (2 * device_sm_count()) / BH;
     if (P > tiles) P = tiles;
     if (P > 64) P = 64;
     if (P < 1) P = 1;

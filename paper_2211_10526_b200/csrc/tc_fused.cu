@@ -531,7 +531,8 @@ cudaError_t launch_fused_ks(const Problem& p, unsigned* status, cudaStream_t st)
                           : packed ? opt_in_smem(tc_fused_kernel<KS, true, false>, kSmemBytes, opt_in[1])
                                    : opt_in_smem(tc_fused_kernel<KS, false, false>, kSmemBytes, opt_in[0]);
     if (e != cudaSuccess) return e;
-    const int grid = p.BH < 2 * 148 ? p.BH : 2 * 148;  // two CTAs per SM
+    const int resident = 2 * device_sm_count();  // two CTAs per multiprocessor
+    const int grid = p.BH < resident ? p.BH : resident;
     if (pair)
         tc_fused_kernel<KS, true, true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(tmK, tmV, tmQ, tmVplain, prm);
     else if (packed)

@@ -48,7 +48,8 @@ cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned
 // Output rows of the off-grid leading tokens (p.prefix of them per plane), from the final state.
 cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_t st);
 
-// Single-kernel forward for short sequences (bf16, d = 64, N <= 256, 3x3 or 5x5 filters): no workspace.
+// Single-kernel forward for short sequences (bf16, 3x3 or 5x5 filters, at most 256 128-byte rows per plane:
+// d = 64 with N <= 256, two width-32 heads per row with N <= 256, or width-32 token pairs with N <= 512): no workspace.
 bool fused_supports(const Problem& p);
 cudaError_t launch_fused(const Problem& p, unsigned* status, cudaStream_t st);
 

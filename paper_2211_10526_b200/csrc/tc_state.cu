@@ -327,10 +327,11 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
         if (e != cudaSuccess) return e;
     }
     float* dst = P > 1 ? partial : final_state;
-    // P == 1: a CTA serves several consecutive (b,h); at most 296 CTAs (two per SM) so all are resident
+    // P == 1: a CTA serves several consecutive (b,h); at most two CTAs per multiprocessor so all are resident
     int grid = p.BH * P, items = 1;
-    if (P == 1 && p.BH > 296) {
-        items = (p.BH + 295) / 296;
+    const int resident = 2 * device_sm_count();
+    if (P == 1 && p.BH > resident) {
+        items = (p.BH + resident - 1) / resident;
         grid = (p.BH + items - 1) / items;
     }
     if (halves)

@@ -196,6 +196,36 @@ def test_host_entry_point_pipelines_batch_chunks():
         assert err <= 2e-2
 
 
+# Pipelined chunks whose plane count differs from the head count: more planes than heads (a chunk spans
+# several batches), fewer planes than heads (a chunk starts and ends inside one batch), and a head count
+# that does not divide the chunk.  B, H, gridH, gridW, d, ksize, chunks expected, kernel family expected
+CHUNK_CASES = [(16, 3, 54, 54, 64, 3, 2, 2), (2, 8, 128, 128, 64, 3, 4, 2), (5, 7, 96, 64, 64, 5, 3, 2),
+               (7, 6, 96, 96, 32, 3, 2, 2)]
+
+
+@pytest.mark.parametrize("case", CHUNK_CASES, ids=lambda c: "x".join(map(str, c[:6])))
+def test_host_entry_point_chunks_that_do_not_align_with_heads(case):
+    from paper_2211_10526_b200 import CastlingAttn, binding
+    B, H, gh, gw, d, ks, chunks, family = case
+    c = workloads.custom_call(B, H, gh, gw, d, ks, "bf16", seed=445 + sum(case[:6]))
+    per_tensor = c.q.numel() * 2
+    assert min(8, B * H, per_tensor // (8 << 20)) == chunks, "the case no longer makes the intended chunk count"
+    pinned = [t.pin_memory() for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias)]
+    out_h = torch.full_like(c.q, float("nan")).pin_memory()
+    with CastlingAttn(ksize=ks) as attn:
+        attn.forward_host(*pinned, gh, gw, out=out_h)
+        assert attn.device_status() == (0, 0)
+        assert attn.last_path()[0] == family, "a chunk fell back to the other kernel family"
+    g = out_h.double().numpy()
+    assert np.all(np.isfinite(g)), "part of the output was never written"
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, gh, gw, ks, threads=16)
+    err = np.max(np.abs(g - ref)) / np.max(np.abs(ref))
+    assert err <= 2e-2
+    # per plane as well: a plane computed from another plane's data would still be of the right size
+    per_plane = np.max(np.abs(g - ref), axis=(2, 3)) / np.max(np.abs(ref), axis=(2, 3))
+    assert per_plane.max() <= 2e-2, f"worst plane {np.unravel_index(per_plane.argmax(), per_plane.shape)}"
+
+
 @pytest.mark.parametrize("shape", [(2, 4, 1, 14, 14, 32, 3, "f32"), (4, 8, 2, 128, 64, 64, 3, "bf16"), (3, 5, 1, 14, 14, 64, 3, "bf16")],
                          ids=lambda s: "x".join(map(str, s)))
 def test_host_entry_point_with_leading_tokens(shape):

@@ -5,7 +5,8 @@ while they run (a serving loop that must not hit cudaMalloc's implicit synchroni
 plug-in living inside another program's fixed memory budget): it keeps the state that passes
 between its kernels in an array built into the library.  This file calls it through the C ABI,
 twice in a row per case, and requires the result to agree with `castling_attn_forward` within
-the tolerances the parity tests use.  It is named to be collected last, so a run that stops at
+the tolerances the parity tests use, and with the float64 CPU oracle within the same bound.  It is
+named to be collected last, so a run that stops at
 the first failure has already run every other test.
 """
 from __future__ import annotations
@@ -14,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import workloads
 
 pytestmark = pytest.mark.gpu
@@ -32,6 +34,7 @@ CASES = [
     (2, 3, 9, 11, 64, 3, "bf16"),      # the ordinary entry point runs its tensor-core kernels here
     (1, 2, 48, 50, 32, 5, "f32"),      # token range split: partial states in the scratch too
     (4, 12, 14, 14, 64, 3, "bf16"),
+    (200, 1, 32, 32, 64, 3, "bf16"),   # the split partial states would not fit the array: one split per plane instead
 ]
 
 
@@ -55,6 +58,9 @@ def test_static_entry_point_matches_handle_entry_point(case):
             assert torch.isfinite(got.float()).all()
             err = _rel(got, want)
             assert err <= TOL[dtype], f"call {rep}: max-rel difference {err:.3e}"
+            ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, gh, gw, ks, threads=8)
+            err = float(np.max(np.abs(got.double().cpu().numpy() - ref)) / np.max(np.abs(ref)))
+            assert err <= TOL[dtype], f"call {rep}: max-rel error against the oracle {err:.3e}"
 
 
 def test_static_entry_point_rejects_what_does_not_fit():
@@ -75,4 +81,10 @@ def test_static_entry_point_rejects_what_does_not_fit():
                                           1, 1, 2, 2, 64, 3, 0.0, b.CASTLING_BF16, 0) == b.ERR_INVALID_ARG
     assert b.castling_attn_forward_static(x.data_ptr(), x.data_ptr(), x.data_ptr(), w.data_ptr(), None, out.data_ptr(),
                                           1, 1, 2, 2, 64, 4, 0.0, b.CASTLING_BF16, 0) == b.ERR_INVALID_ARG
+    # the output may overlap none of the inputs, the filters and the bias included
+    big = torch.zeros(4 * 64 + 64 * 9, dtype=torch.bfloat16, device=dev)
+    assert b.castling_attn_forward_static(x.data_ptr(), x.data_ptr(), x.data_ptr(), big[128:].data_ptr(), None,
+                                          big.data_ptr(), 1, 1, 2, 2, 64, 3, 0.0, b.CASTLING_BF16, 0) == b.ERR_INVALID_ARG
+    assert b.castling_attn_forward_static(x.data_ptr(), x.data_ptr(), x.data_ptr(), w.data_ptr(), big[64:].data_ptr(),
+                                          big.data_ptr(), 1, 1, 2, 2, 64, 3, 0.0, b.CASTLING_BF16, 0) == b.ERR_INVALID_ARG
     torch.cuda.synchronize()
