@@ -322,7 +322,7 @@ def main():
     # algorithmic bytes per launch: the state kernel must read K and V, the apply kernel must read Q
     # and write O (V's one compulsory read is booked to the state kernel); a single-kernel forward moves
     # all four tensors; the split reduction and the leading-token rows move no algorithmic bytes
-    per_kernel = {"tc_state": 2, "tc_apply": 2, "simt_state": 2, "simt_apply": 2, "tc_fused": 4, "simt_fused": 4}
+    per_kernel = {"tc_state": 2, "tc_apply": 2, "simt_state": 2, "simt_apply": 2, "tc_fused": 4, "simt_fused": 4, "tc_pipe": 4}
     alg = {n: per_kernel.get(n, 0) * tensor_bytes for n in kernels}
     top = max(kernels, key=kernels.get) if kernels else None
     roofline = None

@@ -52,14 +52,14 @@ size_t workspace_words(int BH, int N, int d, bool bf16) {
     int P = castling::simt_choose_splits(BH, N);
     size_t words = castling::state_words(d);
     if (bf16 && (d == 64 || d == 32)) {  // shapes the tensor-core kernels may take: they keep 64-wide states
-        const int Pt = castling::tc::choose_splits(BH, castling::tc::rows_per_head(N, d));
+        const int Pt = castling::tc::max_splits(BH, castling::tc::rows_per_head(N, d));
         if (Pt > P) P = Pt;
         words = castling::tc::kStateWords;
     }
     size_t slots = (size_t)BH * (P > 1 ? P : 0);  // partial states behind the BH final ones
     if (bf16 && d == 32 && BH % 2 == 0) {
         // two width-32 heads side by side (token-major layouts): BH / 2 planes of N rows each
-        const int Pp = castling::tc::choose_splits(BH / 2, N);
+        const int Pp = castling::tc::max_splits(BH / 2, N);
         if (Pp > 1 && (size_t)(BH / 2) * Pp > slots) slots = (size_t)(BH / 2) * Pp;
     }
     return castling::kHeaderWords + ((size_t)BH + slots) * words;
@@ -105,7 +105,8 @@ int ensure_workspace(castling_attn* h, int BH, int N, int d, bool bf16) {
 }
 
 int ensure_counters(castling_attn* h, int BH) {
-    const size_t want = (size_t)BH * castling::tc::kCountersPerHead;
+    // either variant of the tensor-core path: 17 words per plane, or a header and 20 words per plane
+    const size_t want = castling::tc::kPipeCtrHeader + (size_t)BH * castling::tc::kPipeCtrPerPlane;
     if (want <= h->counters_cap) return CASTLING_OK;
     size_t cap = 4096;
     while (cap < want) cap *= 2;

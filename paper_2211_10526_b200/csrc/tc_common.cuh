@@ -14,6 +14,7 @@ enum : unsigned {
     kStatusStateTimeout = 1u << 0,
     kStatusApplyTimeout = 1u << 1,
     kStatusFusedTimeout = 1u << 2,
+    kStatusPipeTimeout = 1u << 3,
 };
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait, then give up

@@ -2,6 +2,8 @@
 // (the stream is the only synchronisation between the phases; no kernel waits on another).
 #include "tc_host.cuh"
 
+#include <cstdlib>
+
 namespace castling {
 namespace tc {
 
@@ -48,6 +50,19 @@ int choose_splits(int BH, int N) {
     return (tiles + per - 1) / per;
 }
 
+// CASTLING_TC_TWO_KERNELS=1 in the environment selects the separate state and apply kernels instead of the
+// one-kernel forward (for comparisons; read once).
+static bool two_kernels() {
+    static const bool on = [] { const char* e = getenv("CASTLING_TC_TWO_KERNELS"); return e && e[0] == '1'; }();
+    return on;
+}
+
+// Token splits of a plane, whichever of the two variants runs: the workspace holds that many partial states.
+int max_splits(int BH, int rows) {
+    const int a = choose_splits(BH, rows), b = plan_pipe(BH, rows, 16, 8).P;
+    return a > b ? a : b;
+}
+
 cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
@@ -65,16 +80,25 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
         timer->mark(stream, "tc_fused");
         return cudaSuccess;
     }
-    const int tiles = (rows_per_head(p.N, p.d) + kStateTile - 1) / kStateTile;
-    const int per = (tiles + P - 1) / P;
-    cudaError_t e = launch_state(p, ws_partial, ws_state, counters, P, per, status, stream);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-    timer->mark(stream, "tc_state");
-    e = launch_apply(p, ws_state, 1, status, stream);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-    timer->mark(stream, "tc_apply");
+    cudaError_t e;
+    if (!two_kernels()) {
+        // state and apply pipelines in one persistent kernel: V is read from memory once
+        e = launch_pipe(p, ws_partial, ws_state, counters, status, stream);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        timer->mark(stream, "tc_pipe");
+    } else {
+        const int tiles = (rows_per_head(p.N, p.d) + kStateTile - 1) / kStateTile;
+        const int per = (tiles + P - 1) / P;
+        e = launch_state(p, ws_partial, ws_state, counters, P, per, status, stream);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        timer->mark(stream, "tc_state");
+        e = launch_apply(p, ws_state, 1, status, stream);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        timer->mark(stream, "tc_apply");
+    }
     if (p.prefix > 0) {
         e = launch_prefix_rows(p, ws_state, stream);
         if (e != cudaSuccess) return e;

@@ -34,6 +34,8 @@ constexpr int kStateWords = 64 * 64 + 64;
 
 // Token splits of the tensor-core state kernel and the workspace words it needs beyond the state.
 int choose_splits(int BH, int N);
+// The larger of that and the one-kernel forward's splits: what the workspace is sized for.
+int max_splits(int BH, int rows);
 
 // Enqueue state build, split reduction and apply for one problem.  `status` is the device status
 // word; `counters` holds kCountersPerHead zero-initialised arrival counters per (b,h), left at zero by every call.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
@@ -47,6 +49,25 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
 cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st);
 // Output rows of the off-grid leading tokens (p.prefix of them per plane), from the final state.
 cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_t st);
+
+// One-kernel forward for longer sequences (csrc/tc_pipe.cu): a state pipeline and an apply pipeline share
+// every CTA; the CTAs signal one another through counters in global memory.
+// Counter layout: kPipeCtrHeader words (word 0 counts the CTAs that have left), then kPipeCtrPerPlane words per
+// plane: [0, 16) arrivals per group of token splits, then the arrivals of the groups, the plane's
+// "state is final" flag and the count of applied patches (times the conv warps of a CTA).  All zero between calls.
+constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 20;
+constexpr int kPipeCtrGroups = 16, kPipeCtrReady = 17, kPipeCtrApplied = 18;
+constexpr int kPipeMaxSplits = 64;
+struct PipePlan {
+    int grid;          // CTAs (at most one per multiprocessor)
+    int s_tiles;       // 64-row state tiles per plane
+    int s_per, P;      // tiles per token split, token splits per plane
+    int plane_order;   // apply the planes in order on every CTA (V of all planes does not fit L2)
+    int ahead;         // planes the state pipeline may run ahead of the apply pipeline
+};
+PipePlan plan_pipe(int BH, int rows, int cols, int gridH);
+// Partial states live at partial[plane][split], final ones at state[plane]; ctr as described above.
+cudaError_t launch_pipe(const Problem& p, float* partial, float* state, unsigned* ctr, unsigned* status, cudaStream_t st);
 
 // Single-kernel forward for short sequences (bf16, 3x3 or 5x5 filters, at most 256 128-byte rows per plane:
 // d = 64 with N <= 256, two width-32 heads per row with N <= 256, or width-32 token pairs with N <= 512): no workspace.
