@@ -50,11 +50,11 @@ int choose_splits(int BH, int N) {
     return (tiles + per - 1) / per;
 }
 
-// CASTLING_TC_TWO_KERNELS=1 in the environment selects the separate state and apply kernels instead of the
-// one-kernel forward (for comparisons; read once).
+// CASTLING_TC_ONE_KERNEL=1 in the environment selects the one-kernel forward (state and apply pipelines side
+// by side in every CTA) instead of the separate state and apply kernels, which measure faster (read once).
 static bool two_kernels() {
-    static const bool on = [] { const char* e = getenv("CASTLING_TC_TWO_KERNELS"); return e && e[0] == '1'; }();
-    return on;
+    static const bool one = [] { const char* e = getenv("CASTLING_TC_ONE_KERNEL"); return e && e[0] == '1'; }();
+    return !one;
 }
 
 // Token splits of a plane, whichever of the two variants runs: the workspace holds that many partial states.

@@ -248,15 +248,15 @@ PREFIX_CASES = [
     (16, 4, 1, 7, 7, 32, 3, "bf16", "head_major", 1, 1),     # CUDA cores, single-launch kernel (odd N)
     (4, 12, 1, 14, 14, 64, 3, "bf16", "head_major", 2, 1),   # DeiT-shaped with a class token: single tensor-core kernel
     (2, 3, 2, 15, 16, 64, 5, "bf16", "head_major", 2, 1),    # 242 tokens, 5 x 5
-    (2, 2, 1, 24, 20, 64, 3, "bf16", "head_major", 2, 2),    # one-kernel forward + leading rows
-    (1, 2, 3, 37, 53, 64, 5, "bf16", "head_major", 2, 2),
+    (2, 2, 1, 24, 20, 64, 3, "bf16", "head_major", 2, 3),    # state + apply + leading rows
+    (1, 2, 3, 37, 53, 64, 5, "bf16", "head_major", 2, 3),
     (2, 2, 2, 24, 20, 32, 3, "bf16", "head_major", 2, 1),    # width 32, even N: token pairs, single kernel (241 rows)
-    (2, 2, 2, 40, 30, 32, 5, "bf16", "head_major", 2, 2),    # ... one-kernel forward + leading rows
+    (2, 2, 2, 40, 30, 32, 5, "bf16", "head_major", 2, 3),    # ... state + apply + leading rows
     (2, 2, 1, 24, 20, 32, 3, "bf16", "head_major", 1, 3),    # width 32, odd N: CUDA cores (P = 2 splits)
-    (2, 4, 1, 24, 20, 32, 5, "bf16", "token_major", 2, 2),   # width 32 token-major: head pairs
+    (2, 4, 1, 24, 20, 32, 5, "bf16", "token_major", 2, 3),   # width 32 token-major: head pairs
     (2, 4, 1, 12, 12, 32, 3, "bf16", "token_major", 2, 1),   # ... in the single-kernel forward
     (2, 3, 1, 14, 14, 64, 3, "bf16", "token_major", 2, 1),
-    (1, 2, 2, 30, 31, 64, 3, "bf16", "fused_qkv", 2, 2),
+    (1, 2, 2, 30, 31, 64, 3, "bf16", "fused_qkv", 2, 3),
 ]
 
 
