@@ -57,9 +57,9 @@ static bool two_kernels() {
     return !one;
 }
 
-// Token splits of a plane, whichever of the two variants runs: the workspace holds that many partial states.
-int max_splits(int BH, int rows) {
-    const int a = choose_splits(BH, rows), b = plan_pipe(BH, rows, 16, 8).P;
+size_t partial_slots(int BH, int rows) {
+    const int P = choose_splits(BH, rows);
+    const size_t a = P > 1 ? (size_t)BH * P : 0, b = pipe_partial_slots(BH, rows);
     return a > b ? a : b;
 }
 
@@ -81,7 +81,7 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
         return cudaSuccess;
     }
     cudaError_t e;
-    if (!two_kernels()) {
+    if (!two_kernels() && pipe_supports(p)) {
         // state and apply pipelines in one persistent kernel: V is read from memory once
         e = launch_pipe(p, ws_partial, ws_state, counters, status, stream);
         if (e != cudaSuccess) return e;

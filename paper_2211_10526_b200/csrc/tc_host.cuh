@@ -34,8 +34,9 @@ constexpr int kStateWords = 64 * 64 + 64;
 
 // Token splits of the tensor-core state kernel and the workspace words it needs beyond the state.
 int choose_splits(int BH, int N);
-// The larger of that and the one-kernel forward's splits: what the workspace is sized for.
-int max_splits(int BH, int rows);
+// Partial states (of kStateWords each) behind the final ones that either variant of the path needs for
+// BH planes of `rows` 128-byte rows: what the workspace is sized for.
+size_t partial_slots(int BH, int rows);
 
 // Enqueue state build, split reduction and apply for one problem.  `status` is the device status
 // word; `counters` holds kCountersPerHead zero-initialised arrival counters per (b,h), left at zero by every call.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
@@ -50,23 +51,26 @@ cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned
 // Output rows of the off-grid leading tokens (p.prefix of them per plane), from the final state.
 cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_t st);
 
-// One-kernel forward for longer sequences (csrc/tc_pipe.cu): a state pipeline and an apply pipeline share
-// every CTA; the CTAs signal one another through counters in global memory.
+// One-kernel forward for long sequences (csrc/tc_pipe.cu): a state pipeline and an apply pipeline share every
+// CTA; the CTAs signal one another through counters in global memory.
 // Counter layout: kPipeCtrHeader words (word 0 counts the CTAs that have left), then kPipeCtrPerPlane words per
-// plane: [0, 16) arrivals per group of token splits, then the arrivals of the groups, the plane's
-// "state is final" flag and the count of applied patches (times the conv warps of a CTA).  All zero between calls.
-constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 20;
-constexpr int kPipeCtrGroups = 16, kPipeCtrReady = 17, kPipeCtrApplied = 18;
-constexpr int kPipeMaxSplits = 64;
+// plane: CTAs whose sums over their rows of the plane are written, CTAs whose slice of the total is written,
+// CTAs that have applied their share of the plane.  All zero between calls.
+constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 4;
+constexpr int kPipeCtrWritten = 0, kPipeCtrSummed = 1, kPipeCtrApplied = 2;
 struct PipePlan {
+    bool ok;           // the one-kernel forward takes this shape
     int grid;          // CTAs (at most one per multiprocessor)
     int s_tiles;       // 64-row state tiles per plane
-    int s_per, P;      // tiles per token split, token splits per plane
-    int plane_order;   // apply the planes in order on every CTA (V of all planes does not fit L2)
     int ahead;         // planes the state pipeline may run ahead of the apply pipeline
+    int ring;          // planes whose per-CTA sums are kept at a time
 };
+// rows: 128-byte rows per plane (leading tokens included); cols x gridH: the token grid in 128-byte columns.
 PipePlan plan_pipe(int BH, int rows, int cols, int gridH);
-// Partial states live at partial[plane][split], final ones at state[plane]; ctr as described above.
+bool pipe_supports(const Problem& p);
+// Per-CTA sums (of kStateWords each) the workspace must hold behind the final states for such planes.
+size_t pipe_partial_slots(int BH, int rows);
+// Per-CTA sums live at partial[plane % ring][cta], final ones at state[plane]; ctr as described above.
 cudaError_t launch_pipe(const Problem& p, float* partial, float* state, unsigned* ctr, unsigned* status, cudaStream_t st);
 
 // Single-kernel forward for short sequences (bf16, 3x3 or 5x5 filters, at most 256 128-byte rows per plane:

@@ -1,24 +1,29 @@
-// Whole forward pass of the tensor-core path as ONE persistent kernel (bf16; width-64 heads, or width-32
-// heads packed two to a 128-byte row):
+// Whole forward pass of the tensor-core path as ONE persistent kernel for long sequences (bf16; width-64
+// heads, or width-32 heads packed two to a 128-byte row):
 //     S = sum_n k^_n^T v_n,  s = sum_n v_n            (state, per (b,h))
 //     out_t = (1/pi) q^_t S + 1/2 s + bias + DWConv(V)_t                              (Eq. 9)
-// One CTA per multiprocessor, launched cooperatively so that all CTAs are resident.  Every CTA runs two
-// pipelines side by side, in different warps:
+// One CTA per multiprocessor, launched cooperatively so that all CTAs are resident.  The planes (one per
+// (b,h)) are taken in order, and every CTA takes a share of every plane, in two pipelines that run side by
+// side in different warps:
 //   state pipeline   warp 2 (TMA: K and V tiles of 64 rows), warp 3 (UMMAs, A = [K^ ; 1 0 0 ...] so that
 //                    accumulator row 64 is the token sum of V), warps 12..15 (scale every K row by
-//                    1 / max(||k||, eps) in place, read the finished accumulator out of TMEM, reduce the
-//                    token splits of a plane in a fixed order, publish the plane's state and raise its flag)
-//   apply pipeline   warp 0 (TMA: Q patch and V patch with halo), warp 1 (UMMAs: acc = Q S'), warps 4..11
-//                    (||q||, accumulator rows scaled by 1/||q|| to shared memory as fp32), conv warps
-//                    (depthwise convolution of the V patch on CUDA cores, lane = channel pair; add the
-//                    scaled accumulator row, 1/2 s and the bias; one rounding to bf16; 128-byte rows stored
-//                    straight to memory)
-// The state pipeline walks the planes in order and never waits for the apply pipeline (except for an
-// optional bound on how many planes it may run ahead); the apply pipeline of a plane waits for that
-// plane's flag.  While plane p is being applied, the states of the planes after it are being built, so
-// the V rows that the apply pipeline needs were read moments ago and are served from L2: V comes
-// from HBM once.  Every wait is bounded; a wait that runs out raises a bit in the status word, and every
-// CTA that sees the bit leaves.
+//                    1 / max(||k||, eps) in place; write this CTA's sums over its rows of the plane to memory
+//                    and count them)
+//   apply pipeline   warp 0 (TMA: Q patch and V patch with halo), warp 1 (UMMAs: acc = Q S'), conv warps
+//                    (depthwise convolution of the V patch on CUDA cores, lane = channel pair; result plus
+//                    1/2 s and the bias staged in shared memory as fp32), warps 4..11 (||q||, accumulator row
+//                    scaled by 1/||q|| plus the staged row, one rounding to bf16, patch stored with TMA)
+// The sums of the CTAs are added up by the apply pipelines, which have to wait for them anyway: when all
+// CTAs have written their sums of a plane, CTA c adds slice c of the state words over all CTAs (in a fixed
+// order: the result does not depend on timing) and counts its slice; when all slices are counted the
+// plane's state is final.  A CTA adds its slice of the next plane early, when it enters a plane, so that
+// nobody has to wait for a slow CTA at the plane after.  The state pipeline never waits for another CTA's
+// sums; it only keeps a bounded number of planes ahead of the apply pipeline, so that the V rows the
+// apply pipeline needs were read moments ago and are served from L2: V comes from HBM once.
+// Flags are polled by one thread per CTA (many pollers on one address queue up at its L2 slice and slow every
+// other access to that slice); the other threads sleep on a shared-memory barrier that thread completes.
+// Every wait is bounded; a wait that runs out raises a bit in the status word, and every CTA that sees the
+// bit leaves.
 #include "tc_common.cuh"
 #include "tc_host.cuh"
 
@@ -30,18 +35,17 @@ constexpr int kD = 64;
 constexpr int kTY = 8, kTX = 16;            // patch: 8 rows x 16 columns of 128-byte rows
 constexpr int kPatch = kTY * kTX;
 constexpr int kQBytes = kPatch * kD * 2;    // 16 KiB
-constexpr int kStgRow = kD * 4;             // fp32 accumulator row; 16-byte chunk c of row t sits at chunk c ^ (t & 7)
-constexpr int kStgBytes = kPatch * kStgRow; // 32 KiB
+constexpr int kStgStride = kD * 4 + 16;     // fp32 row + 16 B pad: conflict-free row-per-thread reads
+constexpr int kStgBytes = kPatch * kStgStride;
 constexpr int kEpiWarps = 8, kEpiThreads = kEpiWarps * 32;
 constexpr int kNormWarps = 4, kNormThreads = kNormWarps * 32;
 constexpr int kSTile = 64;                  // rows per state stage
 constexpr int kSTileBytes = kSTile * 128;   // 8 KiB per operand tile
 constexpr int kSStage = 2 * kSTileBytes;    // K then V
-constexpr int kSStages = 3;
 constexpr int kOnesBytes = 2048;
 constexpr int kTmemCols = 256;              // [0,128): two apply accumulators; [128,256): two state accumulators
-constexpr int kGroup = 4;                   // splits per first-level reduction group
 constexpr int kWords = kD * kD + kD;        // one state: S then s
+constexpr int kWords4 = kWords / 4;
 constexpr int kFirstWarpEpi = 4, kFirstWarpNorm = kFirstWarpEpi + kEpiWarps, kFirstWarpConv = kFirstWarpNorm + kNormWarps;
 constexpr unsigned kBit = kStatusPipeTimeout;
 
@@ -54,80 +58,75 @@ template <int KS, bool PAIR> struct PGeo {
     static constexpr int HY = kTY + 2 * R, HX = kTX + 2 * HC;
     static constexpr int kVBytes = HY * HX * kD * 2;
     static constexpr int kStage = ((kQBytes + kVBytes + 1023) / 1024) * 1024;
-    static constexpr int kStages = (KS == 3) ? 3 : 2;
-    // 3x3: one staging buffer, the conv warps hold the first half of a patch's results in registers
-    // while the epilogue warps fill it; 5x5 (larger window in registers): two staging buffers
-    static constexpr int kStgBufs = (KS == 3) ? 1 : 2;
-    static constexpr int kHold = (kStgBufs == 1) ? kTX / 4 : 0;   // output columns per warp held back
-    static constexpr int kOffS = 0, kOffStg = 8192, kOffStages = kOffStg + kStgBufs * kStgBytes;
-    static constexpr int kOffSStages = kOffStages + kStages * kStage;
+    static constexpr int kStages = 2;                      // apply stages (Q patch + V patch with halo)
+    static constexpr int kSStages = (KS == 3) ? 3 : 2;     // state stages (K tile + V tile)
+    // S' | out patch | apply stages | staging x2 | state stages | ones | rq x2 | barriers
+    static constexpr int kOffS = 0, kOffOut = 8192, kOffStages = kOffOut + kQBytes;
+    static constexpr int kOffStg = kOffStages + kStages * kStage;
+    static constexpr int kOffSStages = ((kOffStg + 2 * kStgBytes + 1023) / 1024) * 1024;
     static constexpr int kOffOnes = kOffSStages + kSStages * kSStage;
-    static constexpr int kOffRq = kOffOnes + kOnesBytes;          // [2][2][kPatch] partial sums of squares
-    static constexpr int kOffBar = kOffRq + 2 * 2 * kPatch * 4;
+    static constexpr int kOffRq = kOffOnes + kOnesBytes;   // sum of squares of each half of a Q row
+    static constexpr int kOffBar = kOffRq + 2 * kPatch * 4;
     static constexpr size_t kSmem = 1024 + kOffBar + 512;
+    static_assert(kSmem <= 227 * 1024, "shared memory of the one-kernel forward");
 };
 
 struct PipeParams {
-    float* partial;                // [BH][P][kWords] per-split sums (P > 1)
+    float* partial;                // [ring][CTA][kWords] sums of one CTA over its rows of one plane
     float* state;                  // [BH][kWords] final sums
     unsigned* ctr;                 // kPipeCtrHeader words, then kPipeCtrPerPlane per plane; all zero between calls
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
-    __nv_bfloat16* out;            // first grid token of plane 0
-    Layout lo;
     int flat;                      // the planes have one uniform stride: the apply tensor maps are 4-D
     int H, head0, BH, hdiv;
     int tilesX, tilesY;            // patches per plane
-    int gridH, cols;               // grid rows; 128-byte columns per grid row
-    int s_tiles, s_per, P;         // state tiles per plane, tiles per split, splits per plane
-    int plane_order;               // every CTA takes a share of every plane, plane after plane (long sequences)
+    int s_tiles;                   // 64-row state tiles per plane
     int ahead;                     // the state pipeline starts plane p only when plane p - ahead is applied
+    int ring;                      // plane slots of `partial`: plane p uses slot p % ring
     float eps2;
     unsigned* status;
 };
 
-// This CTA's patches, in the order every role of the apply pipeline visits them.
+// This CTA's patches, in the order every role of the apply pipeline visits them: plane after plane, a
+// contiguous share of each plane's patches.  Every CTA has at least one patch in every plane.
 struct PatchWalk {
-    int bh, rem, end, left, tpb, G, cta, BH;
-    bool by_plane;
+    int bh, rem, end, tpb, G, cta, BH;
     __device__ void init(const PipeParams& prm) {
         tpb = prm.tilesX * prm.tilesY; G = (int)gridDim.x; cta = (int)blockIdx.x; BH = prm.BH;
-        by_plane = prm.plane_order != 0;
-        if (!by_plane) {  // one contiguous range of the plane-major patch list
-            const long long n = (long long)BH * tpb;
-            const int g0 = (int)(n * cta / G), g1 = (int)(n * (cta + 1) / G);
-            left = g1 - g0; bh = g0 / tpb; rem = g0 - bh * tpb; end = tpb;
-        } else {
-            bh = -1; rem = end = 0; left = 1;
-            next_plane();
-        }
+        bh = -1; rem = end = 0;
+        next_plane();
     }
     __device__ void next_plane() {
-        while (true) {
-            if (++bh >= BH) { left = 0; return; }
-            const int cc = (cta + 37 * bh) % G;  // the larger shares rotate over the CTAs from plane to plane
-            rem = (int)((long long)tpb * cc / G); end = (int)((long long)tpb * (cc + 1) / G);
-            if (rem < end) return;
-        }
+        if (++bh >= BH) return;
+        const int cc = (cta + 37 * bh) % G;  // the larger shares rotate over the CTAs from plane to plane
+        rem = (int)((long long)tpb * cc / G); end = (int)((long long)tpb * (cc + 1) / G);
     }
-    __device__ bool valid() const { return left > 0; }
-    __device__ void step() {
-        ++rem;
-        if (!by_plane) { --left; if (rem == tpb) { rem = 0; ++bh; } }
-        else if (rem == end) next_plane();
-    }
+    __device__ bool valid() const { return bh < BH; }
+    __device__ void step() { if (++rem == end) next_plane(); }
 };
+
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Adds one to a counter in global memory, ordered after every write that happens before the call: the caller's own
+// and, through a preceding CTA barrier, those of the other threads of the CTA.  One releasing thread per CTA: a
+// device-wide fence in every thread waits for the copies the CTA's pipelines have in flight, again and again.
+__device__ __forceinline__ void signal_add(unsigned* p) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+}
 
 // Bounded wait for a counter in global memory to reach `want`.  Gives up (returns false) when the limit
 // runs out (raising the status bit), when this CTA has given up elsewhere, or when any CTA has raised a bit.
 __device__ __forceinline__ bool wait_counter(const unsigned* p, unsigned want, volatile int* abort_flag, unsigned* status) {
-    auto poll = [&]() { unsigned v; asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v; };
-    if (poll() >= want) return true;
+    if (ld_acquire(p) >= want) return true;
     const unsigned long long t0 = global_ns();
     uint32_t spins = 0;
     while (true) {
-        __nanosleep(100);
-        if (poll() >= want) return true;
+        __nanosleep(200);
+        if (ld_acquire(p) >= want) return true;
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
             if (*reinterpret_cast<volatile unsigned*>(status) != 0) { *abort_flag = 1; return false; }
@@ -145,45 +144,20 @@ __device__ __forceinline__ bool barrier_any(uint32_t id, uint32_t threads, bool 
     return r != 0;
 }
 
-__device__ __forceinline__ void st_global_hint(void* p, uint32_t v, uint64_t policy) {
-    asm volatile("st.global.L2::cache_hint.b32 [%0], %1, %2;" ::"l"(p), "r"(v), "l"(policy) : "memory");
-}
-
-// Sum `n` states of kWords floats, `stride` floats apart, in index order into dst (128 threads).
-__device__ __forceinline__ void sum_states(const float* src, size_t stride, int n, float* dst, int t) {
-    constexpr int kWords4 = kWords / 4;
-    for (int i = t; i < kWords4; i += kNormThreads) {
-        float4 acc = __ldcg(reinterpret_cast<const float4*>(src) + i);
-        int m = 1;
-        for (; m + 3 <= n; m += 3) {
-            const float4 a = __ldcg(reinterpret_cast<const float4*>(src + (size_t)m * stride) + i);
-            const float4 b = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(m + 1) * stride) + i);
-            const float4 c = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(m + 2) * stride) + i);
-            acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
-            acc.x += b.x; acc.y += b.y; acc.z += b.z; acc.w += b.w;
-            acc.x += c.x; acc.y += c.y; acc.z += c.z; acc.w += c.w;
-        }
-        for (; m < n; ++m) {
-            const float4 a = __ldcg(reinterpret_cast<const float4*>(src + (size_t)m * stride) + i);
-            acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
-        }
-        reinterpret_cast<float4*>(dst)[i] = acc;
-    }
-}
-
 // MODE 0: width-64 heads; 1: width-32 heads, two adjacent tokens per 128-byte row; 2: two width-32 heads side
 // by side in one row (block-diagonal state).
 template <int KS, int MODE>
 __global__ void __launch_bounds__((PGeo<KS, MODE == 1>::kThreads), 1)
 tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
                const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmVh,
-               const PipeParams prm) {
+               const __grid_constant__ CUtensorMap tmO, const PipeParams prm) {
     constexpr bool PAIR = (MODE == 1), BLOCKDIAG = (MODE == 2), HALVES = PAIR || BLOCKDIAG;
     using G = PGeo<KS, PAIR>;
-    constexpr int NA = G::kStages, NS = kSStages;
+    constexpr int NA = G::kStages, NS = G::kSStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* S_s = smem + G::kOffS;
+    uint8_t* out_s = smem + G::kOffOut;
     uint8_t* stg = smem + G::kOffStg;
     uint8_t* stages = smem + G::kOffStages;
     uint8_t* sstages = smem + G::kOffSStages;
@@ -193,36 +167,39 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     uint64_t* a_full = bars;                 // [NA] Q and V patch landed
     uint64_t* a_empty = a_full + NA;         // [NA] stage consumed (conv + epilogue warps, UMMA commit)
     uint64_t* acc_full = a_empty + NA;       // [2]  apply UMMAs retired
-    uint64_t* acc_free = acc_full + 2;       // [2]  accumulator read out (epilogue threads)
-    uint64_t* stg_full = acc_free + 2;       // [2]  staging written (epilogue threads)
-    uint64_t* stg_free = stg_full + 2;       // [2]  staging read (conv threads)
-    uint64_t* s_ready = stg_free + 2;        //      S' of the current plane written (epilogue threads)
-    uint64_t* s_full = s_ready + 1;          // [NS] K and V tile landed
+    uint64_t* conv_full = acc_full + 2;      // [2]  staging written (conv threads)
+    uint64_t* buf_free = conv_full + 2;      // [2]  accumulator and staging read out (epilogue threads)
+    uint64_t* s_ready = buf_free + 2;        //      S' of the current plane written (epilogue threads)
+    uint64_t* p_ready = s_ready + 1;         //      the current plane's state is final (one polling thread)
+    uint64_t* s_full = p_ready + 1;          // [NS] K and V tile landed
     uint64_t* s_scaled = s_full + NS;        // [NS] K rows normalised
     uint64_t* s_empty = s_scaled + NS;       // [NS] state UMMAs of the stage retired
-    uint64_t* sacc_full = s_empty + NS;      // [2]  accumulation of an item retired
+    uint64_t* sacc_full = s_empty + NS;      // [2]  accumulation of a plane retired
     uint64_t* sacc_free = sacc_full + 2;     // [2]  accumulator read out
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sacc_free + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* last_slot = reinterpret_cast<int*>(tmem_slot + 2);
+    volatile int* sum_go = reinterpret_cast<volatile int*>(tmem_slot + 3);  // the polling thread's verdict on a slice sum
+    unsigned* applied_s = reinterpret_cast<unsigned*>(tmem_slot + 4);  // [8] conv warps done with plane p, slot p & 7
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_cta = (int)gridDim.x, cta = (int)blockIdx.x;
-    const int n_items = prm.BH * prm.P;
     unsigned* plane_ctr = prm.ctr + kPipeCtrHeader;
+    // this CTA's rows of every plane, as a range of 64-row tiles (never empty: the launcher sees to it)
+    const int t_begin = (int)((long long)prm.s_tiles * cta / n_cta), t_end = (int)((long long)prm.s_tiles * (cta + 1) / n_cta);
 
     if (tid == 0) {
         for (int s = 0; s < NA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], G::kConvThreads + kEpiThreads + 1); }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&acc_full[b], 1); mbar_init(&acc_free[b], kEpiThreads);
-            mbar_init(&stg_full[b], kEpiThreads); mbar_init(&stg_free[b], G::kConvThreads);
+            mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], G::kConvThreads); mbar_init(&buf_free[b], kEpiThreads);
             mbar_init(&sacc_full[b], 1); mbar_init(&sacc_free[b], kNormThreads);
         }
-        mbar_init(s_ready, kEpiThreads);
+        mbar_init(s_ready, kEpiThreads); mbar_init(p_ready, 1);
         for (int s = 0; s < NS; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_scaled[s], kNormThreads); mbar_init(&s_empty[s], 1); }
         *abort_flag = 0;
+        for (int i = 0; i < 8; ++i) applied_s[i] = 0;
         mbar_fence_init();
-        tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmVs); tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmVh);
+        tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmVs); tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmVh); tma_prefetch_desc(&tmO);
     }
     if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
     if (warp >= kFirstWarpNorm && warp < kFirstWarpConv) {
@@ -281,7 +258,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     ++seg; prev_bh = wk.bh;
                 }
                 if (!mbar_wait(&a_full[s], use & 1, abort_flag, prm.status, kBit)) break;
-                if (ub > 0 && !mbar_wait(&acc_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
+                if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
                 tcgen05_fence_after_sync();
                 const uint32_t q_addr = smem_u32(stages + s * G::kStage);
 #pragma unroll
@@ -300,16 +277,13 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             int issued = 0;
             // K is read once; V is read again by the apply pipeline: keep it in L2 as long as possible
             const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_last();
-            const unsigned applied = (unsigned)(prm.tilesX * prm.tilesY * G::kConvWarps);  // arrivals of a whole plane
             bool ok = true;
-            for (int item = cta; item < n_items && ok; item += n_cta) {
-                const int plane = item / prm.P, part = item - plane * prm.P;
-                const int t0 = part * prm.s_per, t1 = min(prm.s_tiles, t0 + prm.s_per);
+            for (int plane = 0; plane < prm.BH && ok; ++plane) {
                 if (plane >= prm.ahead &&
-                    !wait_counter(plane_ctr + (size_t)(plane - prm.ahead) * kPipeCtrPerPlane + kPipeCtrApplied, applied,
+                    !wait_counter(plane_ctr + (size_t)(plane - prm.ahead) * kPipeCtrPerPlane + kPipeCtrApplied, (unsigned)n_cta,
                                   abort_flag, prm.status)) break;
                 const int pb = plane / prm.hdiv, ph = plane - pb * prm.hdiv;
-                for (int t = t0; t < t1; ++t, ++issued) {
+                for (int t = t_begin; t < t_end; ++t, ++issued) {
                     const int s = issued % NS, use = issued / NS;
                     if (use > 0 && !mbar_wait(&s_empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) { ok = false; break; }
                     uint8_t* ks = sstages + s * kSStage;
@@ -329,13 +303,11 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             constexpr uint32_t idesc = umma_idesc_bf16(128, kD, true, true);
             const uint32_t ones_addr = smem_u32(ones);
             bool ok = true;
-            int gt = 0, k_item = 0;  // tiles and items issued so far
-            for (int item = cta; item < n_items && ok; item += n_cta, ++k_item) {
-                const int plane = item / prm.P, part = item - plane * prm.P;
-                const int t0 = part * prm.s_per, t1 = min(prm.s_tiles, t0 + prm.s_per);
-                const int buf = k_item & 1;
-                if (k_item >= 2) ok = mbar_wait(&sacc_free[buf], ((k_item >> 1) - 1) & 1, abort_flag, prm.status, kBit);
-                for (int t = t0; t < t1 && ok; ++t, ++gt) {
+            int gt = 0;  // tiles issued so far
+            for (int plane = 0; plane < prm.BH && ok; ++plane) {
+                const int buf = plane & 1;
+                if (plane >= 2) ok = mbar_wait(&sacc_free[buf], ((plane >> 1) - 1) & 1, abort_flag, prm.status, kBit);
+                for (int t = t_begin; t < t_end && ok; ++t, ++gt) {
                     const int s = gt % NS, use = gt / NS;
                     ok = mbar_wait(&s_scaled[s], use & 1, abort_flag, prm.status, kBit);
                     if (!ok) break;
@@ -345,7 +317,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     for (int j = 0; j < kSTile / 16; ++j) {  // one UMMA per 16 rows (K = 16)
                         const uint32_t a0 = ka + j * 2048, b0 = va + j * 2048;
                         umma_bf16(tmem_state + buf * kD, umma_desc_sw128(a0, ones_addr - a0, 1024),
-                                  umma_desc_sw128(b0, 0, 1024), idesc, (t != t0) || (j != 0));
+                                  umma_desc_sw128(b0, 0, 1024), idesc, (t != t_begin) || (j != 0));
                     }
                     umma_commit(&s_empty[s]);
                 }
@@ -355,24 +327,78 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     } else if (warp < kFirstWarpNorm) {
         // ================= apply pipeline: epilogue, thread = (token row of the patch, half of the channels) =================
         const int quarter = warp & 3, row = quarter * 32 + lane, et = tid - 32 * kFirstWarpEpi;
-        const int half = (warp - kFirstWarpEpi) >> 2;  // channels half*32 .. half*32 + 31
-        int prev_bh = -1;
-        bool failed = false;
+        const int ew = warp - kFirstWarpEpi;
+        const int half = ew >> 2;  // channels half*32 .. half*32 + 31
+        const bool leader = (et == 0);
+        const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
+        // this CTA's slice of the state words (as float4 positions), added over all CTAs' sums
+        const int q0 = (int)((long long)kWords4 * cta / n_cta), q1 = (int)((long long)kWords4 * (cta + 1) / n_cta);
+        // Adds the slice for `plane` once every CTA has written its sums of that plane.  Position by position,
+        // lane l of a warp adds the sums of CTAs l, l + 32, ... in that order and the 32 results meet in a fixed
+        // shuffle tree.  Returns 1 when done, 0 when the sums are not all there yet (only if !blocking), -1 after a
+        // failed wait.  All epilogue threads call it together and get the same answer.
+        auto slice_sum = [&](int plane, bool blocking) -> int {
+            unsigned* pc = plane_ctr + (size_t)plane * kPipeCtrPerPlane;
+            if (leader) {
+                int go;
+                if (blocking) go = wait_counter(&pc[kPipeCtrWritten], (unsigned)n_cta, abort_flag, prm.status) ? 1 : -1;
+                else go = (ld_acquire(&pc[kPipeCtrWritten]) >= (unsigned)n_cta) ? 1 : 0;
+                *sum_go = go;
+            }
+            named_barrier_sync(4, kEpiThreads);
+            const int go = *sum_go;
+            named_barrier_sync(4, kEpiThreads);  // everybody has read the verdict before the next one is written
+            if (go != 1) return go;
+            const float4* base = reinterpret_cast<const float4*>(prm.partial + (size_t)(plane % prm.ring) * n_cta * kWords);
+            float4* fin = reinterpret_cast<float4*>(prm.state + (size_t)plane * kWords);
+            for (int pos = q0 + ew; pos < q1; pos += kEpiWarps) {
+                float4 v[5];
+#pragma unroll
+                for (int j = 0; j < 5; ++j) {
+                    const int m = lane + 32 * j;
+                    v[j] = (m < n_cta) ? __ldcg(base + (size_t)m * kWords4 + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float4 acc = v[0];
+#pragma unroll
+                for (int j = 1; j < 5; ++j) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
+                for (int m = lane + 160; m < n_cta; m += 32) {
+                    const float4 u = __ldcg(base + (size_t)m * kWords4 + pos);
+                    acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
+                }
+#pragma unroll
+                for (int sh = 16; sh >= 1; sh >>= 1) {
+                    acc.x += __shfl_xor_sync(0xffffffffu, acc.x, sh); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, sh);
+                    acc.z += __shfl_xor_sync(0xffffffffu, acc.z, sh); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, sh);
+                }
+                if (lane == 0) fin[pos] = acc;
+            }
+            named_barrier_sync(4, kEpiThreads);
+            if (leader) signal_add(&pc[kPipeCtrSummed]);
+            return 1;
+        };
+        int prev_bh = -1, pseg = 0;
+        int summed = 0;  // this CTA's slices of planes [0, summed) are added
+        bool failed = false;  // the same for every epilogue thread wherever a barrier follows
         PatchWalk wk; wk.init(prm);
         for (int it = 0; wk.valid(); ++it, wk.step()) {
             const int b = it & 1, ub = it >> 1, s = it % NA, use = it / NA;
-            const int sb = (G::kStgBufs == 2) ? b : 0, su = (G::kStgBufs == 2) ? ub : it;  // staging buffer and its use count
             if (wk.bh != prev_bh && !failed) {
-                prev_bh = wk.bh;
+                const int p = wk.bh;
+                prev_bh = p;
+                if (summed <= p) {
+                    if (slice_sum(p, true) == 1) summed = p + 1; else failed = true;
+                }
+                if (!failed) {
+                    // the plane's state is final when every CTA has added its slice
+                    if (leader && wait_counter(plane_ctr + (size_t)p * kPipeCtrPerPlane + kPipeCtrSummed, (unsigned)n_cta, abort_flag, prm.status))
+                        mbar_arrive(p_ready);
+                    failed = barrier_any(4, kEpiThreads, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit));
+                    ++pseg;
+                }
                 // every UMMA that read the previous S' has retired (its acc_full was waited on below)
-                bool ready = true;
-                if (lane == 0)
-                    ready = wait_counter(plane_ctr + (size_t)wk.bh * kPipeCtrPerPlane + kPipeCtrReady, 1u, abort_flag, prm.status);
-                ready = __shfl_sync(0xffffffffu, (int)ready, 0) != 0;
-                if (!ready) { failed = true; }
-                else {
+                if (!failed) {
                     const int i = et >> 2, part = et & 3;  // row i of the operand, 16 columns part*16 ..
-                    const float* st = prm.state + (size_t)wk.bh * kWords;
+                    const float* st = prm.state + (size_t)p * kWords;
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
                         float4 lo, hi;
@@ -403,6 +429,12 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     }
                     fence_proxy_async_smem();
                     mbar_arrive(s_ready);
+                    // the next plane's slice, if its sums are there already: by the time anyone enters that plane,
+                    // every CTA has long since added its slice
+                    if (p + 1 < prm.BH && summed == p + 1) {
+                        const int r = slice_sum(p + 1, false);
+                        if (r == 1) summed = p + 2; else if (r < 0) failed = true;
+                    }
                 }
             }
             float a[32];
@@ -423,7 +455,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                         ss[e] = fmaf(lo, lo, ss[e]); ss[e] = fmaf(hi, hi, ss[e]);
                     }
                 }
-                rq_s[(b * 2 + half) * kPatch + row] = (ss[0] + ss[1]) + (ss[2] + ss[3]);
+                rq_s[half * kPatch + row] = (ss[0] + ss[1]) + (ss[2] + ss[3]);
                 mbar_arrive(&a_empty[s]);  // the Q rows of this stage have been read
                 failed = __any_sync(0xffffffffu, !mbar_wait(&acc_full[b], ub & 1, abort_flag, prm.status, kBit));
             }
@@ -435,102 +467,52 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 16; ++e) { a[e] = a0[e]; a[16 + e] = a1[e]; }
-                tcgen05_fence_before_sync();
-                mbar_arrive(&acc_free[b]);
+                failed = __any_sync(0xffffffffu, !mbar_wait(&conv_full[b], ub & 1, abort_flag, prm.status, kBit));
             }
-            if (!HALVES) {
-                // both halves of every row's sum of squares become visible; every thread learns whether one gave up
-                if (barrier_any(1, kEpiThreads, failed)) break;
-            } else if (failed) break;
-            const float rq = HALVES ? rsqrtf(fmaxf(rq_s[(b * 2 + half) * kPatch + row], prm.eps2))   // half row = one token / one head
-                                    : rsqrtf(fmaxf(rq_s[(b * 2) * kPatch + row] + rq_s[(b * 2 + 1) * kPatch + row], prm.eps2));
-            // the conv warps have read the previous contents of this staging buffer
-            if (su > 0 && __any_sync(0xffffffffu, !mbar_wait(&stg_free[sb], (su - 1) & 1, abort_flag, prm.status, kBit))) {
-                if (!HALVES) { failed = true; continue; }   // leave together at the next barrier
-                break;
-            }
-            uint8_t* srow = stg + sb * kStgBytes + row * kStgRow;
+            // the previous patch's TMA store must have read out_s before it is rewritten; the same barrier makes
+            // both halves of every row's sum of squares visible and tells every thread whether one has given up
+            if (it > 0 && leader) tma_store_wait_read();
+            if (barrier_any(1, kEpiThreads, failed)) break;
+            const float rq = HALVES ? rsqrtf(fmaxf(rq_s[half * kPatch + row], prm.eps2))   // half row = one token / one head
+                                    : rsqrtf(fmaxf(rq_s[row] + rq_s[kPatch + row], prm.eps2));
+            const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
+            uint8_t* orow = out_s + row * 128;
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-                *reinterpret_cast<float4*>(srow + (((half * 8 + e) ^ (row & 7)) << 4)) =
-                    make_float4(a[4 * e] * rq, a[4 * e + 1] * rq, a[4 * e + 2] * rq, a[4 * e + 3] * rq);
-            mbar_arrive(&stg_full[sb]);
+            for (int e = 0; e < 4; ++e) {  // 8 channels -> one 16-byte chunk of the bf16 row
+                const float4 c0 = *reinterpret_cast<const float4*>(srow + e * 32);
+                const float4 c1 = *reinterpret_cast<const float4*>(srow + e * 32 + 16);
+                uint4 pk;
+                pk.x = pack_bf16x2(fmaf(a[8 * e + 0], rq, c0.x), fmaf(a[8 * e + 1], rq, c0.y));
+                pk.y = pack_bf16x2(fmaf(a[8 * e + 2], rq, c0.z), fmaf(a[8 * e + 3], rq, c0.w));
+                pk.z = pack_bf16x2(fmaf(a[8 * e + 4], rq, c1.x), fmaf(a[8 * e + 5], rq, c1.y));
+                pk.w = pack_bf16x2(fmaf(a[8 * e + 6], rq, c1.z), fmaf(a[8 * e + 7], rq, c1.w));
+                *reinterpret_cast<uint4*>(orow + (((half * 4 + e) ^ (row & 7)) << 4)) = pk;
+            }
+            tcgen05_fence_before_sync();
+            mbar_arrive(&buf_free[b]);
+            fence_proxy_async_smem();
+            named_barrier_sync(1, kEpiThreads);
+            if (leader) {
+                const int y0 = (wk.rem / prm.tilesX) * kTY, x0 = (wk.rem % prm.tilesX) * kTX;
+                if (prm.flat) {
+                    tma_store_4d_hint(&tmO, out_s, 0, x0, y0, wk.bh, pol_o);
+                } else {
+                    const int pb = wk.bh / prm.hdiv;
+                    tma_store_5d_hint(&tmO, out_s, 0, x0, y0, wk.bh - pb * prm.hdiv, pb, pol_o);
+                }
+                tma_store_commit();
+            }
         }
+        if (leader) tma_store_wait_all();
     } else if (warp < kFirstWarpConv) {
-        // ================= state pipeline: K normalisation, accumulator read-out, split reduction =================
+        // ================= state pipeline: K normalisation, accumulator read-out =================
         const int t = tid - 32 * kFirstWarpNorm;   // 0..127: row t >> 1 of the stage, half t & 1 of that row
         const int quarter = warp & 3;
         const int r = t >> 1, hf = t & 1;
         bool ok = true;
-        // read the finished accumulator of the k-th item of this CTA out of TMEM: rows 0..63 are S, row 64 is s
-        auto flush = [&](int k_item, float* dst) -> bool {
-            const int buf = k_item & 1;
-            if (!mbar_wait(&sacc_full[buf], (k_item >> 1) & 1, abort_flag, prm.status, kBit)) return false;
-            tcgen05_fence_after_sync();
-            if (quarter < 3) {
-                const int row = quarter * 32 + lane;
-#pragma unroll
-                for (int cc = 0; cc < kD / 16; ++cc) {
-                    float v[16];
-                    tmem_ld16(tmem_state + ((uint32_t)(quarter * 32) << 16) + buf * kD + cc * 16, v);
-                    tmem_ld_wait();
-                    if (row <= kD) {
-                        float4* o4 = reinterpret_cast<float4*>(dst + row * kD + cc * 16);  // row 64 lands on s
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) o4[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-                    }
-                }
-            }
-            tcgen05_fence_before_sync();
-            mbar_arrive(&sacc_free[buf]);
-            return true;
-        };
-        // After an item's partial state is in memory: count it; the last split of a group sums the group, the
-        // last group sums the groups (both in index order: the result does not depend on who came last), writes
-        // the plane's state and raises its flag.  With one split per plane the state is already final.
-        auto publish = [&](int item) {
-            const int plane = item / prm.P, part = item - plane * prm.P;
-            unsigned* pc = plane_ctr + (size_t)plane * kPipeCtrPerPlane;
-            __threadfence();
-            named_barrier_sync(2, kNormThreads);
-            if (prm.P > 1) {
-                const int n_groups = (prm.P + kGroup - 1) / kGroup, grp = part / kGroup;
-                const int first = grp * kGroup, members = min(kGroup, prm.P - first);
-                float* base = prm.partial + (size_t)plane * prm.P * kWords;
-                if (t == 0) *last_slot = (atomicAdd(&pc[grp], 1u) == (unsigned)(members - 1));
-                named_barrier_sync(2, kNormThreads);
-                const bool last_in_group = *last_slot != 0;
-                named_barrier_sync(2, kNormThreads);
-                if (!last_in_group) return;
-                __threadfence();
-                if (members > 1) sum_states(base + (size_t)first * kWords, kWords, members, base + (size_t)first * kWords, t);
-                __threadfence();
-                named_barrier_sync(2, kNormThreads);
-                if (t == 0) { pc[grp] = 0; *last_slot = (atomicAdd(&pc[kPipeCtrGroups], 1u) == (unsigned)(n_groups - 1)); }
-                named_barrier_sync(2, kNormThreads);
-                const bool last_group = *last_slot != 0;
-                named_barrier_sync(2, kNormThreads);
-                if (!last_group) return;
-                __threadfence();
-                sum_states(base, (size_t)kGroup * kWords, n_groups, prm.state + (size_t)plane * kWords, t);
-                __threadfence();
-                named_barrier_sync(2, kNormThreads);
-                if (t == 0) pc[kPipeCtrGroups] = 0;
-            }
-            if (t == 0) {
-                __threadfence();
-                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(pc + kPipeCtrReady), "r"(1u) : "memory");
-            }
-        };
-        auto item_dst = [&](int item) -> float* {
-            return prm.P > 1 ? prm.partial + (size_t)item * kWords : prm.state + (size_t)item * kWords;  // item = plane * P + part
-        };
-        int gt = 0, k_item = 0, prev_item = -1;
-        bool dead = false;  // some thread of the group gave up: everybody leaves (decided at a barrier, so together)
-        for (int item = cta; item < n_items; item += n_cta, ++k_item) {
-            const int plane = item / prm.P, part = item - plane * prm.P;
-            const int t0 = part * prm.s_per, t1 = min(prm.s_tiles, t0 + prm.s_per);
-            for (int tt = t0; tt < t1 && ok; ++tt, ++gt) {
+        int gt = 0;
+        for (int plane = 0; plane < prm.BH; ++plane) {
+            for (int tt = t_begin; tt < t_end && ok; ++tt, ++gt) {
                 const int s = gt % NS, use = gt / NS;
                 ok = mbar_wait(&s_full[s], use & 1, abort_flag, prm.status, kBit);
                 if (!ok) break;
@@ -561,38 +543,57 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 fence_proxy_async_smem();
                 mbar_arrive(&s_scaled[s]);
             }
-            // the previous item is read out one item late, so that its UMMAs overlap this item's normalisation
-            if (prev_item >= 0 && ok) ok = flush(k_item - 1, item_dst(prev_item));
-            if (barrier_any(3, kNormThreads, !ok)) { dead = true; break; }
-            if (prev_item >= 0) publish(prev_item);
-            prev_item = item;
-        }
-        if (!dead && prev_item >= 0) {
-            ok = flush(k_item - 1, item_dst(prev_item));
-            if (!barrier_any(3, kNormThreads, !ok)) publish(prev_item);
+            // this CTA's sums over its rows of the plane leave TMEM: rows 0..63 are S, row 64 is s
+            const int buf = plane & 1;
+            if (ok) ok = mbar_wait(&sacc_full[buf], (plane >> 1) & 1, abort_flag, prm.status, kBit);
+            if (ok) {
+                tcgen05_fence_after_sync();
+                float* dst = prm.partial + ((size_t)(plane % prm.ring) * n_cta + cta) * kWords;
+                if (quarter < 3) {
+                    const int row = quarter * 32 + lane;
+#pragma unroll
+                    for (int cc = 0; cc < kD / 16; ++cc) {
+                        float v[16];
+                        tmem_ld16(tmem_state + ((uint32_t)(quarter * 32) << 16) + buf * kD + cc * 16, v);
+                        tmem_ld_wait();
+                        if (row <= kD) {
+                            float4* o4 = reinterpret_cast<float4*>(dst + row * kD + cc * 16);  // row 64 lands on s
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) o4[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                        }
+                    }
+                }
+                tcgen05_fence_before_sync();
+                mbar_arrive(&sacc_free[buf]);
+            }
+            if (barrier_any(3, kNormThreads, !ok)) break;
+            if (t == 0) signal_add(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrWritten);
         }
     } else {
-        // ================= apply pipeline: depthwise convolution + combine + store =================
+        // ================= apply pipeline: depthwise convolution =================
         const int cwi = warp - kFirstWarpConv;
         const int cw = cwi >> 1, xh = cwi & 1;  // row group and column half of the patch
         constexpr int kCX = kTX / 2;
-        constexpr int R = G::R, RO = G::kConvRows, ROWS = RO + 2 * R, HOLD = G::kHold;
+        constexpr int R = G::R, RO = G::kConvRows, ROWS = RO + 2 * R;
         float2 wreg[KS][KS];
         float2 cinit = make_float2(0.f, 0.f);
-        int prev_bh = -1;
-        const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
-        const long long row_stride = PAIR ? kD : prm.lo.token;  // elements between 128-byte rows of the output
+        int prev_bh = -1, pseg = 0;
+        // When this CTA's share of a plane is done, the conv warp that gets there last says so (once per CTA
+        // and plane: the state pipelines poll that counter, and per-patch arrivals from every warp of every CTA
+        // would queue up on its one address).  Warps are at most a few patches apart, far less than 8 planes.
+        auto plane_done = [&](int plane) {
+            if (lane == 0 && (atomicAdd(&applied_s[plane & 7], 1u) % G::kConvWarps) == G::kConvWarps - 1)
+                atomicAdd(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrApplied, 1u);
+        };
         PatchWalk wk; wk.init(prm);
         for (int it = 0; wk.valid(); ++it, wk.step()) {
             const int s = it % NA, use = it / NA, b = it & 1, ub = it >> 1;
-            const int sb = (G::kStgBufs == 2) ? b : 0, su = (G::kStgBufs == 2) ? ub : it;
             const int bh = wk.bh;
             if (bh != prev_bh) {
+                if (prev_bh >= 0) plane_done(prev_bh);
                 prev_bh = bh;
-                bool ready = true;
-                if (lane == 0)
-                    ready = wait_counter(plane_ctr + (size_t)bh * kPipeCtrPerPlane + kPipeCtrReady, 1u, abort_flag, prm.status);
-                if (!__shfl_sync(0xffffffffu, (int)ready, 0)) break;
+                if (__any_sync(0xffffffffu, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit))) break;
+                ++pseg;
                 // this lane's channel pair: 2*lane of 64 channels, or (PAIR) 2*(lane & 15) of 32 channels
                 // for the token of parity lane >> 4
                 const int cp2 = PAIR ? 2 * (lane & 15) : 2 * lane;
@@ -615,6 +616,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                                                    __bfloat162float(prm.w[(size_t)(ch + 1) * KS * KS + dy * KS + dx]));
             }
             if (__any_sync(0xffffffffu, !mbar_wait(&a_full[s], use & 1, abort_flag, prm.status, kBit))) break;
+            if (ub > 0 && __any_sync(0xffffffffu, !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit))) break;
             // Window of KS tokens per halo row, sliding along x.  Token t (relative to the first token this
             // lane needs) sits U bytes after token t-1: U = 128, one token per column, or (PAIR) 64.
             // One output column advances the window by STEP tokens (2 when PAIR: the lane's token keeps
@@ -623,18 +625,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             const int tok0 = PAIR ? 2 * (xh * kCX + G::HC) + (lane >> 4) - R : xh * kCX;
             const uint8_t* vh = stages + s * G::kStage + kQBytes + (RO * cw) * G::HX * 128 + tok0 * U +
                                 (PAIR ? (lane & 15) * 4 : lane * 4);
-            const int y0 = (wk.rem / prm.tilesX) * kTY + RO * cw, x0 = (wk.rem % prm.tilesX) * kTX + xh * kCX;
-            // lane's 32-bit word of the output row of patch token (RO*cw, xh*kCX)
-            uint32_t* orow = reinterpret_cast<uint32_t*>(prm.out + plane_offset(prm.lo, bh, prm.hdiv) +
-                                                         ((long long)y0 * prm.cols + x0) * row_stride) + lane;
-            const uint8_t* srow = stg + sb * kStgBytes + ((RO * cw) * kTX + xh * kCX) * kStgRow + (lane & 1) * 8;
-            const int sc = lane >> 1;
-            auto combine = [&](int r, int x, float2 acc) {
-                const int t = (RO * cw + r) * kTX + xh * kCX + x;
-                const float2 a2 = *reinterpret_cast<const float2*>(srow + (r * kTX + x) * kStgRow + ((sc ^ (t & 7)) << 4));
-                if (y0 + r < prm.gridH && x0 + x < prm.cols)
-                    st_global_hint(orow + ((long long)r * prm.cols + x) * (row_stride / 2), pack_bf16x2(a2.x + acc.x, a2.y + acc.y), pol_o);
-            };
+            uint8_t* so = stg + b * kStgBytes + ((RO * cw) * kTX + xh * kCX) * kStgStride + lane * 8;
             float2 win[ROWS][KS];
 #pragma unroll
             for (int t = 0; t < KS - STEP; ++t)
@@ -643,8 +634,6 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     const uint32_t wv = *reinterpret_cast<const uint32_t*>(vh + r * G::HX * 128 + t * U);
                     win[r][t % KS] = make_float2(bf16lo(wv), bf16hi(wv));
                 }
-            float2 held[HOLD > 0 ? HOLD : 1][RO];
-            bool ok = true;
 #pragma unroll
             for (int x = 0; x < kCX; ++x) {
 #pragma unroll
@@ -666,35 +655,18 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 #pragma unroll
                         for (int r = 0; r < RO; ++r)
                             acc[r] = ffma2(wreg[dy][dx], win[dy + r][(STEP * x + dx) % KS], acc[r]);
-                if (x < HOLD) {
 #pragma unroll
-                    for (int r = 0; r < RO; ++r) held[x][r] = acc[r];
-                } else {
-                    if (x == HOLD) {  // the scaled accumulator rows of this patch are in the staging buffer
-                        ok = !__any_sync(0xffffffffu, !mbar_wait(&stg_full[sb], su & 1, abort_flag, prm.status, kBit));
-                        if (ok) {
-#pragma unroll
-                            for (int xx = 0; xx < HOLD; ++xx)
-#pragma unroll
-                                for (int r = 0; r < RO; ++r) combine(r, xx, held[xx][r]);
-                        }
-                    }
-                    if (ok) {
-#pragma unroll
-                        for (int r = 0; r < RO; ++r) combine(r, x, acc[r]);
-                    }
-                }
+                for (int r = 0; r < RO; ++r) *reinterpret_cast<float2*>(so + (r * kTX + x) * kStgStride) = acc[r];
             }
-            if (!ok) break;
             mbar_arrive(&a_empty[s]);      // the V patch of this stage is no longer needed
-            mbar_arrive(&stg_free[sb]);    // nor the staging buffer
-            if (lane == 0) atomicAdd(plane_ctr + (size_t)bh * kPipeCtrPerPlane + kPipeCtrApplied, 1u);
+            mbar_arrive(&conv_full[b]);
         }
+        if (prev_bh >= 0 && !*abort_flag) plane_done(prev_bh);
     }
     tcgen05_fence_before_sync();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-    // The CTA that leaves last puts the per-plane flags and counters back to zero for the next call.
+    // The CTA that leaves last puts the per-plane counters back to zero for the next call.
     if (tid == 0) {
         __threadfence();
         *last_slot = (atomicAdd(prm.ctr, 1u) == (unsigned)(n_cta - 1));
@@ -702,10 +674,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     __syncthreads();
     if (*last_slot) {
         __threadfence();
-        for (int i = tid; i < prm.BH; i += blockDim.x) {
-            plane_ctr[(size_t)i * kPipeCtrPerPlane + kPipeCtrReady] = 0;
-            plane_ctr[(size_t)i * kPipeCtrPerPlane + kPipeCtrApplied] = 0;
-        }
+        for (int i = tid; i < prm.BH * kPipeCtrPerPlane; i += blockDim.x) plane_ctr[i] = 0;
         if (tid == 0) prm.ctr[0] = 0;
     }
 }
@@ -717,8 +686,10 @@ cudaError_t launch_pipe_ks(const Problem& p, float* partial, float* state, unsig
     const bool pair = PAIR;
     const int rows = pair ? p.N / 2 : p.N;            // 128-byte rows per plane (leading off-grid tokens included)
     const int cols = pair ? p.gridW / 2 : p.gridW;    // 128-byte columns per grid row
+    const PipePlan plan = plan_pipe(p.BH, rows, cols, p.gridH);
+    if (!plan.ok) return cudaErrorNotSupported;
     const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
-    CUtensorMap tmK, tmVs, tmQ, tmVh;
+    CUtensorMap tmK, tmVs, tmQ, tmVh, tmO;
     {   // state: [64, rows, planes per batch step, batch steps]
         const uint64_t dims[4] = {(uint64_t)kD, (uint64_t)rows, (uint64_t)p.hdiv, nb};
         const uint32_t box[4] = {kD, kSTile, 1, 1};
@@ -740,26 +711,23 @@ cudaError_t launch_pipe_ks(const Problem& p, float* partial, float* state, unsig
             s[2] = (uint64_t)l.head;
             s[3] = (uint64_t)(nb > 1 ? l.batch : l.head * p.hdiv);
         };
-        uint64_t sq[4], sv[4];
-        strides(p.lq, sq); strides(p.lv, sv);
+        uint64_t sq[4], sv[4], so[4];
+        strides(p.lq, sq); strides(p.lv, sv); strides(p.lo, so);
         const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + p.prefix * p.lq.token;
         const __nv_bfloat16* vg = static_cast<const __nv_bfloat16*>(p.v) + p.prefix * p.lv.token;
-        if (!make_tensor_map_bf16(&tmQ, qg, rank, dims, sq, box, true) || !make_tensor_map_bf16(&tmVh, vg, rank, dims, sv, boxv, false))
+        __nv_bfloat16* og = static_cast<__nv_bfloat16*>(p.out) + p.prefix * p.lo.token;
+        if (!make_tensor_map_bf16(&tmQ, qg, rank, dims, sq, box, true) || !make_tensor_map_bf16(&tmVh, vg, rank, dims, sv, boxv, false) ||
+            !make_tensor_map_bf16(&tmO, og, rank, dims, so, box, true))
             return cudaErrorNotSupported;
     }
     PipeParams prm;
     prm.partial = partial; prm.state = state; prm.ctr = ctr;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
-    prm.out = static_cast<__nv_bfloat16*>(p.out) + p.prefix * p.lo.token;
-    prm.lo = p.lo;
     prm.flat = (rank == 4) ? 1 : 0;
     prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
-    prm.gridH = p.gridH; prm.cols = cols;
-    const PipePlan plan = plan_pipe(p.BH, rows, cols, p.gridH);
-    prm.s_tiles = plan.s_tiles; prm.s_per = plan.s_per; prm.P = plan.P;
-    prm.plane_order = plan.plane_order; prm.ahead = plan.ahead;
+    prm.s_tiles = plan.s_tiles; prm.ahead = plan.ahead; prm.ring = plan.ring;
     prm.eps2 = p.eps2; prm.status = status;
     static PerDevice opt_in;  // one per instantiation
     {
@@ -773,40 +741,44 @@ cudaError_t launch_pipe_ks(const Problem& p, float* partial, float* state, unsig
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc_pipe_kernel<KS, MODE>, tmK, tmVs, tmQ, tmVh, prm);
+    return cudaLaunchKernelEx(&cfg, tc_pipe_kernel<KS, MODE>, tmK, tmVs, tmQ, tmVh, tmO, prm);
+}
+
+// Planes that the state pipeline may be ahead of the apply pipeline: as many as keep the V rows read and not
+// yet applied within a part of L2 that the other streams leave alone.
+int planes_ahead(int BH, int rows) {
+    const long long budget = 40ll << 20;
+    long long ahead = budget / ((long long)(rows < 1 ? 1 : rows) * 128);
+    if (ahead < 1) ahead = 1;
+    return (int)(ahead < BH ? ahead : BH);
 }
 
 }  // namespace
 
-// Work split of the one-kernel forward: CTAs, state tiles per plane, token splits per plane, and whether the
-// planes are applied in order with the state pipeline running a bounded number of planes ahead.
+// Work split of the one-kernel forward.  It takes planes with at least two thirds as many patches as there are
+// multiprocessors (every CTA gets a share of every plane); shorter planes go to the separate kernels.
 PipePlan plan_pipe(int BH, int rows, int cols, int gridH) {
-    PipePlan pl;
+    PipePlan pl = {};
     const int sms = device_sm_count();
-    if (rows < 1) rows = 1;  // size queries reach here with shapes the kernel never takes
-    if (BH < 1) BH = 1;
+    if (rows < 1 || BH < 1 || cols < 1 || gridH < 1) return pl;
     pl.s_tiles = (rows + kSTile - 1) / kSTile;
     const int patches = ((cols + kTX - 1) / kTX) * ((gridH + kTY - 1) / kTY);
-    // splits: about eight tiles each, but at least enough to give every CTA a share when there are few planes
-    int P = pl.s_tiles / 8;
-    const int spread = sms / BH;
-    if (P < spread) P = spread;
-    if (P > pl.s_tiles) P = pl.s_tiles;
-    if (P > kPipeMaxSplits) P = kPipeMaxSplits;
-    if (P < 1) P = 1;
-    pl.s_per = (pl.s_tiles + P - 1) / P;
-    pl.P = (pl.s_tiles + pl.s_per - 1) / pl.s_per;
-    const long long items = (long long)BH * pl.P, total_patches = (long long)BH * patches;
-    long long want = items > total_patches ? items : total_patches;
-    pl.grid = (int)(want < sms ? want : sms);
-    // V of all planes beyond what L2 can hold until it is applied: walk the planes in order
-    const long long v_bytes = (long long)BH * rows * 128;
-    const long long budget = 40ll << 20;
-    pl.plane_order = (v_bytes > budget && patches >= pl.grid) ? 1 : 0;
-    long long ahead = budget / ((long long)rows * 128);
-    if (ahead < 1) ahead = 1;
-    pl.ahead = pl.plane_order ? (int)(ahead < BH ? ahead : BH) : BH;
+    pl.grid = patches < sms ? patches : sms;
+    pl.ahead = planes_ahead(BH, rows);
+    pl.ring = pl.ahead;  // plane p + ring starts after plane p + ring - ahead >= p is applied, so plane p's sums are used up
+    pl.ok = (3 * patches >= 2 * sms) && pl.s_tiles >= pl.grid;
     return pl;
+}
+
+// Per-CTA sums that the workspace has to hold for any grid of `rows` 128-byte rows per plane.
+size_t pipe_partial_slots(int BH, int rows) {
+    if (rows < 1 || BH < 1) return 0;
+    return (size_t)planes_ahead(BH, rows) * device_sm_count();
+}
+
+bool pipe_supports(const Problem& p) {
+    const bool pair = (p.d == 32);
+    return plan_pipe(p.BH, pair ? p.N / 2 : p.N, pair ? p.gridW / 2 : p.gridW, p.gridH).ok;
 }
 
 cudaError_t launch_pipe(const Problem& p, float* partial, float* state, unsigned* ctr, unsigned* status, cudaStream_t st) {
