@@ -51,26 +51,29 @@ cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned
 // Output rows of the off-grid leading tokens (p.prefix of them per plane), from the final state.
 cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_t st);
 
-// One-kernel forward for long sequences (csrc/tc_pipe.cu): a state pipeline and an apply pipeline share every
-// CTA; the CTAs signal one another through counters in global memory.
-// Counter layout: kPipeCtrHeader words (word 0 counts the CTAs that have left), then kPipeCtrPerPlane words per
-// plane: CTAs whose sums over their rows of the plane are written, CTAs whose slice of the total is written,
-// CTAs that have applied their share of the plane.  All zero between calls.
+// One-kernel forward (csrc/tc_pipe.cu): a state pipeline and an apply pipeline share every CTA; work is handed
+// out, and progress is signalled, through counters in global memory.
+// Counter layout: kPipeCtrHeader words (CTAs that have left, next patch to hand out, next chunk of rows to hand
+// out), then kPipeCtrPerPlane words per plane: chunks whose sums are written, summation slices handed out, slices
+// added, patches applied.  All zero between calls.
 constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 4;
-constexpr int kPipeCtrWritten = 0, kPipeCtrSummed = 1, kPipeCtrApplied = 2;
+constexpr int kPipeCtrNextPatch = 1, kPipeCtrNextChunk = 2;
+constexpr int kPipeCtrWritten = 0, kPipeCtrClaimed = 1, kPipeCtrSummed = 2, kPipeCtrApplied = 3;
 struct PipePlan {
     bool ok;           // the one-kernel forward takes this shape
     int grid;          // CTAs (at most one per multiprocessor)
     int s_tiles;       // 64-row state tiles per plane
+    int chunk_tiles;   // tiles per chunk of rows (one partial sum per chunk)
+    int n_chunks;      // chunks per plane
     int ahead;         // planes the state pipeline may run ahead of the apply pipeline
-    int ring;          // planes whose per-CTA sums are kept at a time
+    int ring;          // planes whose chunk sums are kept at a time
 };
 // rows: 128-byte rows per plane (leading tokens included); cols x gridH: the token grid in 128-byte columns.
 PipePlan plan_pipe(int BH, int rows, int cols, int gridH);
 bool pipe_supports(const Problem& p);
-// Per-CTA sums (of kStateWords each) the workspace must hold behind the final states for such planes.
+// Chunk sums (of kStateWords each) the workspace must hold behind the final states for such planes.
 size_t pipe_partial_slots(int BH, int rows);
-// Per-CTA sums live at partial[plane % ring][cta], final ones at state[plane]; ctr as described above.
+// Chunk sums live at partial[plane % ring][chunk], final ones at state[plane]; ctr as described above.
 cudaError_t launch_pipe(const Problem& p, float* partial, float* state, unsigned* ctr, unsigned* status, cudaStream_t st);
 
 // Single-kernel forward for short sequences (bf16, 3x3 or 5x5 filters, at most 256 128-byte rows per plane:

@@ -72,7 +72,7 @@ template <int KS, bool PAIR> struct PGeo {
 };
 
 struct PipeParams {
-    float* partial;                // [ring][CTA][kWords] sums of one CTA over its rows of one plane
+    float* partial;                // [ring][chunk][kWords] sums over one chunk of rows of one plane
     float* state;                  // [BH][kWords] final sums
     unsigned* ctr;                 // kPipeCtrHeader words, then kPipeCtrPerPlane per plane; all zero between calls
     const __nv_bfloat16* w;        // [H*d][KS][KS]
@@ -81,29 +81,16 @@ struct PipeParams {
     int H, head0, BH, hdiv;
     int tilesX, tilesY;            // patches per plane
     int s_tiles;                   // 64-row state tiles per plane
-    int ahead;                     // the state pipeline starts plane p only when plane p - ahead is applied
+    int chunk_tiles, n_chunks;     // tiles per chunk, chunks per plane
+    int ahead;                     // a chunk of plane p is started only when plane p - ahead is applied
     int ring;                      // plane slots of `partial`: plane p uses slot p % ring
     float eps2;
     unsigned* status;
 };
 
-// This CTA's patches, in the order every role of the apply pipeline visits them: plane after plane, a
-// contiguous share of each plane's patches.  Every CTA has at least one patch in every plane.
-struct PatchWalk {
-    int bh, rem, end, tpb, G, cta, BH;
-    __device__ void init(const PipeParams& prm) {
-        tpb = prm.tilesX * prm.tilesY; G = (int)gridDim.x; cta = (int)blockIdx.x; BH = prm.BH;
-        bh = -1; rem = end = 0;
-        next_plane();
-    }
-    __device__ void next_plane() {
-        if (++bh >= BH) return;
-        const int cc = (cta + 37 * bh) % G;  // the larger shares rotate over the CTAs from plane to plane
-        rem = (int)((long long)tpb * cc / G); end = (int)((long long)tpb * (cc + 1) / G);
-    }
-    __device__ bool valid() const { return bh < BH; }
-    __device__ void step() { if (++rem == end) next_plane(); }
-};
+constexpr int kNoWork = -1;            // stage info: nothing more to do
+constexpr int kSliceWords4 = kEpiWarps;  // float4 positions of a summation slice: one per epilogue warp
+constexpr int kSlices = (kWords4 + kSliceWords4 - 1) / kSliceWords4;
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
@@ -180,13 +167,16 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* last_slot = reinterpret_cast<int*>(tmem_slot + 2);
     volatile int* sum_go = reinterpret_cast<volatile int*>(tmem_slot + 3);  // the polling thread's verdict on a slice sum
-    unsigned* applied_s = reinterpret_cast<unsigned*>(tmem_slot + 4);  // [8] conv warps done with plane p, slot p & 7
+    unsigned* applied_s = reinterpret_cast<unsigned*>(tmem_slot + 4);  // [8] conv warps done with the CTA's i-th patch, slot i & 7
+    volatile int* a_info = reinterpret_cast<volatile int*>(tmem_slot + 12);  // [NA] patch in the apply stage, or kNoWork
+    volatile int* s_info = a_info + 4;                                      // [NS] chunk * 4 + (first tile) + 2 * (last tile), or kNoWork
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_cta = (int)gridDim.x, cta = (int)blockIdx.x;
     unsigned* plane_ctr = prm.ctr + kPipeCtrHeader;
-    // this CTA's rows of every plane, as a range of 64-row tiles (never empty: the launcher sees to it)
-    const int t_begin = (int)((long long)prm.s_tiles * cta / n_cta), t_end = (int)((long long)prm.s_tiles * (cta + 1) / n_cta);
+    const int tpb = prm.tilesX * prm.tilesY;                 // patches per plane
+    const int n_patches = prm.BH * tpb, n_chunks_all = prm.BH * prm.n_chunks;
+    (void)cta;
 
     if (tid == 0) {
         for (int s = 0; s < NA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], G::kConvThreads + kEpiThreads + 1); }
@@ -222,22 +212,33 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (lane == 0) {
             int issued = 0;
             const uint64_t pol_q = l2_policy_evict_first();  // Q is read once
-            PatchWalk wk; wk.init(prm);
-            for (int it = 0; wk.valid(); ++it, wk.step()) {
+            // Patches are handed out one at a time, in plane order, from a counter in global memory: a slower
+            // multiprocessor simply takes fewer.  The next claim is under way while this patch is loaded.
+            int g = (int)atomicAdd(prm.ctr + kPipeCtrNextPatch, 1u);
+            for (int it = 0;; ++it) {
                 const int s = it % NA, use = it / NA;
                 if (use > 0 && !mbar_wait(&a_empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) break;
-                const int y0 = (wk.rem / prm.tilesX) * kTY, x0 = (wk.rem % prm.tilesX) * kTX;
+                if (g >= n_patches) {  // tell the other roles that this was all
+                    a_info[s] = kNoWork;
+                    mbar_arrive(&a_full[s]);
+                    break;
+                }
+                const int g_next = (int)atomicAdd(prm.ctr + kPipeCtrNextPatch, 1u);
+                const int bh = g / tpb, rem = g - bh * tpb;
+                const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
                 uint8_t* qs = stages + s * G::kStage;
+                a_info[s] = g;
                 mbar_expect_tx(&a_full[s], kQBytes + G::kVBytes);
                 if (prm.flat) {
-                    tma_load_4d_hint(qs, &tmQ, &a_full[s], 0, x0, y0, wk.bh, pol_q);
-                    tma_load_4d(qs + kQBytes, &tmVh, &a_full[s], 0, x0 - G::HC, y0 - G::R, wk.bh);
+                    tma_load_4d_hint(qs, &tmQ, &a_full[s], 0, x0, y0, bh, pol_q);
+                    tma_load_4d(qs + kQBytes, &tmVh, &a_full[s], 0, x0 - G::HC, y0 - G::R, bh);
                 } else {
-                    const int pb = wk.bh / prm.hdiv, ph = wk.bh - pb * prm.hdiv;
+                    const int pb = bh / prm.hdiv, ph = bh - pb * prm.hdiv;
                     tma_load_5d_hint(qs, &tmQ, &a_full[s], 0, x0, y0, ph, pb, pol_q);
                     tma_load_5d(qs + kQBytes, &tmVh, &a_full[s], 0, x0 - G::HC, y0 - G::R, ph, pb);
                 }
                 ++issued;
+                g = g_next;
             }
             if (*abort_flag) {  // giving up: let copies already in flight land before shared memory goes away
                 for (int i = max(0, issued - NA); i < issued; ++i)
@@ -250,14 +251,16 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             constexpr uint32_t idesc = umma_idesc_bf16(128, kD, false, true);
             const uint32_t s_addr = smem_u32(S_s);
             int prev_bh = -1, seg = 0;
-            PatchWalk wk; wk.init(prm);
-            for (int it = 0; wk.valid(); ++it, wk.step()) {
+            for (int it = 0;; ++it) {
                 const int s = it % NA, use = it / NA, b = it & 1, ub = it >> 1;
-                if (wk.bh != prev_bh) {
-                    if (!mbar_wait(s_ready, seg & 1, abort_flag, prm.status, kBit)) break;
-                    ++seg; prev_bh = wk.bh;
-                }
                 if (!mbar_wait(&a_full[s], use & 1, abort_flag, prm.status, kBit)) break;
+                const int g = a_info[s];
+                if (g == kNoWork) break;
+                const int bh = g / tpb;
+                if (bh != prev_bh) {
+                    if (!mbar_wait(s_ready, seg & 1, abort_flag, prm.status, kBit)) break;
+                    ++seg; prev_bh = bh;
+                }
                 if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
                 tcgen05_fence_after_sync();
                 const uint32_t q_addr = smem_u32(stages + s * G::kStage);
@@ -278,19 +281,33 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             // K is read once; V is read again by the apply pipeline: keep it in L2 as long as possible
             const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_last();
             bool ok = true;
-            for (int plane = 0; plane < prm.BH && ok; ++plane) {
+            // Chunks of rows are handed out like the patches, in plane order.
+            int g = (int)atomicAdd(prm.ctr + kPipeCtrNextChunk, 1u);
+            while (ok) {
+                if (g >= n_chunks_all) {
+                    const int s = issued % NS, use = issued / NS;
+                    if (use > 0 && !mbar_wait(&s_empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) break;
+                    s_info[s] = kNoWork;
+                    mbar_arrive(&s_full[s]);
+                    break;
+                }
+                const int g_next = (int)atomicAdd(prm.ctr + kPipeCtrNextChunk, 1u);
+                const int plane = g / prm.n_chunks, j = g - plane * prm.n_chunks;
                 if (plane >= prm.ahead &&
-                    !wait_counter(plane_ctr + (size_t)(plane - prm.ahead) * kPipeCtrPerPlane + kPipeCtrApplied, (unsigned)n_cta,
+                    !wait_counter(plane_ctr + (size_t)(plane - prm.ahead) * kPipeCtrPerPlane + kPipeCtrApplied, (unsigned)tpb,
                                   abort_flag, prm.status)) break;
                 const int pb = plane / prm.hdiv, ph = plane - pb * prm.hdiv;
-                for (int t = t_begin; t < t_end; ++t, ++issued) {
+                const int t0 = j * prm.chunk_tiles, t1 = min(prm.s_tiles, t0 + prm.chunk_tiles);
+                for (int t = t0; t < t1; ++t, ++issued) {
                     const int s = issued % NS, use = issued / NS;
                     if (use > 0 && !mbar_wait(&s_empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) { ok = false; break; }
                     uint8_t* ks = sstages + s * kSStage;
+                    s_info[s] = g * 4 + (t == t0 ? 1 : 0) + (t == t1 - 1 ? 2 : 0);
                     mbar_expect_tx(&s_full[s], kSStage);
                     tma_load_4d_hint(ks, &tmK, &s_full[s], 0, t * kSTile, ph, pb, pol_k);
                     tma_load_4d_hint(ks + kSTileBytes, &tmVs, &s_full[s], 0, t * kSTile, ph, pb, pol_v);
                 }
+                g = g_next;
             }
             if (*abort_flag) {
                 for (int i = max(0, issued - NS); i < issued; ++i)
@@ -302,26 +319,26 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, kD, true, true);
             const uint32_t ones_addr = smem_u32(ones);
-            bool ok = true;
-            int gt = 0;  // tiles issued so far
-            for (int plane = 0; plane < prm.BH && ok; ++plane) {
-                const int buf = plane & 1;
-                if (plane >= 2) ok = mbar_wait(&sacc_free[buf], ((plane >> 1) - 1) & 1, abort_flag, prm.status, kBit);
-                for (int t = t_begin; t < t_end && ok; ++t, ++gt) {
-                    const int s = gt % NS, use = gt / NS;
-                    ok = mbar_wait(&s_scaled[s], use & 1, abort_flag, prm.status, kBit);
-                    if (!ok) break;
-                    tcgen05_fence_after_sync();
-                    const uint32_t ka = smem_u32(sstages + s * kSStage), va = ka + kSTileBytes;
+            int k_chunk = 0;  // chunks started so far
+            for (int gt = 0;; ++gt) {
+                const int s = gt % NS, use = gt / NS;
+                if (!mbar_wait(&s_scaled[s], use & 1, abort_flag, prm.status, kBit)) break;
+                const int info = s_info[s];
+                if (info == kNoWork) break;
+                const bool first = (info & 1) != 0, last = (info & 2) != 0;
+                if (first) ++k_chunk;
+                const int buf = (k_chunk - 1) & 1;
+                if (first && k_chunk > 2 && !mbar_wait(&sacc_free[buf], (((k_chunk - 1) >> 1) - 1) & 1, abort_flag, prm.status, kBit)) break;
+                tcgen05_fence_after_sync();
+                const uint32_t ka = smem_u32(sstages + s * kSStage), va = ka + kSTileBytes;
 #pragma unroll
-                    for (int j = 0; j < kSTile / 16; ++j) {  // one UMMA per 16 rows (K = 16)
-                        const uint32_t a0 = ka + j * 2048, b0 = va + j * 2048;
-                        umma_bf16(tmem_state + buf * kD, umma_desc_sw128(a0, ones_addr - a0, 1024),
-                                  umma_desc_sw128(b0, 0, 1024), idesc, (t != t_begin) || (j != 0));
-                    }
-                    umma_commit(&s_empty[s]);
+                for (int j = 0; j < kSTile / 16; ++j) {  // one UMMA per 16 rows (K = 16)
+                    const uint32_t a0 = ka + j * 2048, b0 = va + j * 2048;
+                    umma_bf16(tmem_state + buf * kD, umma_desc_sw128(a0, ones_addr - a0, 1024),
+                              umma_desc_sw128(b0, 0, 1024), idesc, !first || (j != 0));
                 }
-                if (ok) umma_commit(&sacc_full[buf]);
+                umma_commit(&s_empty[s]);
+                if (last) umma_commit(&sacc_full[buf]);
             }
         }
     } else if (warp < kFirstWarpNorm) {
@@ -331,66 +348,78 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         const int half = ew >> 2;  // channels half*32 .. half*32 + 31
         const bool leader = (et == 0);
         const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
-        // this CTA's slice of the state words (as float4 positions), added over all CTAs' sums
-        const int q0 = (int)((long long)kWords4 * cta / n_cta), q1 = (int)((long long)kWords4 * (cta + 1) / n_cta);
-        // Adds the slice for `plane` once every CTA has written its sums of that plane.  Position by position,
-        // lane l of a warp adds the sums of CTAs l, l + 32, ... in that order and the 32 results meet in a fixed
-        // shuffle tree.  Returns 1 when done, 0 when the sums are not all there yet (only if !blocking), -1 after a
-        // failed wait.  All epilogue threads call it together and get the same answer.
-        auto slice_sum = [&](int plane, bool blocking) -> int {
+        // Adds up the chunk sums of `plane`, slice by slice, for as long as there are unclaimed slices (at most
+        // `max_claims` of them).  Slices are handed out from a counter; a slice is kEpiWarps float4 positions, one
+        // per warp: lane l adds the sums of chunks l, l + 32, ... in that order and the 32 results meet in a fixed
+        // shuffle tree, so the total does not depend on who added what when.  The chunk sums must all be written:
+        // with `blocking` the call waits for that, otherwise it returns at once when they are not.  Returns false
+        // after a failed wait.  All epilogue threads call it together and get the same answer.
+        auto sum_slices = [&](int plane, int max_claims, bool blocking) -> bool {
             unsigned* pc = plane_ctr + (size_t)plane * kPipeCtrPerPlane;
-            if (leader) {
-                int go;
-                if (blocking) go = wait_counter(&pc[kPipeCtrWritten], (unsigned)n_cta, abort_flag, prm.status) ? 1 : -1;
-                else go = (ld_acquire(&pc[kPipeCtrWritten]) >= (unsigned)n_cta) ? 1 : 0;
-                *sum_go = go;
-            }
-            named_barrier_sync(4, kEpiThreads);
-            const int go = *sum_go;
-            named_barrier_sync(4, kEpiThreads);  // everybody has read the verdict before the next one is written
-            if (go != 1) return go;
-            const float4* base = reinterpret_cast<const float4*>(prm.partial + (size_t)(plane % prm.ring) * n_cta * kWords);
+            const float4* base = reinterpret_cast<const float4*>(prm.partial + (size_t)(plane % prm.ring) * prm.n_chunks * kWords);
             float4* fin = reinterpret_cast<float4*>(prm.state + (size_t)plane * kWords);
-            for (int pos = q0 + ew; pos < q1; pos += kEpiWarps) {
-                float4 v[5];
-#pragma unroll
-                for (int j = 0; j < 5; ++j) {
-                    const int m = lane + 32 * j;
-                    v[j] = (m < n_cta) ? __ldcg(base + (size_t)m * kWords4 + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int claim = 0; claim < max_claims; ++claim) {
+                if (leader) {
+                    int go = kNoWork;  // slice to add, kNoWork: nothing (left) to do, -2: failed
+                    bool there = true;
+                    if (claim == 0) {
+                        if (blocking) { if (!wait_counter(&pc[kPipeCtrWritten], (unsigned)prm.n_chunks, abort_flag, prm.status)) { there = false; go = -2; } }
+                        else there = ld_acquire(&pc[kPipeCtrWritten]) >= (unsigned)prm.n_chunks;
+                    }
+                    if (there && ld_acquire(&pc[kPipeCtrClaimed]) < (unsigned)kSlices) {
+                        const unsigned c = atomicAdd(&pc[kPipeCtrClaimed], 1u);
+                        if (c < (unsigned)kSlices) go = (int)c;
+                    }
+                    *sum_go = go;
                 }
-                float4 acc = v[0];
+                named_barrier_sync(4, kEpiThreads);
+                const int go = *sum_go;
+                named_barrier_sync(4, kEpiThreads);  // everybody has read the verdict before the next one is written
+                if (go == -2) return false;
+                if (go == kNoWork) return true;
+                const int pos = go * kSliceWords4 + ew;
+                if (pos < kWords4) {
+                    float4 v[4];
 #pragma unroll
-                for (int j = 1; j < 5; ++j) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
-                for (int m = lane + 160; m < n_cta; m += 32) {
-                    const float4 u = __ldcg(base + (size_t)m * kWords4 + pos);
-                    acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
-                }
+                    for (int j = 0; j < 4; ++j) {
+                        const int m = lane + 32 * j;
+                        v[j] = (m < prm.n_chunks) ? __ldcg(base + (size_t)m * kWords4 + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    float4 acc = v[0];
 #pragma unroll
-                for (int sh = 16; sh >= 1; sh >>= 1) {
-                    acc.x += __shfl_xor_sync(0xffffffffu, acc.x, sh); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, sh);
-                    acc.z += __shfl_xor_sync(0xffffffffu, acc.z, sh); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, sh);
+                    for (int j = 1; j < 4; ++j) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
+                    for (int m = lane + 128; m < prm.n_chunks; m += 32) {
+                        const float4 u = __ldcg(base + (size_t)m * kWords4 + pos);
+                        acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
+                    }
+#pragma unroll
+                    for (int sh = 16; sh >= 1; sh >>= 1) {
+                        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, sh); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, sh);
+                        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, sh); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, sh);
+                    }
+                    if (lane == 0) fin[pos] = acc;
                 }
-                if (lane == 0) fin[pos] = acc;
+                named_barrier_sync(4, kEpiThreads);
+                if (leader) signal_add(&pc[kPipeCtrSummed]);
             }
-            named_barrier_sync(4, kEpiThreads);
-            if (leader) signal_add(&pc[kPipeCtrSummed]);
-            return 1;
+            return true;
         };
         int prev_bh = -1, pseg = 0;
-        int summed = 0;  // this CTA's slices of planes [0, summed) are added
         bool failed = false;  // the same for every epilogue thread wherever a barrier follows
-        PatchWalk wk; wk.init(prm);
-        for (int it = 0; wk.valid(); ++it, wk.step()) {
+        for (int it = 0;; ++it) {
             const int b = it & 1, ub = it >> 1, s = it % NA, use = it / NA;
-            if (wk.bh != prev_bh && !failed) {
-                const int p = wk.bh;
+            // every epilogue thread learns the stage's patch (or that there is none, or that a wait failed)
+            if (barrier_any(1, kEpiThreads, !mbar_wait(&a_full[s], use & 1, abort_flag, prm.status, kBit))) break;
+            const int g = a_info[s];
+            if (g == kNoWork) break;
+            const int bh = g / tpb, rem = g - bh * tpb;
+            if (bh != prev_bh) {
+                const int p = bh;
                 prev_bh = p;
-                if (summed <= p) {
-                    if (slice_sum(p, true) == 1) summed = p + 1; else failed = true;
-                }
+                // the plane's state is final when every slice of it has been added; help with that first
+                failed = !sum_slices(p, kSlices, true);
                 if (!failed) {
-                    // the plane's state is final when every CTA has added its slice
-                    if (leader && wait_counter(plane_ctr + (size_t)p * kPipeCtrPerPlane + kPipeCtrSummed, (unsigned)n_cta, abort_flag, prm.status))
+                    if (leader && wait_counter(plane_ctr + (size_t)p * kPipeCtrPerPlane + kPipeCtrSummed, (unsigned)kSlices, abort_flag, prm.status))
                         mbar_arrive(p_ready);
                     failed = barrier_any(4, kEpiThreads, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit));
                     ++pseg;
@@ -429,20 +458,14 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     }
                     fence_proxy_async_smem();
                     mbar_arrive(s_ready);
-                    // the next plane's slice, if its sums are there already: by the time anyone enters that plane,
-                    // every CTA has long since added its slice
-                    if (p + 1 < prm.BH && summed == p + 1) {
-                        const int r = slice_sum(p + 1, false);
-                        if (r == 1) summed = p + 2; else if (r < 0) failed = true;
-                    }
+                    // a slice or two of the next plane, if its chunk sums are there already: by the time anyone
+                    // gets to that plane, its state is final
+                    if (p + 1 < prm.BH) failed = !sum_slices(p + 1, 2, false);
                 }
             }
             float a[32];
             if (!failed) {
                 // this thread's half of sum(q^2) for its token; the other half comes from the partner warp
-                failed = __any_sync(0xffffffffu, !mbar_wait(&a_full[s], use & 1, abort_flag, prm.status, kBit));
-            }
-            if (!failed) {
                 const uint8_t* qrow = stages + s * G::kStage + row * 128;
                 float ss[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -493,12 +516,12 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             fence_proxy_async_smem();
             named_barrier_sync(1, kEpiThreads);
             if (leader) {
-                const int y0 = (wk.rem / prm.tilesX) * kTY, x0 = (wk.rem % prm.tilesX) * kTX;
+                const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
                 if (prm.flat) {
-                    tma_store_4d_hint(&tmO, out_s, 0, x0, y0, wk.bh, pol_o);
+                    tma_store_4d_hint(&tmO, out_s, 0, x0, y0, bh, pol_o);
                 } else {
-                    const int pb = wk.bh / prm.hdiv;
-                    tma_store_5d_hint(&tmO, out_s, 0, x0, y0, wk.bh - pb * prm.hdiv, pb, pol_o);
+                    const int pb = bh / prm.hdiv;
+                    tma_store_5d_hint(&tmO, out_s, 0, x0, y0, bh - pb * prm.hdiv, pb, pol_o);
                 }
                 tma_store_commit();
             }
@@ -509,13 +532,16 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         const int t = tid - 32 * kFirstWarpNorm;   // 0..127: row t >> 1 of the stage, half t & 1 of that row
         const int quarter = warp & 3;
         const int r = t >> 1, hf = t & 1;
-        bool ok = true;
-        int gt = 0;
-        for (int plane = 0; plane < prm.BH; ++plane) {
-            for (int tt = t_begin; tt < t_end && ok; ++tt, ++gt) {
-                const int s = gt % NS, use = gt / NS;
-                ok = mbar_wait(&s_full[s], use & 1, abort_flag, prm.status, kBit);
-                if (!ok) break;
+        int k_chunk = 0;  // chunks started so far
+        for (int gt = 0;; ++gt) {
+            const int s = gt % NS, use = gt / NS;
+            // every thread learns the stage's chunk (or that there is none, or that a wait failed)
+            if (barrier_any(3, kNormThreads, !mbar_wait(&s_full[s], use & 1, abort_flag, prm.status, kBit))) break;
+            const int info = s_info[s];
+            if (info == kNoWork) { mbar_arrive(&s_scaled[s]); break; }  // passes the word on to the UMMA issuer
+            const bool first = (info & 1) != 0, last = (info & 2) != 0;
+            if (first) ++k_chunk;
+            {
                 uint8_t* rowp = sstages + s * kSStage + r * 128;
                 uint4 c[4];
                 float ss = 0.f;
@@ -543,12 +569,14 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 fence_proxy_async_smem();
                 mbar_arrive(&s_scaled[s]);
             }
-            // this CTA's sums over its rows of the plane leave TMEM: rows 0..63 are S, row 64 is s
-            const int buf = plane & 1;
-            if (ok) ok = mbar_wait(&sacc_full[buf], (plane >> 1) & 1, abort_flag, prm.status, kBit);
+            if (!last) continue;
+            // the chunk's sums leave TMEM: rows 0..63 are S, row 64 is s
+            const int chunk = info >> 2, plane = chunk / prm.n_chunks, j_chunk = chunk - plane * prm.n_chunks;
+            const int buf = (k_chunk - 1) & 1;
+            const bool ok = mbar_wait(&sacc_full[buf], ((k_chunk - 1) >> 1) & 1, abort_flag, prm.status, kBit);
             if (ok) {
                 tcgen05_fence_after_sync();
-                float* dst = prm.partial + ((size_t)(plane % prm.ring) * n_cta + cta) * kWords;
+                float* dst = prm.partial + ((size_t)(plane % prm.ring) * prm.n_chunks + j_chunk) * kWords;
                 if (quarter < 3) {
                     const int row = quarter * 32 + lane;
 #pragma unroll
@@ -578,19 +606,13 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         float2 wreg[KS][KS];
         float2 cinit = make_float2(0.f, 0.f);
         int prev_bh = -1, pseg = 0;
-        // When this CTA's share of a plane is done, the conv warp that gets there last says so (once per CTA
-        // and plane: the state pipelines poll that counter, and per-patch arrivals from every warp of every CTA
-        // would queue up on its one address).  Warps are at most a few patches apart, far less than 8 planes.
-        auto plane_done = [&](int plane) {
-            if (lane == 0 && (atomicAdd(&applied_s[plane & 7], 1u) % G::kConvWarps) == G::kConvWarps - 1)
-                atomicAdd(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrApplied, 1u);
-        };
-        PatchWalk wk; wk.init(prm);
-        for (int it = 0; wk.valid(); ++it, wk.step()) {
+        for (int it = 0;; ++it) {
             const int s = it % NA, use = it / NA, b = it & 1, ub = it >> 1;
-            const int bh = wk.bh;
+            if (__any_sync(0xffffffffu, !mbar_wait(&a_full[s], use & 1, abort_flag, prm.status, kBit))) break;
+            const int g = a_info[s];
+            if (g == kNoWork) break;
+            const int bh = g / tpb;
             if (bh != prev_bh) {
-                if (prev_bh >= 0) plane_done(prev_bh);
                 prev_bh = bh;
                 if (__any_sync(0xffffffffu, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit))) break;
                 ++pseg;
@@ -615,7 +637,6 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                         wreg[dy][dx] = make_float2(__bfloat162float(prm.w[(size_t)ch * KS * KS + dy * KS + dx]),
                                                    __bfloat162float(prm.w[(size_t)(ch + 1) * KS * KS + dy * KS + dx]));
             }
-            if (__any_sync(0xffffffffu, !mbar_wait(&a_full[s], use & 1, abort_flag, prm.status, kBit))) break;
             if (ub > 0 && __any_sync(0xffffffffu, !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit))) break;
             // Window of KS tokens per halo row, sliding along x.  Token t (relative to the first token this
             // lane needs) sits U bytes after token t-1: U = 128, one token per column, or (PAIR) 64.
@@ -660,13 +681,16 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             }
             mbar_arrive(&a_empty[s]);      // the V patch of this stage is no longer needed
             mbar_arrive(&conv_full[b]);
+            // The conv warp that finishes a patch last counts it as applied (one arrival per patch and CTA: the state
+            // pipelines poll these counters).  Warps are at most a few patches apart, far less than 8.
+            if (lane == 0 && (atomicAdd(&applied_s[it & 7], 1u) % G::kConvWarps) == G::kConvWarps - 1)
+                atomicAdd(plane_ctr + (size_t)bh * kPipeCtrPerPlane + kPipeCtrApplied, 1u);
         }
-        if (prev_bh >= 0 && !*abort_flag) plane_done(prev_bh);
     }
     tcgen05_fence_before_sync();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-    // The CTA that leaves last puts the per-plane counters back to zero for the next call.
+    // The CTA that leaves last puts the counters back to zero for the next call.
     if (tid == 0) {
         __threadfence();
         *last_slot = (atomicAdd(prm.ctr, 1u) == (unsigned)(n_cta - 1));
@@ -675,7 +699,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (*last_slot) {
         __threadfence();
         for (int i = tid; i < prm.BH * kPipeCtrPerPlane; i += blockDim.x) plane_ctr[i] = 0;
-        if (tid == 0) prm.ctr[0] = 0;
+        if (tid < kPipeCtrHeader) prm.ctr[tid] = 0;
     }
 }
 
@@ -727,7 +751,8 @@ cudaError_t launch_pipe_ks(const Problem& p, float* partial, float* state, unsig
     prm.flat = (rank == 4) ? 1 : 0;
     prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
-    prm.s_tiles = plan.s_tiles; prm.ahead = plan.ahead; prm.ring = plan.ring;
+    prm.s_tiles = plan.s_tiles; prm.chunk_tiles = plan.chunk_tiles; prm.n_chunks = plan.n_chunks;
+    prm.ahead = plan.ahead; prm.ring = plan.ring;
     prm.eps2 = p.eps2; prm.status = status;
     static PerDevice opt_in;  // one per instantiation
     {
@@ -755,25 +780,32 @@ int planes_ahead(int BH, int rows) {
 
 }  // namespace
 
-// Work split of the one-kernel forward.  It takes planes with at least two thirds as many patches as there are
-// multiprocessors (every CTA gets a share of every plane); shorter planes go to the separate kernels.
+// Work split of the one-kernel forward: the rows of a plane are cut into chunks of kChunkTiles 64-row tiles,
+// the grid into patches; one CTA per multiprocessor, or fewer when there is less work than that.
+constexpr int kChunkTiles = 8;
+
 PipePlan plan_pipe(int BH, int rows, int cols, int gridH) {
     PipePlan pl = {};
     const int sms = device_sm_count();
     if (rows < 1 || BH < 1 || cols < 1 || gridH < 1) return pl;
     pl.s_tiles = (rows + kSTile - 1) / kSTile;
-    const int patches = ((cols + kTX - 1) / kTX) * ((gridH + kTY - 1) / kTY);
-    pl.grid = patches < sms ? patches : sms;
+    pl.chunk_tiles = kChunkTiles;
+    pl.n_chunks = (pl.s_tiles + kChunkTiles - 1) / kChunkTiles;
+    const long long patches = (long long)BH * ((cols + kTX - 1) / kTX) * ((gridH + kTY - 1) / kTY);
+    const long long chunks = (long long)BH * pl.n_chunks;
+    const long long work = patches > chunks ? patches : chunks;
+    pl.grid = (int)(work < sms ? work : sms);
     pl.ahead = planes_ahead(BH, rows);
-    pl.ring = pl.ahead;  // plane p + ring starts after plane p + ring - ahead >= p is applied, so plane p's sums are used up
-    pl.ok = (3 * patches >= 2 * sms) && pl.s_tiles >= pl.grid;
+    pl.ring = pl.ahead;  // plane p + ring starts only after plane p is applied, so plane p's chunk sums are used up by then
+    pl.ok = true;
     return pl;
 }
 
-// Per-CTA sums that the workspace has to hold for any grid of `rows` 128-byte rows per plane.
+// Chunk sums (of kStateWords each) that the workspace has to hold for planes of `rows` 128-byte rows.
 size_t pipe_partial_slots(int BH, int rows) {
     if (rows < 1 || BH < 1) return 0;
-    return (size_t)planes_ahead(BH, rows) * device_sm_count();
+    const int s_tiles = (rows + kSTile - 1) / kSTile;
+    return (size_t)planes_ahead(BH, rows) * ((s_tiles + kChunkTiles - 1) / kChunkTiles);
 }
 
 bool pipe_supports(const Problem& p) {
