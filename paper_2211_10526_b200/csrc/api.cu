@@ -49,18 +49,18 @@ size_t elem_bytes(castling_dtype_t t) { return t == CASTLING_F32 ? 4 : 2; }
 
 // header | state [BH] | partial [BH][P] (only when the token range is split)
 size_t workspace_words(int BH, int N, int d, bool bf16) {
-    const int P = castling::simt_choose_splits(BH, N);
+    int P = castling::simt_choose_splits(BH, N);
     size_t words = castling::state_words(d);
-    size_t slots = (size_t)BH * (P > 1 ? P : 0);  // partial states behind the BH final ones
     if (bf16 && (d == 64 || d == 32)) {  // shapes the tensor-core kernels may take: they keep 64-wide states
-        const size_t st = castling::tc::partial_slots(BH, castling::tc::rows_per_head(N, d));
-        if (st > slots) slots = st;
+        const int Pt = castling::tc::choose_splits(BH, castling::tc::rows_per_head(N, d));
+        if (Pt > P) P = Pt;
         words = castling::tc::kStateWords;
-        if (d == 32 && BH % 2 == 0) {
-            // two width-32 heads side by side (token-major layouts): BH / 2 planes of N rows each
-            const size_t sp = castling::tc::partial_slots(BH / 2, N);
-            if (sp > slots) slots = sp;
-        }
+    }
+    size_t slots = (size_t)BH * (P > 1 ? P : 0);  // partial states behind the BH final ones
+    if (bf16 && d == 32 && BH % 2 == 0) {
+        // two width-32 heads side by side (token-major layouts): BH / 2 planes of N rows each
+        const int Pp = castling::tc::choose_splits(BH / 2, N);
+        if (Pp > 1 && (size_t)(BH / 2) * Pp > slots) slots = (size_t)(BH / 2) * Pp;
     }
     return castling::kHeaderWords + ((size_t)BH + slots) * words;
 }
@@ -105,7 +105,7 @@ int ensure_workspace(castling_attn* h, int BH, int N, int d, bool bf16) {
 }
 
 int ensure_counters(castling_attn* h, int BH) {
-    // either variant of the tensor-core path: 17 words per plane, or a header and 4 words per plane
+    // either variant of the tensor-core path: 17 words per plane, or a header and 2 words per plane
     const size_t a = (size_t)BH * castling::tc::kCountersPerHead;
     const size_t b = castling::tc::kPipeCtrHeader + (size_t)BH * castling::tc::kPipeCtrPerPlane;
     const size_t want = a > b ? a : b;

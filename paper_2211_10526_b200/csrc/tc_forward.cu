@@ -57,12 +57,6 @@ static bool two_kernels() {
     return !one;
 }
 
-size_t partial_slots(int BH, int rows) {
-    const int P = choose_splits(BH, rows);
-    const size_t a = P > 1 ? (size_t)BH * P : 0, b = pipe_partial_slots(BH, rows);
-    return a > b ? a : b;
-}
-
 cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
@@ -83,7 +77,7 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
     cudaError_t e;
     if (!two_kernels() && pipe_supports(p)) {
         // state and apply pipelines in one persistent kernel: V is read from memory once
-        e = launch_pipe(p, ws_partial, ws_state, counters, status, stream);
+        e = launch_pipe(p, ws_state, counters, status, stream);
         if (e != cudaSuccess) return e;
         ++*launches;
         timer->mark(stream, "tc_pipe");

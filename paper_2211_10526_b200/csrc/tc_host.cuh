@@ -34,9 +34,6 @@ constexpr int kStateWords = 64 * 64 + 64;
 
 // Token splits of the tensor-core state kernel and the workspace words it needs beyond the state.
 int choose_splits(int BH, int N);
-// Partial states (of kStateWords each) behind the final ones that either variant of the path needs for
-// BH planes of `rows` 128-byte rows: what the workspace is sized for.
-size_t partial_slots(int BH, int rows);
 
 // Enqueue state build, split reduction and apply for one problem.  `status` is the device status
 // word; `counters` holds kCountersPerHead zero-initialised arrival counters per (b,h), left at zero by every call.  Returns the cudaError_t of the launches; cudaErrorNotSupported if a tensor map could not
@@ -54,27 +51,24 @@ cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_
 // One-kernel forward (csrc/tc_pipe.cu): a state pipeline and an apply pipeline share every CTA; work is handed
 // out, and progress is signalled, through counters in global memory.
 // Counter layout: kPipeCtrHeader words (CTAs that have left, next patch to hand out, next chunk of rows to hand
-// out), then kPipeCtrPerPlane words per plane: chunks whose sums are written, summation slices handed out, slices
-// added, patches applied.  All zero between calls.
-constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 4;
-constexpr int kPipeCtrNextPatch = 1, kPipeCtrNextChunk = 2;
-constexpr int kPipeCtrWritten = 0, kPipeCtrClaimed = 1, kPipeCtrSummed = 2, kPipeCtrApplied = 3;
+// out, CTAs that have cleared their part of the states), then kPipeCtrPerPlane words per plane: chunks whose
+// sums are added to the plane's state, patches applied.  All zero between calls.
+constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 2;
+constexpr int kPipeCtrNextPatch = 1, kPipeCtrNextChunk = 2, kPipeCtrCleared = 3;
+constexpr int kPipeCtrWritten = 0, kPipeCtrApplied = 1;
 struct PipePlan {
     bool ok;           // the one-kernel forward takes this shape
     int grid;          // CTAs (at most one per multiprocessor)
     int s_tiles;       // 64-row state tiles per plane
-    int chunk_tiles;   // tiles per chunk of rows (one partial sum per chunk)
+    int chunk_tiles;   // tiles per chunk of rows
     int n_chunks;      // chunks per plane
     int ahead;         // planes the state pipeline may run ahead of the apply pipeline
-    int ring;          // planes whose chunk sums are kept at a time
 };
 // rows: 128-byte rows per plane (leading tokens included); cols x gridH: the token grid in 128-byte columns.
 PipePlan plan_pipe(int BH, int rows, int cols, int gridH);
 bool pipe_supports(const Problem& p);
-// Chunk sums (of kStateWords each) the workspace must hold behind the final states for such planes.
-size_t pipe_partial_slots(int BH, int rows);
-// Chunk sums live at partial[plane % ring][chunk], final ones at state[plane]; ctr as described above.
-cudaError_t launch_pipe(const Problem& p, float* partial, float* state, unsigned* ctr, unsigned* status, cudaStream_t st);
+// The plane sums end up at state[plane] (cleared by the kernel itself); ctr as described above.
+cudaError_t launch_pipe(const Problem& p, float* state, unsigned* ctr, unsigned* status, cudaStream_t st);
 
 // Single-kernel forward for short sequences (bf16, 3x3 or 5x5 filters, at most 256 128-byte rows per plane:
 // d = 64 with N <= 256, two width-32 heads per row with N <= 256, or width-32 token pairs with N <= 512): no workspace.

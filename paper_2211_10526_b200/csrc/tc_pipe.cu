@@ -72,8 +72,7 @@ template <int KS, bool PAIR> struct PGeo {
 };
 
 struct PipeParams {
-    float* partial;                // [ring][chunk][kWords] sums over one chunk of rows of one plane
-    float* state;                  // [BH][kWords] final sums
+    float* state;                  // [BH][kWords] sums S then s of every plane
     unsigned* ctr;                 // kPipeCtrHeader words, then kPipeCtrPerPlane per plane; all zero between calls
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
@@ -83,14 +82,11 @@ struct PipeParams {
     int s_tiles;                   // 64-row state tiles per plane
     int chunk_tiles, n_chunks;     // tiles per chunk, chunks per plane
     int ahead;                     // a chunk of plane p is started only when plane p - ahead is applied
-    int ring;                      // plane slots of `partial`: plane p uses slot p % ring
     float eps2;
     unsigned* status;
 };
 
 constexpr int kNoWork = -1;            // stage info: nothing more to do
-constexpr int kSliceWords4 = kEpiWarps;  // float4 positions of a summation slice: one per epilogue warp
-constexpr int kSlices = (kWords4 + kSliceWords4 - 1) / kSliceWords4;
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
@@ -103,6 +99,11 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
 // device-wide fence in every thread waits for the copies the CTA's pipelines have in flight, again and again.
 __device__ __forceinline__ void signal_add(unsigned* p) {
     asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+}
+
+// Adds four floats to four consecutive words of global memory (performed at the L2, no value returned).
+__device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float c, float d) {
+    asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
 // Bounded wait for a counter in global memory to reach `want`.  Gives up (returns false) when the limit
@@ -166,7 +167,6 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sacc_free + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* last_slot = reinterpret_cast<int*>(tmem_slot + 2);
-    volatile int* sum_go = reinterpret_cast<volatile int*>(tmem_slot + 3);  // the polling thread's verdict on a slice sum
     unsigned* applied_s = reinterpret_cast<unsigned*>(tmem_slot + 4);  // [8] conv warps done with the CTA's i-th patch, slot i & 7
     volatile int* a_info = reinterpret_cast<volatile int*>(tmem_slot + 12);  // [NA] patch in the apply stage, or kNoWork
     volatile int* s_info = a_info + 4;                                      // [NS] chunk * 4 + (first tile) + 2 * (last tile), or kNoWork
@@ -176,7 +176,6 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     unsigned* plane_ctr = prm.ctr + kPipeCtrHeader;
     const int tpb = prm.tilesX * prm.tilesY;                 // patches per plane
     const int n_patches = prm.BH * tpb, n_chunks_all = prm.BH * prm.n_chunks;
-    (void)cta;
 
     if (tid == 0) {
         for (int s = 0; s < NA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], G::kConvThreads + kEpiThreads + 1); }
@@ -201,9 +200,18 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         *reinterpret_cast<uint4*>(ones + r * 128 + c * 16) = val;
         fence_proxy_async_smem();
     }
+    // Every CTA clears its part of the states, which the chunk sums are added to; the first addition of any CTA
+    // waits until all parts are cleared (by then they long are).
+    {
+        const int n4 = prm.BH * kWords4;
+        float4* st4 = reinterpret_cast<float4*>(prm.state);
+        for (int i = (int)((long long)n4 * cta / n_cta) + tid, e = (int)((long long)n4 * (cta + 1) / n_cta); i < e; i += blockDim.x)
+            st4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     tcgen05_fence_before_sync();
     __syncthreads();
     tcgen05_fence_after_sync();
+    if (tid == 0) signal_add(prm.ctr + kPipeCtrCleared);
     const uint32_t tmem = *tmem_slot;
     const uint32_t tmem_state = tmem + 128;
 
@@ -224,6 +232,14 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     break;
                 }
                 const int g_next = (int)atomicAdd(prm.ctr + kPipeCtrNextPatch, 1u);
+                if (g_next < n_patches) {
+                    // the next patch's Q on its way from memory to L2 already: the stages hold too little to cover
+                    // that latency (V was read by the state pipeline moments ago and is in L2 anyway)
+                    const int nb = g_next / tpb, nr = g_next - nb * tpb;
+                    const int ny = (nr / prm.tilesX) * kTY, nx = (nr % prm.tilesX) * kTX;
+                    if (prm.flat) tma_prefetch_4d(&tmQ, 0, nx, ny, nb);
+                    else tma_prefetch_5d(&tmQ, 0, nx, ny, nb % prm.hdiv, nb / prm.hdiv);
+                }
                 const int bh = g / tpb, rem = g - bh * tpb;
                 const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
                 uint8_t* qs = stages + s * G::kStage;
@@ -292,6 +308,16 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     break;
                 }
                 const int g_next = (int)atomicAdd(prm.ctr + kPipeCtrNextChunk, 1u);
+                if (g_next < n_chunks_all) {
+                    // the next chunk's rows on their way from memory to L2 already (see the patches above)
+                    const int np = g_next / prm.n_chunks, nj = g_next - np * prm.n_chunks;
+                    const int nb = np / prm.hdiv, nh = np - nb * prm.hdiv;
+                    const int n0 = nj * prm.chunk_tiles, n1 = min(prm.s_tiles, n0 + prm.chunk_tiles);
+                    for (int t = n0; t < n1; ++t) {
+                        tma_prefetch_4d(&tmK, 0, t * kSTile, nh, nb);
+                        tma_prefetch_4d(&tmVs, 0, t * kSTile, nh, nb);
+                    }
+                }
                 const int plane = g / prm.n_chunks, j = g - plane * prm.n_chunks;
                 if (plane >= prm.ahead &&
                     !wait_counter(plane_ctr + (size_t)(plane - prm.ahead) * kPipeCtrPerPlane + kPipeCtrApplied, (unsigned)tpb,
@@ -348,62 +374,6 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         const int half = ew >> 2;  // channels half*32 .. half*32 + 31
         const bool leader = (et == 0);
         const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
-        // Adds up the chunk sums of `plane`, slice by slice, for as long as there are unclaimed slices (at most
-        // `max_claims` of them).  Slices are handed out from a counter; a slice is kEpiWarps float4 positions, one
-        // per warp: lane l adds the sums of chunks l, l + 32, ... in that order and the 32 results meet in a fixed
-        // shuffle tree, so the total does not depend on who added what when.  The chunk sums must all be written:
-        // with `blocking` the call waits for that, otherwise it returns at once when they are not.  Returns false
-        // after a failed wait.  All epilogue threads call it together and get the same answer.
-        auto sum_slices = [&](int plane, int max_claims, bool blocking) -> bool {
-            unsigned* pc = plane_ctr + (size_t)plane * kPipeCtrPerPlane;
-            const float4* base = reinterpret_cast<const float4*>(prm.partial + (size_t)(plane % prm.ring) * prm.n_chunks * kWords);
-            float4* fin = reinterpret_cast<float4*>(prm.state + (size_t)plane * kWords);
-            for (int claim = 0; claim < max_claims; ++claim) {
-                if (leader) {
-                    int go = kNoWork;  // slice to add, kNoWork: nothing (left) to do, -2: failed
-                    bool there = true;
-                    if (claim == 0) {
-                        if (blocking) { if (!wait_counter(&pc[kPipeCtrWritten], (unsigned)prm.n_chunks, abort_flag, prm.status)) { there = false; go = -2; } }
-                        else there = ld_acquire(&pc[kPipeCtrWritten]) >= (unsigned)prm.n_chunks;
-                    }
-                    if (there && ld_acquire(&pc[kPipeCtrClaimed]) < (unsigned)kSlices) {
-                        const unsigned c = atomicAdd(&pc[kPipeCtrClaimed], 1u);
-                        if (c < (unsigned)kSlices) go = (int)c;
-                    }
-                    *sum_go = go;
-                }
-                named_barrier_sync(4, kEpiThreads);
-                const int go = *sum_go;
-                named_barrier_sync(4, kEpiThreads);  // everybody has read the verdict before the next one is written
-                if (go == -2) return false;
-                if (go == kNoWork) return true;
-                const int pos = go * kSliceWords4 + ew;
-                if (pos < kWords4) {
-                    float4 v[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int m = lane + 32 * j;
-                        v[j] = (m < prm.n_chunks) ? __ldcg(base + (size_t)m * kWords4 + pos) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                    float4 acc = v[0];
-#pragma unroll
-                    for (int j = 1; j < 4; ++j) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
-                    for (int m = lane + 128; m < prm.n_chunks; m += 32) {
-                        const float4 u = __ldcg(base + (size_t)m * kWords4 + pos);
-                        acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
-                    }
-#pragma unroll
-                    for (int sh = 16; sh >= 1; sh >>= 1) {
-                        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, sh); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, sh);
-                        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, sh); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, sh);
-                    }
-                    if (lane == 0) fin[pos] = acc;
-                }
-                named_barrier_sync(4, kEpiThreads);
-                if (leader) signal_add(&pc[kPipeCtrSummed]);
-            }
-            return true;
-        };
         int prev_bh = -1, pseg = 0;
         bool failed = false;  // the same for every epilogue thread wherever a barrier follows
         for (int it = 0;; ++it) {
@@ -416,14 +386,11 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             if (bh != prev_bh) {
                 const int p = bh;
                 prev_bh = p;
-                // the plane's state is final when every slice of it has been added; help with that first
-                failed = !sum_slices(p, kSlices, true);
-                if (!failed) {
-                    if (leader && wait_counter(plane_ctr + (size_t)p * kPipeCtrPerPlane + kPipeCtrSummed, (unsigned)kSlices, abort_flag, prm.status))
-                        mbar_arrive(p_ready);
-                    failed = barrier_any(4, kEpiThreads, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit));
-                    ++pseg;
-                }
+                // the plane's state is final when the sums of all its chunks of rows have been added to it
+                if (leader && wait_counter(plane_ctr + (size_t)p * kPipeCtrPerPlane + kPipeCtrWritten, (unsigned)prm.n_chunks, abort_flag, prm.status))
+                    mbar_arrive(p_ready);
+                failed = barrier_any(4, kEpiThreads, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit));
+                ++pseg;
                 // every UMMA that read the previous S' has retired (its acc_full was waited on below)
                 if (!failed) {
                     const int i = et >> 2, part = et & 3;  // row i of the operand, 16 columns part*16 ..
@@ -458,9 +425,6 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     }
                     fence_proxy_async_smem();
                     mbar_arrive(s_ready);
-                    // a slice or two of the next plane, if its chunk sums are there already: by the time anyone
-                    // gets to that plane, its state is final
-                    if (p + 1 < prm.BH) failed = !sum_slices(p + 1, 2, false);
                 }
             }
             float a[32];
@@ -570,13 +534,18 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 mbar_arrive(&s_scaled[s]);
             }
             if (!last) continue;
-            // the chunk's sums leave TMEM: rows 0..63 are S, row 64 is s
-            const int chunk = info >> 2, plane = chunk / prm.n_chunks, j_chunk = chunk - plane * prm.n_chunks;
+            // the chunk's sums leave TMEM (rows 0..63 are S, row 64 is s) and are added to the plane's state
+            const int chunk = info >> 2, plane = chunk / prm.n_chunks;
             const int buf = (k_chunk - 1) & 1;
-            const bool ok = mbar_wait(&sacc_full[buf], ((k_chunk - 1) >> 1) & 1, abort_flag, prm.status, kBit);
+            bool ok = mbar_wait(&sacc_full[buf], ((k_chunk - 1) >> 1) & 1, abort_flag, prm.status, kBit);
+            if (k_chunk == 1) {
+                // the first sums of this CTA: every CTA must have cleared its part of the states by now
+                if (t == 0 && ok) ok = wait_counter(prm.ctr + kPipeCtrCleared, (unsigned)n_cta, abort_flag, prm.status);
+                ok = !barrier_any(3, kNormThreads, !ok);
+            }
             if (ok) {
                 tcgen05_fence_after_sync();
-                float* dst = prm.partial + ((size_t)(plane % prm.ring) * prm.n_chunks + j_chunk) * kWords;
+                float* dst = prm.state + (size_t)plane * kWords;
                 if (quarter < 3) {
                     const int row = quarter * 32 + lane;
 #pragma unroll
@@ -585,9 +554,9 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                         tmem_ld16(tmem_state + ((uint32_t)(quarter * 32) << 16) + buf * kD + cc * 16, v);
                         tmem_ld_wait();
                         if (row <= kD) {
-                            float4* o4 = reinterpret_cast<float4*>(dst + row * kD + cc * 16);  // row 64 lands on s
+                            float* o4 = dst + row * kD + cc * 16;  // row 64 lands on s
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) o4[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                            for (int e = 0; e < 4; ++e) red_add_f32x4(o4 + 4 * e, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
                         }
                     }
                 }
@@ -704,7 +673,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 }
 
 template <int KS, int MODE>
-cudaError_t launch_pipe_ks(const Problem& p, float* partial, float* state, unsigned* ctr, unsigned* status, cudaStream_t st) {
+cudaError_t launch_pipe_ks(const Problem& p, float* state, unsigned* ctr, unsigned* status, cudaStream_t st) {
     constexpr bool PAIR = (MODE == 1);
     using G = PGeo<KS, PAIR>;
     const bool pair = PAIR;
@@ -745,14 +714,14 @@ cudaError_t launch_pipe_ks(const Problem& p, float* partial, float* state, unsig
             return cudaErrorNotSupported;
     }
     PipeParams prm;
-    prm.partial = partial; prm.state = state; prm.ctr = ctr;
+    prm.state = state; prm.ctr = ctr;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.flat = (rank == 4) ? 1 : 0;
     prm.H = p.H; prm.head0 = p.head0; prm.BH = p.BH; prm.hdiv = p.hdiv;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.s_tiles = plan.s_tiles; prm.chunk_tiles = plan.chunk_tiles; prm.n_chunks = plan.n_chunks;
-    prm.ahead = plan.ahead; prm.ring = plan.ring;
+    prm.ahead = plan.ahead;
     prm.eps2 = p.eps2; prm.status = status;
     static PerDevice opt_in;  // one per instantiation
     {
@@ -796,16 +765,8 @@ PipePlan plan_pipe(int BH, int rows, int cols, int gridH) {
     const long long work = patches > chunks ? patches : chunks;
     pl.grid = (int)(work < sms ? work : sms);
     pl.ahead = planes_ahead(BH, rows);
-    pl.ring = pl.ahead;  // plane p + ring starts only after plane p is applied, so plane p's chunk sums are used up by then
     pl.ok = true;
     return pl;
-}
-
-// Chunk sums (of kStateWords each) that the workspace has to hold for planes of `rows` 128-byte rows.
-size_t pipe_partial_slots(int BH, int rows) {
-    if (rows < 1 || BH < 1) return 0;
-    const int s_tiles = (rows + kSTile - 1) / kSTile;
-    return (size_t)planes_ahead(BH, rows) * ((s_tiles + kChunkTiles - 1) / kChunkTiles);
 }
 
 bool pipe_supports(const Problem& p) {
@@ -813,15 +774,15 @@ bool pipe_supports(const Problem& p) {
     return plan_pipe(p.BH, pair ? p.N / 2 : p.N, pair ? p.gridW / 2 : p.gridW, p.gridH).ok;
 }
 
-cudaError_t launch_pipe(const Problem& p, float* partial, float* state, unsigned* ctr, unsigned* status, cudaStream_t st) {
+cudaError_t launch_pipe(const Problem& p, float* state, unsigned* ctr, unsigned* status, cudaStream_t st) {
     if (p.d == 32)
-        return p.ksize == 3 ? launch_pipe_ks<3, 1>(p, partial, state, ctr, status, st)
-                            : launch_pipe_ks<5, 1>(p, partial, state, ctr, status, st);
+        return p.ksize == 3 ? launch_pipe_ks<3, 1>(p, state, ctr, status, st)
+                            : launch_pipe_ks<5, 1>(p, state, ctr, status, st);
     if (p.blockdiag)
-        return p.ksize == 3 ? launch_pipe_ks<3, 2>(p, partial, state, ctr, status, st)
-                            : launch_pipe_ks<5, 2>(p, partial, state, ctr, status, st);
-    return p.ksize == 3 ? launch_pipe_ks<3, 0>(p, partial, state, ctr, status, st)
-                        : launch_pipe_ks<5, 0>(p, partial, state, ctr, status, st);
+        return p.ksize == 3 ? launch_pipe_ks<3, 2>(p, state, ctr, status, st)
+                            : launch_pipe_ks<5, 2>(p, state, ctr, status, st);
+    return p.ksize == 3 ? launch_pipe_ks<3, 0>(p, state, ctr, status, st)
+                        : launch_pipe_ks<5, 0>(p, state, ctr, status, st);
 }
 
 }  // namespace tc
