@@ -62,7 +62,12 @@ size_t workspace_words(int BH, int N, int d, bool bf16) {
         const int Pp = castling::tc::choose_splits(BH / 2, N);
         if (Pp > 1 && (size_t)(BH / 2) * Pp > slots) slots = (size_t)(BH / 2) * Pp;
     }
-    return castling::kHeaderWords + ((size_t)BH + slots) * words;
+    size_t behind = slots * words;  // what follows the BH final states
+    if (bf16 && (d == 64 || d == 32)) {  // the one-kernel forward keeps its per-plane operand blocks there
+        const size_t r = castling::tc::pipe_ready_words(BH);
+        if (r > behind) behind = r;
+    }
+    return castling::kHeaderWords + (size_t)BH * words + behind;
 }
 
 int fail_cuda(castling_attn* h, cudaError_t e, int code = CASTLING_ERR_CUDA) {
@@ -105,7 +110,7 @@ int ensure_workspace(castling_attn* h, int BH, int N, int d, bool bf16) {
 }
 
 int ensure_counters(castling_attn* h, int BH) {
-    // either variant of the tensor-core path: 17 words per plane, or a header and 2 words per plane
+    // either variant of the tensor-core path: 17 words per plane, or a header and 4 words per plane
     const size_t a = (size_t)BH * castling::tc::kCountersPerHead;
     const size_t b = castling::tc::kPipeCtrHeader + (size_t)BH * castling::tc::kPipeCtrPerPlane;
     const size_t want = a > b ? a : b;

@@ -77,7 +77,7 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
     cudaError_t e;
     if (!two_kernels() && pipe_supports(p)) {
         // state and apply pipelines in one persistent kernel: V is read from memory once
-        e = launch_pipe(p, ws_state, counters, status, stream);
+        e = launch_pipe(p, ws_state, ws_partial, counters, status, stream);
         if (e != cudaSuccess) return e;
         ++*launches;
         timer->mark(stream, "tc_pipe");

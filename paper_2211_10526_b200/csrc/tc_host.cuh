@@ -52,10 +52,10 @@ cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_
 // out, and progress is signalled, through counters in global memory.
 // Counter layout: kPipeCtrHeader words (CTAs that have left, next patch to hand out, next chunk of rows to hand
 // out, CTAs that have cleared their part of the states), then kPipeCtrPerPlane words per plane: chunks whose
-// sums are added to the plane's state, patches applied.  All zero between calls.
-constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 2;
+// sums are added to the plane's state, patches applied, the plane's operand block is ready.  All zero between calls.
+constexpr int kPipeCtrHeader = 4, kPipeCtrPerPlane = 4;
 constexpr int kPipeCtrNextPatch = 1, kPipeCtrNextChunk = 2, kPipeCtrCleared = 3;
-constexpr int kPipeCtrWritten = 0, kPipeCtrApplied = 1;
+constexpr int kPipeCtrWritten = 0, kPipeCtrApplied = 1, kPipeCtrReady = 2;
 struct PipePlan {
     bool ok;           // the one-kernel forward takes this shape
     int grid;          // CTAs (at most one per multiprocessor)
@@ -67,8 +67,10 @@ struct PipePlan {
 // rows: 128-byte rows per plane (leading tokens included); cols x gridH: the token grid in 128-byte columns.
 PipePlan plan_pipe(int BH, int rows, int cols, int gridH);
 bool pipe_supports(const Problem& p);
-// The plane sums end up at state[plane] (cleared by the kernel itself); ctr as described above.
-cudaError_t launch_pipe(const Problem& p, float* state, unsigned* ctr, unsigned* status, cudaStream_t st);
+// The plane sums end up at state[plane] (cleared by the kernel itself); `ready` holds pipe_ready_words(BH) words
+// for the per-plane operand blocks that the apply pipelines copy; ctr as described above.
+size_t pipe_ready_words(int BH);
+cudaError_t launch_pipe(const Problem& p, float* state, float* ready, unsigned* ctr, unsigned* status, cudaStream_t st);
 
 // Single-kernel forward for short sequences (bf16, 3x3 or 5x5 filters, at most 256 128-byte rows per plane:
 // d = 64 with N <= 256, two width-32 heads per row with N <= 256, or width-32 token pairs with N <= 512): no workspace.

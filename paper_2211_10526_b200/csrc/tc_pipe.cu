@@ -35,8 +35,11 @@ constexpr int kD = 64;
 constexpr int kTY = 8, kTX = 16;            // patch: 8 rows x 16 columns of 128-byte rows
 constexpr int kPatch = kTY * kTX;
 constexpr int kQBytes = kPatch * kD * 2;    // 16 KiB
-constexpr int kStgStride = kD * 4 + 16;     // fp32 row + 16 B pad: conflict-free row-per-thread reads
+constexpr int kStgStride = kD * 4;          // fp32 row; 16-byte chunk c of row t sits at chunk c ^ (t & 7)
 constexpr int kStgBytes = kPatch * kStgStride;
+constexpr int kSpBytes = kD * kD * 2;       // S' = S / pi as the bf16 B operand of the apply UMMAs (swizzled image)
+constexpr int kHsBytes = kD * 4;            // 1/2 s
+constexpr int kReadyWords = (kSpBytes + kHsBytes) / 4;  // per plane in global memory: S' image, then 1/2 s
 constexpr int kEpiWarps = 8, kEpiThreads = kEpiWarps * 32;
 constexpr int kNormWarps = 4, kNormThreads = kNormWarps * 32;
 constexpr int kSTile = 64;                  // rows per state stage
@@ -60,19 +63,21 @@ template <int KS, bool PAIR> struct PGeo {
     static constexpr int kStage = ((kQBytes + kVBytes + 1023) / 1024) * 1024;
     static constexpr int kStages = 2;                      // apply stages (Q patch + V patch with halo)
     static constexpr int kSStages = (KS == 3) ? 3 : 2;     // state stages (K tile + V tile)
-    // S' | out patch | apply stages | staging x2 | state stages | ones | rq x2 | barriers
-    static constexpr int kOffS = 0, kOffOut = 8192, kOffStages = kOffOut + kQBytes;
+    // S' x2 | out patch | apply stages | staging x2 | state stages | ones | rq x2 | 1/2 s x2 | barriers
+    static constexpr int kOffS = 0, kOffOut = 2 * kSpBytes, kOffStages = kOffOut + kQBytes;
     static constexpr int kOffStg = kOffStages + kStages * kStage;
     static constexpr int kOffSStages = ((kOffStg + 2 * kStgBytes + 1023) / 1024) * 1024;
     static constexpr int kOffOnes = kOffSStages + kSStages * kSStage;
     static constexpr int kOffRq = kOffOnes + kOnesBytes;   // sum of squares of each half of a Q row
-    static constexpr int kOffBar = kOffRq + 2 * kPatch * 4;
-    static constexpr size_t kSmem = 1024 + kOffBar + 512;
+    static constexpr int kOffHs = kOffRq + 2 * kPatch * 4;
+    static constexpr int kOffBar = kOffHs + 2 * kHsBytes;
+    static constexpr size_t kSmem = kOffBar + 512;
     static_assert(kSmem <= 227 * 1024, "shared memory of the one-kernel forward");
 };
 
 struct PipeParams {
     float* state;                  // [BH][kWords] sums S then s of every plane
+    float* ready;                  // [BH][kReadyWords] what the apply pipelines load per plane: S' image, 1/2 s
     unsigned* ctr;                 // kPipeCtrHeader words, then kPipeCtrPerPlane per plane; all zero between calls
     const __nv_bfloat16* w;        // [H*d][KS][KS]
     const __nv_bfloat16* bias;     // [H*d] or nullptr
@@ -104,6 +109,19 @@ __device__ __forceinline__ void signal_add(unsigned* p) {
 // Adds four floats to four consecutive words of global memory (performed at the L2, no value returned).
 __device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float c, float d) {
     asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// The same with the old value returned, and ordered before what follows as well.
+__device__ __forceinline__ unsigned signal_add_fetch(unsigned* p) {
+    unsigned old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(p) : "memory");
+    return old;
+}
+
+// Copy `bytes` (a multiple of 16) from global to shared memory; completion is counted on `bar`.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 // Bounded wait for a counter in global memory to reach `want`.  Gives up (returns false) when the limit
@@ -142,8 +160,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     constexpr bool PAIR = (MODE == 1), BLOCKDIAG = (MODE == 2), HALVES = PAIR || BLOCKDIAG;
     using G = PGeo<KS, PAIR>;
     constexpr int NA = G::kStages, NS = G::kSStages;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* S_s = smem + G::kOffS;
     uint8_t* out_s = smem + G::kOffOut;
     uint8_t* stg = smem + G::kOffStg;
@@ -151,15 +168,16 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     uint8_t* sstages = smem + G::kOffSStages;
     uint8_t* ones = smem + G::kOffOnes;
     float* rq_s = reinterpret_cast<float*>(smem + G::kOffRq);
+    float* hs_s = reinterpret_cast<float*>(smem + G::kOffHs);   // [2][64] 1/2 s of the plane in S' buffer 0 / 1
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G::kOffBar);
     uint64_t* a_full = bars;                 // [NA] Q and V patch landed
     uint64_t* a_empty = a_full + NA;         // [NA] stage consumed (conv + epilogue warps, UMMA commit)
     uint64_t* acc_full = a_empty + NA;       // [2]  apply UMMAs retired
     uint64_t* conv_full = acc_full + 2;      // [2]  staging written (conv threads)
     uint64_t* buf_free = conv_full + 2;      // [2]  accumulator and staging read out (epilogue threads)
-    uint64_t* s_ready = buf_free + 2;        //      S' of the current plane written (epilogue threads)
-    uint64_t* p_ready = s_ready + 1;         //      the current plane's state is final (one polling thread)
-    uint64_t* s_full = p_ready + 1;          // [NS] K and V tile landed
+    uint64_t* sp_full = buf_free + 2;        // [2]  S' and 1/2 s of a plane landed
+    uint64_t* sig_bar = sp_full + 2;         //      a chunk's sums are on their way to the plane's state (norm threads)
+    uint64_t* s_full = sig_bar + 1;          // [NS] K and V tile landed
     uint64_t* s_scaled = s_full + NS;        // [NS] K rows normalised
     uint64_t* s_empty = s_scaled + NS;       // [NS] state UMMAs of the stage retired
     uint64_t* sacc_full = s_empty + NS;      // [2]  accumulation of a plane retired
@@ -170,6 +188,9 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     unsigned* applied_s = reinterpret_cast<unsigned*>(tmem_slot + 4);  // [8] conv warps done with the CTA's i-th patch, slot i & 7
     volatile int* a_info = reinterpret_cast<volatile int*>(tmem_slot + 12);  // [NA] patch in the apply stage, or kNoWork
     volatile int* s_info = a_info + 4;                                      // [NS] chunk * 4 + (first tile) + 2 * (last tile), or kNoWork
+    volatile int* sig_info = s_info + 4;     // [4] plane of the k-th chunk this CTA has summed (slot k & 3), or kNoWork
+    volatile int* fin_req = sig_info + 4;    // [4] planes whose sums are complete and that this CTA is to finish (slot i & 3)
+    volatile int* fin_head = fin_req + 4;    // [2] number of such requests so far; 1 when the signalling thread has left
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_cta = (int)gridDim.x, cta = (int)blockIdx.x;
@@ -183,7 +204,8 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             mbar_init(&acc_full[b], 1); mbar_init(&conv_full[b], G::kConvThreads); mbar_init(&buf_free[b], kEpiThreads);
             mbar_init(&sacc_full[b], 1); mbar_init(&sacc_free[b], kNormThreads);
         }
-        mbar_init(s_ready, kEpiThreads); mbar_init(p_ready, 1);
+        mbar_init(&sp_full[0], 1); mbar_init(&sp_full[1], 1); mbar_init(sig_bar, kNormThreads);
+        fin_head[0] = 0; fin_head[1] = 0;
         for (int s = 0; s < NS; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_scaled[s], kNormThreads); mbar_init(&s_empty[s], 1); }
         *abort_flag = 0;
         for (int i = 0; i < 8; ++i) applied_s[i] = 0;
@@ -223,6 +245,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             // Patches are handed out one at a time, in plane order, from a counter in global memory: a slower
             // multiprocessor simply takes fewer.  The next claim is under way while this patch is loaded.
             int g = (int)atomicAdd(prm.ctr + kPipeCtrNextPatch, 1u);
+            int prev_bh = -1, seg = 0;
             for (int it = 0;; ++it) {
                 const int s = it % NA, use = it / NA;
                 if (use > 0 && !mbar_wait(&a_empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) break;
@@ -241,6 +264,18 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                     else tma_prefetch_5d(&tmQ, 0, nx, ny, nb % prm.hdiv, nb / prm.hdiv);
                 }
                 const int bh = g / tpb, rem = g - bh * tpb;
+                if (bh != prev_bh) {
+                    // a new plane: its S' and 1/2 s, once they are ready, into the S' buffer that the plane before
+                    // the previous one used (every patch of that plane has left its stage: see the wait above)
+                    prev_bh = bh;
+                    if (!wait_counter(plane_ctr + (size_t)bh * kPipeCtrPerPlane + kPipeCtrReady, 1u, abort_flag, prm.status)) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    const float* blk = prm.ready + (size_t)bh * kReadyWords;
+                    mbar_expect_tx(&sp_full[seg & 1], kSpBytes + kHsBytes);
+                    bulk_load(S_s + (seg & 1) * kSpBytes, blk, kSpBytes, &sp_full[seg & 1]);
+                    bulk_load(hs_s + (seg & 1) * kD, blk + kSpBytes / 4, kHsBytes, &sp_full[seg & 1]);
+                    ++seg;
+                }
                 const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
                 uint8_t* qs = stages + s * G::kStage;
                 a_info[s] = g;
@@ -265,7 +300,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         // ================= apply pipeline: UMMA issuer =================
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, kD, false, true);
-            const uint32_t s_addr = smem_u32(S_s);
+            uint32_t s_addr = smem_u32(S_s);
             int prev_bh = -1, seg = 0;
             for (int it = 0;; ++it) {
                 const int s = it % NA, use = it / NA, b = it & 1, ub = it >> 1;
@@ -274,7 +309,8 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 if (g == kNoWork) break;
                 const int bh = g / tpb;
                 if (bh != prev_bh) {
-                    if (!mbar_wait(s_ready, seg & 1, abort_flag, prm.status, kBit)) break;
+                    if (!mbar_wait(&sp_full[seg & 1], (seg >> 1) & 1, abort_flag, prm.status, kBit)) break;
+                    s_addr = smem_u32(S_s) + (seg & 1) * kSpBytes;
                     ++seg; prev_bh = bh;
                 }
                 if (ub > 0 && !mbar_wait(&buf_free[b], (ub - 1) & 1, abort_flag, prm.status, kBit)) break;
@@ -341,8 +377,27 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             }
         }
     } else if (warp == 3) {
-        // ================= state pipeline: UMMA issuer =================
-        if (lane == 0) {
+        if (lane == 1) {
+            // ================= state pipeline: signalling thread =================
+            // Counts every chunk of this CTA once its sums are on their way (ordered after them), so that the
+            // threads that produced them need not wait for memory to acknowledge anything.  Whoever counts the
+            // last chunk of a plane has its CTA finish that plane (see the norm warps).
+            for (int k = 0;; ++k) {
+                if (!mbar_wait(sig_bar, k & 1, abort_flag, prm.status, kBit)) break;
+                const int plane = sig_info[k & 3];
+                if (plane == kNoWork) break;
+                const unsigned old = signal_add_fetch(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrWritten);
+                if (old == (unsigned)prm.n_chunks - 1u) {
+                    const int h = fin_head[0];
+                    fin_req[h & 3] = plane;
+                    __threadfence_block();
+                    fin_head[0] = h + 1;
+                }
+            }
+            __threadfence_block();
+            fin_head[1] = 1;
+        } else if (lane == 0) {
+            // ================= state pipeline: UMMA issuer =================
             constexpr uint32_t idesc = umma_idesc_bf16(128, kD, true, true);
             const uint32_t ones_addr = smem_u32(ones);
             int k_chunk = 0;  // chunks started so far
@@ -370,11 +425,9 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     } else if (warp < kFirstWarpNorm) {
         // ================= apply pipeline: epilogue, thread = (token row of the patch, half of the channels) =================
         const int quarter = warp & 3, row = quarter * 32 + lane, et = tid - 32 * kFirstWarpEpi;
-        const int ew = warp - kFirstWarpEpi;
-        const int half = ew >> 2;  // channels half*32 .. half*32 + 31
+        const int half = (warp - kFirstWarpEpi) >> 2;  // channels half*32 .. half*32 + 31
         const bool leader = (et == 0);
         const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
-        int prev_bh = -1, pseg = 0;
         bool failed = false;  // the same for every epilogue thread wherever a barrier follows
         for (int it = 0;; ++it) {
             const int b = it & 1, ub = it >> 1, s = it % NA, use = it / NA;
@@ -383,50 +436,6 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             const int g = a_info[s];
             if (g == kNoWork) break;
             const int bh = g / tpb, rem = g - bh * tpb;
-            if (bh != prev_bh) {
-                const int p = bh;
-                prev_bh = p;
-                // the plane's state is final when the sums of all its chunks of rows have been added to it
-                if (leader && wait_counter(plane_ctr + (size_t)p * kPipeCtrPerPlane + kPipeCtrWritten, (unsigned)prm.n_chunks, abort_flag, prm.status))
-                    mbar_arrive(p_ready);
-                failed = barrier_any(4, kEpiThreads, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit));
-                ++pseg;
-                // every UMMA that read the previous S' has retired (its acc_full was waited on below)
-                if (!failed) {
-                    const int i = et >> 2, part = et & 3;  // row i of the operand, 16 columns part*16 ..
-                    const float* st = prm.state + (size_t)p * kWords;
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        float4 lo, hi;
-                        if (!PAIR) {
-                            const float4* src = reinterpret_cast<const float4*>(st + i * kD + part * 16);
-                            lo = __ldcg(src + 2 * c); hi = __ldcg(src + 2 * c + 1);
-                            if (BLOCKDIAG && ((i < 32) != (part < 2))) {  // off-diagonal block: the other head's keys
-                                lo = make_float4(0.f, 0.f, 0.f, 0.f); hi = lo;
-                            }
-                        } else {
-                            // operand = blockdiag(S32, S32) with S32 = block(0,0) + block(1,1) of the paired sums
-                            const int col = part * 16 + c * 8;  // first of 8 columns
-                            if ((i < 32) == (col < 32)) {
-                                const int a = i & 31, bcol = col & 31;
-                                const float4* s0 = reinterpret_cast<const float4*>(st + a * kD + bcol);
-                                const float4* s1 = reinterpret_cast<const float4*>(st + (32 + a) * kD + 32 + bcol);
-                                const float4 l0 = __ldcg(s0), h0 = __ldcg(s0 + 1), l1 = __ldcg(s1), h1 = __ldcg(s1 + 1);
-                                lo = make_float4(l0.x + l1.x, l0.y + l1.y, l0.z + l1.z, l0.w + l1.w);
-                                hi = make_float4(h0.x + h1.x, h0.y + h1.y, h0.z + h1.z, h0.w + h1.w);
-                            } else {
-                                lo = make_float4(0.f, 0.f, 0.f, 0.f); hi = lo;
-                            }
-                        }
-                        uint4 o;
-                        o.x = pack_bf16x2(lo.x * kInvPi, lo.y * kInvPi); o.y = pack_bf16x2(lo.z * kInvPi, lo.w * kInvPi);
-                        o.z = pack_bf16x2(hi.x * kInvPi, hi.y * kInvPi); o.w = pack_bf16x2(hi.z * kInvPi, hi.w * kInvPi);
-                        *reinterpret_cast<uint4*>(S_s + i * 128 + (((part * 2 + c) ^ (i & 7)) << 4)) = o;
-                    }
-                    fence_proxy_async_smem();
-                    mbar_arrive(s_ready);
-                }
-            }
             float a[32];
             if (!failed) {
                 // this thread's half of sum(q^2) for its token; the other half comes from the partner warp
@@ -462,12 +471,12 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             if (barrier_any(1, kEpiThreads, failed)) break;
             const float rq = HALVES ? rsqrtf(fmaxf(rq_s[half * kPatch + row], prm.eps2))   // half row = one token / one head
                                     : rsqrtf(fmaxf(rq_s[row] + rq_s[kPatch + row], prm.eps2));
-            const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
+            const uint8_t* srow = stg + b * kStgBytes + row * kStgStride;
             uint8_t* orow = out_s + row * 128;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {  // 8 channels -> one 16-byte chunk of the bf16 row
-                const float4 c0 = *reinterpret_cast<const float4*>(srow + e * 32);
-                const float4 c1 = *reinterpret_cast<const float4*>(srow + e * 32 + 16);
+                const float4 c0 = *reinterpret_cast<const float4*>(srow + (((half * 8 + 2 * e) ^ (row & 7)) << 4));
+                const float4 c1 = *reinterpret_cast<const float4*>(srow + (((half * 8 + 2 * e + 1) ^ (row & 7)) << 4));
                 uint4 pk;
                 pk.x = pack_bf16x2(fmaf(a[8 * e + 0], rq, c0.x), fmaf(a[8 * e + 1], rq, c0.y));
                 pk.y = pack_bf16x2(fmaf(a[8 * e + 2], rq, c0.z), fmaf(a[8 * e + 3], rq, c0.w));
@@ -496,11 +505,57 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         const int t = tid - 32 * kFirstWarpNorm;   // 0..127: row t >> 1 of the stage, half t & 1 of that row
         const int quarter = warp & 3;
         const int r = t >> 1, hf = t & 1;
-        int k_chunk = 0;  // chunks started so far
+        volatile int* fin_seen = fin_head + 2;  // [4] what thread 0 saw of fin_head, for everybody
+        int k_chunk = 0;   // chunks started so far
+        int fin_done = 0;  // planes finished by this CTA so far
+        bool dead = false; // a wait has failed: the same for all norm threads wherever a barrier follows
+        // Finishes a plane whose sums are complete: S' = S / pi as the bf16 operand image of the apply UMMAs (16-byte
+        // chunk c of row i at chunk c ^ (i & 7)) and 1/2 s go to memory, where the apply pipelines of all CTAs copy
+        // them from; then the plane's flag is raised.
+        auto finish_plane = [&](int plane) {
+            const float* st = prm.state + (size_t)plane * kWords;
+            uint8_t* blk = reinterpret_cast<uint8_t*>(prm.ready + (size_t)plane * kReadyWords);
+            const int i = t >> 1;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                const int c = (t & 1) * 4 + cc, col = c * 8;
+                float4 lo, hi;
+                if (!PAIR) {
+                    const float4* src = reinterpret_cast<const float4*>(st + i * kD + col);
+                    lo = __ldcg(src); hi = __ldcg(src + 1);
+                    if (BLOCKDIAG && ((i < 32) != (col < 32))) {  // off-diagonal block: the other head's keys
+                        lo = make_float4(0.f, 0.f, 0.f, 0.f); hi = lo;
+                    }
+                } else if ((i < 32) == (col < 32)) {
+                    // operand = blockdiag(S32, S32) with S32 = block(0,0) + block(1,1) of the paired sums
+                    const int a = i & 31, bcol = col & 31;
+                    const float4* s0 = reinterpret_cast<const float4*>(st + a * kD + bcol);
+                    const float4* s1 = reinterpret_cast<const float4*>(st + (32 + a) * kD + 32 + bcol);
+                    const float4 l0 = __ldcg(s0), h0 = __ldcg(s0 + 1), l1 = __ldcg(s1), h1 = __ldcg(s1 + 1);
+                    lo = make_float4(l0.x + l1.x, l0.y + l1.y, l0.z + l1.z, l0.w + l1.w);
+                    hi = make_float4(h0.x + h1.x, h0.y + h1.y, h0.z + h1.z, h0.w + h1.w);
+                } else {
+                    lo = make_float4(0.f, 0.f, 0.f, 0.f); hi = lo;
+                }
+                uint4 o;
+                o.x = pack_bf16x2(lo.x * kInvPi, lo.y * kInvPi); o.y = pack_bf16x2(lo.z * kInvPi, lo.w * kInvPi);
+                o.z = pack_bf16x2(hi.x * kInvPi, hi.y * kInvPi); o.w = pack_bf16x2(hi.z * kInvPi, hi.w * kInvPi);
+                *reinterpret_cast<uint4*>(blk + i * 128 + ((c ^ (i & 7)) << 4)) = o;
+            }
+            if (t < kD) {
+                const float* sv = st + kD * kD;
+                const float h = PAIR ? 0.5f * (__ldcg(sv + (t & 31)) + __ldcg(sv + 32 + (t & 31))) : 0.5f * __ldcg(sv + t);
+                reinterpret_cast<float*>(blk + kSpBytes)[t] = h;
+            }
+            named_barrier_sync(2, kNormThreads);
+            if (t == 0) signal_add(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrReady);
+        };
         for (int gt = 0;; ++gt) {
             const int s = gt % NS, use = gt / NS;
+            if (t == 0) fin_seen[gt & 1] = fin_head[0];
             // every thread learns the stage's chunk (or that there is none, or that a wait failed)
-            if (barrier_any(3, kNormThreads, !mbar_wait(&s_full[s], use & 1, abort_flag, prm.status, kBit))) break;
+            if (barrier_any(3, kNormThreads, dead || !mbar_wait(&s_full[s], use & 1, abort_flag, prm.status, kBit))) { dead = true; break; }
+            while (fin_done < fin_seen[gt & 1]) { finish_plane(fin_req[fin_done & 3]); ++fin_done; }
             const int info = s_info[s];
             if (info == kNoWork) { mbar_arrive(&s_scaled[s]); break; }  // passes the word on to the UMMA issuer
             const bool first = (info & 1) != 0, last = (info & 2) != 0;
@@ -538,33 +593,52 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             const int chunk = info >> 2, plane = chunk / prm.n_chunks;
             const int buf = (k_chunk - 1) & 1;
             bool ok = mbar_wait(&sacc_full[buf], ((k_chunk - 1) >> 1) & 1, abort_flag, prm.status, kBit);
-            if (k_chunk == 1) {
-                // the first sums of this CTA: every CTA must have cleared its part of the states by now
-                if (t == 0 && ok) ok = wait_counter(prm.ctr + kPipeCtrCleared, (unsigned)n_cta, abort_flag, prm.status);
-                ok = !barrier_any(3, kNormThreads, !ok);
-            }
-            if (ok) {
-                tcgen05_fence_after_sync();
-                float* dst = prm.state + (size_t)plane * kWords;
-                if (quarter < 3) {
-                    const int row = quarter * 32 + lane;
+            // the first sums of this CTA: every CTA must have cleared its part of the states by now
+            if (k_chunk == 1 && t == 0 && ok) ok = wait_counter(prm.ctr + kPipeCtrCleared, (unsigned)n_cta, abort_flag, prm.status);
+            if (barrier_any(2, kNormThreads, !ok)) { dead = true; continue; }  // everybody, or nobody
+            tcgen05_fence_after_sync();
+            float* dst = prm.state + (size_t)plane * kWords;
+            if (quarter < 3) {
+                const int row = quarter * 32 + lane;
 #pragma unroll
-                    for (int cc = 0; cc < kD / 16; ++cc) {
-                        float v[16];
-                        tmem_ld16(tmem_state + ((uint32_t)(quarter * 32) << 16) + buf * kD + cc * 16, v);
-                        tmem_ld_wait();
-                        if (row <= kD) {
-                            float* o4 = dst + row * kD + cc * 16;  // row 64 lands on s
+                for (int cc = 0; cc < kD / 16; ++cc) {
+                    float v[16];
+                    tmem_ld16(tmem_state + ((uint32_t)(quarter * 32) << 16) + buf * kD + cc * 16, v);
+                    tmem_ld_wait();
+                    if (row <= kD) {
+                        float* o4 = dst + row * kD + cc * 16;  // row 64 lands on s
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) red_add_f32x4(o4 + 4 * e, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-                        }
+                        for (int e = 0; e < 4; ++e) red_add_f32x4(o4 + 4 * e, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
                     }
                 }
-                tcgen05_fence_before_sync();
-                mbar_arrive(&sacc_free[buf]);
             }
-            if (barrier_any(3, kNormThreads, !ok)) break;
-            if (t == 0) signal_add(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrWritten);
+            tcgen05_fence_before_sync();
+            mbar_arrive(&sacc_free[buf]);
+            // the signalling thread counts the chunk, ordered after these additions
+            if (t == 0) sig_info[(k_chunk - 1) & 3] = plane;
+            named_barrier_sync(2, kNormThreads);
+            mbar_arrive(sig_bar);
+        }
+        if (!dead) {
+            // no more chunks: the signalling thread leaves after the last count; planes may still come up for finishing
+            if (t == 0) sig_info[k_chunk & 3] = kNoWork;
+            named_barrier_sync(2, kNormThreads);
+            mbar_arrive(sig_bar);
+            const unsigned long long t_start = global_ns();
+            while (true) {
+                if (t == 0) {
+                    const int left = fin_head[1];
+                    __threadfence_block();
+                    fin_seen[2] = fin_head[0]; fin_seen[3] = left;
+                    if (!left && (*abort_flag || global_ns() - t_start > kWaitLimitNs)) { fin_seen[3] = 2; *abort_flag = 1; atomicOr(prm.status, kBit); }
+                }
+                named_barrier_sync(2, kNormThreads);
+                const int seen = fin_seen[2], left = fin_seen[3];
+                named_barrier_sync(2, kNormThreads);
+                if (left != 2) while (fin_done < seen) { finish_plane(fin_req[fin_done & 3]); ++fin_done; }
+                if (left) break;
+                __nanosleep(200);
+            }
         }
     } else {
         // ================= apply pipeline: depthwise convolution =================
@@ -583,21 +657,15 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             const int bh = g / tpb;
             if (bh != prev_bh) {
                 prev_bh = bh;
-                if (__any_sync(0xffffffffu, !mbar_wait(p_ready, pseg & 1, abort_flag, prm.status, kBit))) break;
+                // the plane's 1/2 s arrives with its S'
+                if (__any_sync(0xffffffffu, !mbar_wait(&sp_full[pseg & 1], (pseg >> 1) & 1, abort_flag, prm.status, kBit))) break;
+                const float* hs = hs_s + (pseg & 1) * kD;
                 ++pseg;
                 // this lane's channel pair: 2*lane of 64 channels, or (PAIR) 2*(lane & 15) of 32 channels
                 // for the token of parity lane >> 4
                 const int cp2 = PAIR ? 2 * (lane & 15) : 2 * lane;
                 const int ch = ((prm.head0 + bh) % prm.H) * (PAIR ? 32 : kD) + cp2;
-                const float* sv = prm.state + (size_t)bh * kWords + kD * kD;
-                float s0, s1;
-                if (PAIR) {  // token sum = sum of the two halves of the paired sums
-                    s0 = __ldcg(sv + cp2) + __ldcg(sv + 32 + cp2);
-                    s1 = __ldcg(sv + cp2 + 1) + __ldcg(sv + 32 + cp2 + 1);
-                } else {
-                    s0 = __ldcg(sv + cp2); s1 = __ldcg(sv + cp2 + 1);
-                }
-                cinit.x = 0.5f * s0; cinit.y = 0.5f * s1;
+                cinit.x = hs[cp2]; cinit.y = hs[cp2 + 1];
                 if (prm.bias) { cinit.x += __bfloat162float(prm.bias[ch]); cinit.y += __bfloat162float(prm.bias[ch + 1]); }
 #pragma unroll
                 for (int dy = 0; dy < KS; ++dy)
@@ -615,7 +683,9 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             const int tok0 = PAIR ? 2 * (xh * kCX + G::HC) + (lane >> 4) - R : xh * kCX;
             const uint8_t* vh = stages + s * G::kStage + kQBytes + (RO * cw) * G::HX * 128 + tok0 * U +
                                 (PAIR ? (lane & 15) * 4 : lane * 4);
-            uint8_t* so = stg + b * kStgBytes + ((RO * cw) * kTX + xh * kCX) * kStgStride + lane * 8;
+            // fp32 rows of the staging buffer: 16-byte chunk c of patch token t at chunk c ^ (t & 7); t & 7 = x below
+            uint8_t* so = stg + b * kStgBytes + ((RO * cw) * kTX + xh * kCX) * kStgStride + (lane & 1) * 8;
+            const int sc = lane >> 1;
             float2 win[ROWS][KS];
 #pragma unroll
             for (int t = 0; t < KS - STEP; ++t)
@@ -646,7 +716,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                         for (int r = 0; r < RO; ++r)
                             acc[r] = ffma2(wreg[dy][dx], win[dy + r][(STEP * x + dx) % KS], acc[r]);
 #pragma unroll
-                for (int r = 0; r < RO; ++r) *reinterpret_cast<float2*>(so + (r * kTX + x) * kStgStride) = acc[r];
+                for (int r = 0; r < RO; ++r) *reinterpret_cast<float2*>(so + (r * kTX + x) * kStgStride + ((sc ^ x) << 4)) = acc[r];
             }
             mbar_arrive(&a_empty[s]);      // the V patch of this stage is no longer needed
             mbar_arrive(&conv_full[b]);
@@ -673,7 +743,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 }
 
 template <int KS, int MODE>
-cudaError_t launch_pipe_ks(const Problem& p, float* state, unsigned* ctr, unsigned* status, cudaStream_t st) {
+cudaError_t launch_pipe_ks(const Problem& p, float* state, float* ready, unsigned* ctr, unsigned* status, cudaStream_t st) {
     constexpr bool PAIR = (MODE == 1);
     using G = PGeo<KS, PAIR>;
     const bool pair = PAIR;
@@ -714,7 +784,7 @@ cudaError_t launch_pipe_ks(const Problem& p, float* state, unsigned* ctr, unsign
             return cudaErrorNotSupported;
     }
     PipeParams prm;
-    prm.state = state; prm.ctr = ctr;
+    prm.state = state; prm.ready = ready; prm.ctr = ctr;
     prm.w = static_cast<const __nv_bfloat16*>(p.w);
     prm.bias = static_cast<const __nv_bfloat16*>(p.bias);
     prm.flat = (rank == 4) ? 1 : 0;
@@ -743,7 +813,7 @@ cudaError_t launch_pipe_ks(const Problem& p, float* state, unsigned* ctr, unsign
 int planes_ahead(int BH, int rows) {
     const long long budget = 40ll << 20;
     long long ahead = budget / ((long long)(rows < 1 ? 1 : rows) * 128);
-    if (ahead < 1) ahead = 1;
+    if (ahead < 2) ahead = 2;  // at least two: a CTA finishes plane p between two of its chunks, and the next may belong to plane p + 1
     return (int)(ahead < BH ? ahead : BH);
 }
 
@@ -769,20 +839,22 @@ PipePlan plan_pipe(int BH, int rows, int cols, int gridH) {
     return pl;
 }
 
+size_t pipe_ready_words(int BH) { return (size_t)(BH < 0 ? 0 : BH) * kReadyWords; }
+
 bool pipe_supports(const Problem& p) {
     const bool pair = (p.d == 32);
     return plan_pipe(p.BH, pair ? p.N / 2 : p.N, pair ? p.gridW / 2 : p.gridW, p.gridH).ok;
 }
 
-cudaError_t launch_pipe(const Problem& p, float* state, unsigned* ctr, unsigned* status, cudaStream_t st) {
+cudaError_t launch_pipe(const Problem& p, float* state, float* ready, unsigned* ctr, unsigned* status, cudaStream_t st) {
     if (p.d == 32)
-        return p.ksize == 3 ? launch_pipe_ks<3, 1>(p, state, ctr, status, st)
-                            : launch_pipe_ks<5, 1>(p, state, ctr, status, st);
+        return p.ksize == 3 ? launch_pipe_ks<3, 1>(p, state, ready, ctr, status, st)
+                            : launch_pipe_ks<5, 1>(p, state, ready, ctr, status, st);
     if (p.blockdiag)
-        return p.ksize == 3 ? launch_pipe_ks<3, 2>(p, state, ctr, status, st)
-                            : launch_pipe_ks<5, 2>(p, state, ctr, status, st);
-    return p.ksize == 3 ? launch_pipe_ks<3, 0>(p, state, ctr, status, st)
-                        : launch_pipe_ks<5, 0>(p, state, ctr, status, st);
+        return p.ksize == 3 ? launch_pipe_ks<3, 2>(p, state, ready, ctr, status, st)
+                            : launch_pipe_ks<5, 2>(p, state, ready, ctr, status, st);
+    return p.ksize == 3 ? launch_pipe_ks<3, 0>(p, state, ready, ctr, status, st)
+                        : launch_pipe_ks<5, 0>(p, state, ready, ctr, status, st);
 }
 
 }  // namespace tc
