@@ -191,6 +191,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     volatile int* sig_info = s_info + 4;     // [4] plane of the k-th chunk this CTA has summed (slot k & 3), or kNoWork
     volatile int* fin_req = sig_info + 4;    // [4] planes whose sums are complete and that this CTA is to finish (slot i & 3)
     volatile int* fin_head = fin_req + 4;    // [2] number of such requests so far; 1 when the signalling thread has left
+    volatile int* sig_tail = fin_head + 6;   // [2] chunk counts the signalling thread has taken over; planes finished by the norm warps
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_cta = (int)gridDim.x, cta = (int)blockIdx.x;
@@ -205,7 +206,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             mbar_init(&sacc_full[b], 1); mbar_init(&sacc_free[b], kNormThreads);
         }
         mbar_init(&sp_full[0], 1); mbar_init(&sp_full[1], 1); mbar_init(sig_bar, kNormThreads);
-        fin_head[0] = 0; fin_head[1] = 0;
+        fin_head[0] = 0; fin_head[1] = 0; sig_tail[0] = 0; sig_tail[1] = 0;
         for (int s = 0; s < NS; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_scaled[s], kNormThreads); mbar_init(&s_empty[s], 1); }
         *abort_flag = 0;
         for (int i = 0; i < 8; ++i) applied_s[i] = 0;
@@ -385,10 +386,13 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             for (int k = 0;; ++k) {
                 if (!mbar_wait(sig_bar, k & 1, abort_flag, prm.status, kBit)) break;
                 const int plane = sig_info[k & 3];
+                __threadfence_block();
+                sig_tail[0] = k + 1;  // the norm warps complete the barrier's next phase only after this
                 if (plane == kNoWork) break;
                 const unsigned old = signal_add_fetch(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrWritten);
                 if (old == (unsigned)prm.n_chunks - 1u) {
                     const int h = fin_head[0];
+                    for (uint32_t spin = 0; h - sig_tail[1] >= 4 && spin < (1u << 22) && !*abort_flag; ++spin) __nanosleep(100);
                     fin_req[h & 3] = plane;
                     __threadfence_block();
                     fin_head[0] = h + 1;
@@ -548,7 +552,7 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 reinterpret_cast<float*>(blk + kSpBytes)[t] = h;
             }
             named_barrier_sync(2, kNormThreads);
-            if (t == 0) signal_add(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrReady);
+            if (t == 0) { signal_add(plane_ctr + (size_t)plane * kPipeCtrPerPlane + kPipeCtrReady); sig_tail[1] = sig_tail[1] + 1; }
         };
         for (int gt = 0;; ++gt) {
             const int s = gt % NS, use = gt / NS;
@@ -614,14 +618,21 @@ tc_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             }
             tcgen05_fence_before_sync();
             mbar_arrive(&sacc_free[buf]);
-            // the signalling thread counts the chunk, ordered after these additions
-            if (t == 0) sig_info[(k_chunk - 1) & 3] = plane;
+            // the signalling thread counts the chunk, ordered after these additions; it has to have seen the previous
+            // phase of its barrier complete before this one may (a waiter can be one phase behind, not two)
+            if (t == 0) {
+                for (uint32_t spin = 0; sig_tail[0] < k_chunk - 1 && spin < (1u << 22) && !*abort_flag; ++spin) __nanosleep(100);
+                sig_info[(k_chunk - 1) & 3] = plane;
+            }
             named_barrier_sync(2, kNormThreads);
             mbar_arrive(sig_bar);
         }
         if (!dead) {
             // no more chunks: the signalling thread leaves after the last count; planes may still come up for finishing
-            if (t == 0) sig_info[k_chunk & 3] = kNoWork;
+            if (t == 0) {
+                for (uint32_t spin = 0; sig_tail[0] < k_chunk && spin < (1u << 22) && !*abort_flag; ++spin) __nanosleep(100);
+                sig_info[k_chunk & 3] = kNoWork;
+            }
             named_barrier_sync(2, kNormThreads);
             mbar_arrive(sig_bar);
             const unsigned long long t_start = global_ns();
