@@ -251,16 +251,22 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int i = tid + j * kThreads;
                 if (i < kWords4) acc[j] = __ldcg(base + (size_t)first * kWords4 + i);
             }
-            for (int m = 1; m < members; ++m) {
-                float4 v[kIter];
+            // every load of the group is issued before the first addition (one trip to L2, not one per member);
+            // the additions keep the members' order
+            float4 v[kGroup - 1][kIter];
+#pragma unroll
+            for (int m = 1; m < kGroup; ++m)
 #pragma unroll
                 for (int j = 0; j < kIter; ++j) {
                     const int i = tid + j * kThreads;
-                    if (i < kWords4) v[j] = __ldcg(base + (size_t)(first + m) * kWords4 + i);
+                    v[m - 1][j] = (m < members && i < kWords4) ? __ldcg(base + (size_t)(first + m) * kWords4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
-                for (int j = 0; j < kIter; ++j) { acc[j].x += v[j].x; acc[j].y += v[j].y; acc[j].z += v[j].z; acc[j].w += v[j].w; }
-            }
+            for (int m = 1; m < kGroup; ++m)
+#pragma unroll
+                for (int j = 0; j < kIter; ++j) {
+                    if (m < members) { acc[j].x += v[m - 1][j].x; acc[j].y += v[m - 1][j].y; acc[j].z += v[m - 1][j].z; acc[j].w += v[m - 1][j].w; }
+                }
 #pragma unroll
             for (int j = 0; j < kIter; ++j) {
                 const int i = tid + j * kThreads;
@@ -283,15 +289,22 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const int i = tid + j * kThreads;
             if (i < kWords4) acc[j] = __ldcg(base + i);
         }
-        for (int g = 1; g < n_groups; ++g) {
-            float4 v[kIter];
+        for (int g0 = 1; g0 < n_groups; g0 += 4) {  // four groups per trip to L2, added in the groups' order
+            float4 v[4][kIter];
 #pragma unroll
-            for (int j = 0; j < kIter; ++j) {
-                const int i = tid + j * kThreads;
-                if (i < kWords4) v[j] = __ldcg(base + (size_t)g * kGroup * kWords4 + i);
-            }
+            for (int u = 0; u < 4; ++u)
 #pragma unroll
-            for (int j = 0; j < kIter; ++j) { acc[j].x += v[j].x; acc[j].y += v[j].y; acc[j].z += v[j].z; acc[j].w += v[j].w; }
+                for (int j = 0; j < kIter; ++j) {
+                    const int i = tid + j * kThreads;
+                    v[u][j] = (g0 + u < n_groups && i < kWords4) ? __ldcg(base + (size_t)(g0 + u) * kGroup * kWords4 + i)
+                                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int j = 0; j < kIter; ++j) {
+                    if (g0 + u < n_groups) { acc[j].x += v[u][j].x; acc[j].y += v[u][j].y; acc[j].z += v[u][j].z; acc[j].w += v[u][j].w; }
+                }
         }
 #pragma unroll
         for (int j = 0; j < kIter; ++j) {
