@@ -38,11 +38,33 @@ UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "c5_sweep_bf16:3"
 L2_BYTES = 126 * 1000 * 1000  # a workload under twice this is timed over a ring of buffer sets
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
-# one ncu capture of this command at full size (profiles/tc_kernels_c5_sweep.md); None for workloads
-# or kernels without a capture of the current code.
-NCU_TRAFFIC_BYTES = {("c5_sweep_bf16:3", "tc_apply"): 252.5e6 + 98.8e6,
-                     ("c3_deit_base_bf16", "tc_fused"): 57.9e6 + 1.8e6}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from one ncu
+# capture, with the summary file and the last commit that touched that kernel's source when it was taken.
+# bench.py reports the figure only while `git log` still names that commit as the kernel's latest: after
+# any later change to the kernel the counters are stale and `traffic` is null.
+NCU_TRAFFIC = {
+    ("c5_sweep_bf16:3", "tc_apply"): {"bytes": 252.5e6 + 98.8e6, "profile": "profiles/tc_kernels_c5_sweep.md",
+                                      "source": "paper_2211_10526_b200/csrc/tc_apply.cu", "commit": "d209734"},
+    ("c3_deit_base_bf16", "tc_fused"): {"bytes": 57.9e6 + 1.8e6, "profile": "profiles/tc_fused_c3_deit_base.md",
+                                        "source": "paper_2211_10526_b200/csrc/tc_fused.cu", "commit": "d209734"},
+}
+REPEATS = 5          # timed repeats; the median is reported
+MIN_FORWARDS = 100   # forwards per repeat, at least
+
+
+def ncu_traffic(workload: str, kernel: str):
+    """(bytes per launch or None, where the figure comes from)."""
+    ent = NCU_TRAFFIC.get((workload, kernel))
+    if ent is None:
+        return None, "no capture of this kernel on this workload"
+    try:
+        head = subprocess.run(["git", "-C", ROOT, "log", "-1", "--format=%h", "--", ent["source"]],
+                              capture_output=True, text=True, timeout=10).stdout.strip()
+    except Exception:
+        head = ""
+    if head and head[:7] != ent["commit"][:7]:
+        return None, f"{ent['profile']} was captured at {ent['commit']}; {ent['source']} last changed at {head}"
+    return ent["bytes"], f"{ent['profile']} (captured at {ent['commit']})"
 
 
 def parse_args():
@@ -290,22 +312,28 @@ def main():
             step(i)
         torch.cuda.synchronize()
 
-    # ---- timed region: K forwards, device time between two events on the launching stream ----
+    # ---- timed region: REPEATS repeats of max(K, MIN_FORWARDS) forwards each, device time between two events
+    # on the launching stream, maximum over the ranks per repeat; the median repeat is the reported one.  The
+    # clock sampler runs across all repeats.
+    n_fwd = max(args.steps, MIN_FORWARDS)
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.25)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier(world)
-    torch.cuda.synchronize()
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    barrier(world)
-    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    rep_ms = []
+    for _ in range(REPEATS):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier(world)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(n_fwd):
+            step(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world)
+        rep_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev) / n_fwd)
     clocks = sampler.stop()
-    ms_per_step = ms_total / args.steps
+    rep_sorted = sorted(rep_ms)
+    ms_per_step = rep_sorted[len(rep_sorted) // 2]
     value = world * s.image_tokens / (ms_per_step * 1e-3)
 
     # ---- per-kernel durations: same loop with events between the kernels (not part of `value`) ----
@@ -329,8 +357,9 @@ def main():
     if top is not None:
         achieved = alg[top] / (kernels[top] * 1e-3) / 1e9
         path_gbs = s.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
+        traffic, traffic_src = ncu_traffic(args.workload, top)
         roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get((args.workload, top)),
+                    "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_src,
                     "traffic_unit": "bytes per launch, ncu", "peak_source": peak_src,
                     "kernel_ms": kernels, "path_achieved": path_gbs, "path_frac": path_gbs / peak,
                     "path_frac_of_8000": path_gbs / 8000.0}
@@ -347,10 +376,18 @@ def main():
         for _ in range(n_e2e):
             attn.forward_host(*host, s.gridH, s.gridW, out=out_h, stream=stream.cuda_stream)
         dt = max_over_ranks(time.perf_counter() - t0, world, dev)
+        # the end-to-end result against the device-path result of the same inputs (the chunked pipeline splits
+        # the token sums differently, so the two agree to rounding, not bit for bit)
+        step(0)
+        torch.cuda.synchronize()
+        ref_o = ring[0][3].float().cpu()
+        e2e_err = float((out_h.float() - ref_o).abs().max() / ref_o.abs().max().clamp_min(1e-30))
+        if not e2e_err <= (2e-2 if s.dtype == "bf16" else 1e-5):
+            raise SystemExit(f"end-to-end output differs from the device-path output: max-rel {e2e_err:.3e}")
         h2d = sum(t.numel() * t.element_size() for t in host)
         e2e = {"value": world * s.image_tokens * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": out_h.numel() * out_h.element_size(), "steps": n_e2e,
-               "ms_per_step": 1e3 * dt / n_e2e}
+               "ms_per_step": 1e3 * dt / n_e2e, "max_rel_diff_vs_device_path": e2e_err}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -372,7 +409,9 @@ def main():
                        "parallelism": "independent replicas" if world > 1 else "single GPU",
                        "arithmetic": "bf16 tensor-core operands, fp32 accumulation" if s.dtype == "bf16" else "fp32",
                        "kernel_path": {1: "cuda-core", 2: "tensor-core"}.get(path, str(path))},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "timing": {"repeats": REPEATS, "forwards_per_repeat": n_fwd, "ms_per_step_min": rep_sorted[0],
+                       "ms_per_step_median": ms_per_step, "ms_per_step_max": rep_sorted[-1]},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * n_fwd * REPEATS,
             "roofline": roofline, "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)

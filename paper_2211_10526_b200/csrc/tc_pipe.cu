@@ -1,24 +1,26 @@
-// Whole forward pass of the tensor-core path as ONE persistent kernel for long sequences (bf16; width-64
-// heads, or width-32 heads packed two to a 128-byte row):
+// Whole forward pass of the tensor-core path as ONE persistent kernel (bf16; width-64 heads, or width-32
+// heads packed two to a 128-byte row), an alternative to the separate state and apply kernels:
 //     S = sum_n k^_n^T v_n,  s = sum_n v_n            (state, per (b,h))
 //     out_t = (1/pi) q^_t S + 1/2 s + bias + DWConv(V)_t                              (Eq. 9)
-// One CTA per multiprocessor, launched cooperatively so that all CTAs are resident.  The planes (one per
-// (b,h)) are taken in order, and every CTA takes a share of every plane, in two pipelines that run side by
-// side in different warps:
-//   state pipeline   warp 2 (TMA: K and V tiles of 64 rows), warp 3 (UMMAs, A = [K^ ; 1 0 0 ...] so that
-//                    accumulator row 64 is the token sum of V), warps 12..15 (scale every K row by
-//                    1 / max(||k||, eps) in place; write this CTA's sums over its rows of the plane to memory
-//                    and count them)
-//   apply pipeline   warp 0 (TMA: Q patch and V patch with halo), warp 1 (UMMAs: acc = Q S'), conv warps
-//                    (depthwise convolution of the V patch on CUDA cores, lane = channel pair; result plus
-//                    1/2 s and the bias staged in shared memory as fp32), warps 4..11 (||q||, accumulator row
-//                    scaled by 1/||q|| plus the staged row, one rounding to bf16, patch stored with TMA)
-// The sums of the CTAs are added up by the apply pipelines, which have to wait for them anyway: when all
-// CTAs have written their sums of a plane, CTA c adds slice c of the state words over all CTAs (in a fixed
-// order: the result does not depend on timing) and counts its slice; when all slices are counted the
-// plane's state is final.  A CTA adds its slice of the next plane early, when it enters a plane, so that
-// nobody has to wait for a slow CTA at the plane after.  The state pipeline never waits for another CTA's
-// sums; it only keeps a bounded number of planes ahead of the apply pipeline, so that the V rows the
+// One CTA per multiprocessor, launched cooperatively so that all CTAs are resident.  Every CTA runs two
+// pipelines side by side, in different warps, and takes its work from two counters in global memory, in plane
+// order (a plane is one (b,h)): chunks of rows for the state pipeline, patches of the token grid for the
+// apply pipeline.  A slower multiprocessor simply takes fewer.
+//   state pipeline   warp 2 (claims chunks; TMA: K and V tiles of 64 rows), warp 3 lane 0 (UMMAs, A = [K^ ; 1 0 0 ...]
+//                    so that accumulator row 64 is the token sum of V), warps 12..15 (scale every K row by
+//                    1 / max(||k||, eps) in place; add the chunk's sums to the plane's state in memory with
+//                    vector atomics), warp 3 lane 1 (counts the chunk once its sums are on their way)
+//   apply pipeline   warp 0 (claims patches; TMA: Q patch and V patch with halo; per plane S' and 1/2 s), warp 1
+//                    (UMMAs: acc = Q S'), conv warps (depthwise convolution of the V patch on CUDA cores, lane =
+//                    channel pair; result plus 1/2 s and the bias staged in shared memory as fp32), warps 4..11
+//                    (||q||, accumulator row scaled by 1/||q|| plus the staged row, one rounding to bf16, patch
+//                    stored with TMA)
+// The CTA that counts the last chunk of a plane finishes it: its norm warps turn the sums into the bf16
+// operand image S' = S / pi and 1/2 s, write both to memory and raise the plane's flag; the apply producers of
+// all CTAs wait for that flag when they first take a patch of the plane and copy the block into shared memory.
+// The states are cleared by the kernel itself.  The sums of a plane are added in the order the chunks happen
+// to finish, so the result varies in the last bits from run to run (the separate kernels add in a fixed order).
+// The state pipeline keeps a bounded number of planes ahead of the apply pipeline, so that the V rows the
 // apply pipeline needs were read moments ago and are served from L2: V comes from HBM once.
 // Flags are polled by one thread per CTA (many pollers on one address queue up at its L2 slice and slow every
 // other access to that slice); the other threads sleep on a shared-memory barrier that thread completes.
