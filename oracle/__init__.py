@@ -46,6 +46,14 @@ def _declare(lib: ctypes.CDLL) -> ctypes.CDLL:
     lib.castling_oracle_forward_bruteforce.argtypes = [_dp] * 6 + [i] * 6 + [dbl]
     lib.castling_oracle_similarity.restype = i
     lib.castling_oracle_similarity.argtypes = [_dp] * 3 + [i, i, dbl]
+    lib.castling_oracle_forward_rownorm.restype = i
+    lib.castling_oracle_forward_rownorm.argtypes = [_dp] * 6 + [i] * 7 + [dbl, i, i]
+    lib.castling_oracle_attention_weights.restype = i
+    lib.castling_oracle_attention_weights.argtypes = [_dp] * 3 + [i, i, dbl, i, i, i, dbl]
+    lib.castling_oracle_forward_matrix.restype = i
+    lib.castling_oracle_forward_matrix.argtypes = [_dp] * 6 + [i] * 6 + [dbl, i, i, i, dbl, i, i]
+    lib.castling_oracle_softmax_probs.restype = i
+    lib.castling_oracle_softmax_probs.argtypes = [_dp] * 3 + [i, i, dbl]
     lib.castling_oracle_angular_exact.restype = dbl
     lib.castling_oracle_angular_exact.argtypes = [dbl]
     lib.castling_oracle_angular_series.restype = dbl
@@ -164,3 +172,77 @@ def angular_series(x: float, kmax: int) -> float:
 def angular_series_coeff(k: int) -> float:
     """Eq. 8's coefficient (2k)! / (2^(2k) (k!)^2 (2k+1))."""
     return load().castling_oracle_angular_series_coeff(int(k))
+
+
+def _threaded(run, BH: int, threads: int, what: str) -> None:
+    threads = max(1, min(int(threads), BH))
+    if threads == 1:
+        rcs = [run(0, BH)]
+    else:
+        cuts = [BH * t // threads for t in range(threads + 1)]
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            rcs = list(pool.map(lambda ab: run(*ab), zip(cuts[:-1], cuts[1:])))
+    if any(rcs):
+        raise RuntimeError(f"{what} failed")
+
+
+def forward_rownorm(q, k, v, dw_weight, dw_bias, gridH: int, gridW: int, ksize: int,
+                    eps: float = DEFAULT_EPS, threads: int = 1, lib: Optional[ctypes.CDLL] = None,
+                    prefix: int = 0) -> np.ndarray:
+    """The core with every row of attention weights divided by its sum (Eq. 3's denominator applied to
+    the kept kernel of Eq. 8), linear in the number of tokens; the convolution is added unchanged."""
+    lib = lib or load()
+    q, k, v, w = _f64(q), _f64(k), _f64(v), _f64(dw_weight)
+    bias = None if dw_bias is None else _f64(dw_bias)
+    B, H, N, d = _check_shapes(q, k, v, w, bias, gridH, gridW, ksize, prefix)
+    out = np.empty_like(q)
+    _threaded(lambda lo, hi: lib.castling_oracle_forward_rownorm(
+        _ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(bias), _ptr(out), B, H, int(prefix), gridH, gridW, d, ksize,
+        float(eps), lo, hi), B * H, threads, "castling_oracle_forward_rownorm")
+    return out
+
+
+KERNEL_LINEAR, KERNEL_EXACT = 0, 1
+
+
+def attention_weights(q, k, kernel: int = KERNEL_LINEAR, rownorm: bool = False, sparse_eps: Optional[float] = None,
+                      eps: float = DEFAULT_EPS, lib: Optional[ctypes.CDLL] = None) -> np.ndarray:
+    """Explicit [N,N] attention weights of one head (q, k: [N,d]): the kept kernel of Eq. 8 or the exact
+    angular kernel of Eq. 5, optionally with rows divided by their sums, optionally plus the masked softmax
+    of Eq. 10 with threshold ``sparse_eps``."""
+    lib = lib or load()
+    q, k = _f64(q), _f64(k)
+    N, d = q.shape
+    wts = np.empty((N, N), dtype=np.float64)
+    rc = lib.castling_oracle_attention_weights(_ptr(q), _ptr(k), _ptr(wts), N, d, float(eps), int(kernel), int(bool(rownorm)),
+                                               int(sparse_eps is not None), float(sparse_eps or 0.0))
+    if rc:
+        raise RuntimeError("castling_oracle_attention_weights failed")
+    return wts
+
+
+def forward_matrix(q, k, v, dw_weight, dw_bias, gridH: int, gridW: int, ksize: int, kernel: int = KERNEL_LINEAR,
+                   rownorm: bool = False, sparse_eps: Optional[float] = None, eps: float = DEFAULT_EPS,
+                   threads: int = 1, lib: Optional[ctypes.CDLL] = None) -> np.ndarray:
+    """weights . V + DWConv(V) with the explicit weight matrix of ``attention_weights``; O(N^2 d) per head."""
+    lib = lib or load()
+    q, k, v, w = _f64(q), _f64(k), _f64(v), _f64(dw_weight)
+    bias = None if dw_bias is None else _f64(dw_bias)
+    B, H, N, d = _check_shapes(q, k, v, w, bias, gridH, gridW, ksize)
+    out = np.empty_like(q)
+    _threaded(lambda lo, hi: lib.castling_oracle_forward_matrix(
+        _ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(bias), _ptr(out), B, H, gridH, gridW, d, ksize, float(eps),
+        int(kernel), int(bool(rownorm)), int(sparse_eps is not None), float(sparse_eps or 0.0), lo, hi),
+        B * H, threads, "castling_oracle_forward_matrix")
+    return out
+
+
+def softmax_probs(q, k, eps: float = DEFAULT_EPS, lib: Optional[ctypes.CDLL] = None) -> np.ndarray:
+    """Softmax over the keys of the cosines of one head (q, k: [N,d]) -> [N,N]."""
+    lib = lib or load()
+    q, k = _f64(q), _f64(k)
+    N, d = q.shape
+    p = np.empty((N, N), dtype=np.float64)
+    if lib.castling_oracle_softmax_probs(_ptr(q), _ptr(k), _ptr(p), N, d, float(eps)):
+        raise RuntimeError("castling_oracle_softmax_probs failed")
+    return p

@@ -281,3 +281,177 @@ int castling_oracle_similarity(const double* q, const double* k, double* sim, in
     free(qh); free(kh);
     return 0;
 }
+
+/* ==== variants of the attention beyond the inference-time core ==================================
+ *
+ * (a) Row-sum normalisation.  Kernel-based linear attention as Sec. 3.1 states it (Eq. 3) divides
+ *     row t by phi(Q_t) . sum_j phi(K_j), i.e. by the sum of that row's similarities; Eq. 9 prints
+ *     no such denominator, so the core above has none.  With the kept kernel of Eq. 8 the row sum
+ *     is  sum_j (1/2 + q^_t.k^_j/pi) = T/2 + q^_t . (sum_j k^_j)/pi  over the T tokens of the
+ *     sequence, and the normalised attention term is A_t divided by it.  The depthwise convolution
+ *     is added afterwards, unchanged.
+ * (b) The exact angular kernel, Sim = 1 - arccos(q^.k^)/pi (Eq. 4-5), in place of its kept part.
+ * (c) The auxiliary branch of training, Mask_eps(Softmax_j(q^_t . k^_j)) (Eq. 10, Sec. 3.2.2),
+ *     Mask_eps(x) = x if x > eps else 0, added to the attention weights.  Readings taken: the
+ *     softmax runs over the keys of one query, on the cosines of the unit rows (Sec. 3.2.1, last
+ *     sentence: the normalisation is inserted into the sparse branch as well), without 1/sqrt(d)
+ *     (Eq. 10 has none) and without renormalising what survives the mask.
+ * (b) and (c) have no re-associated form: they are written with the explicit T x T weight matrix.
+ */
+
+/* (a), linear in the number of tokens.  prefix leading tokens are off the grid, as in
+ * castling_oracle_forward_prefix; prefix = 0 is the plain grid. */
+int castling_oracle_forward_rownorm(const double* q, const double* k, const double* v,
+                                    const double* w, const double* bias, double* out,
+                                    int B, int H, int prefix, int gridH, int gridW, int d, int ksize,
+                                    double eps, int bh_begin, int bh_end)
+{
+    if (!q || !k || !v || !w || !out) return -1;
+    if (B <= 0 || H <= 0 || prefix < 0 || gridH <= 0 || gridW <= 0 || d <= 0) return -1;
+    if (ksize <= 0 || (ksize & 1) == 0) return -1;
+    if (bh_begin < 0 || bh_end > B * H || bh_begin > bh_end) return -1;
+    const int G = gridH * gridW, T = prefix + G;
+    double* kv = (double*)malloc(sizeof(double) * d * d);     /* sum_j k^_j^T v_j */
+    double* vtot = (double*)malloc(sizeof(double) * d);       /* sum_j v_j        */
+    double* ktot = (double*)malloc(sizeof(double) * d);       /* sum_j k^_j       */
+    double* u = (double*)malloc(sizeof(double) * d);
+    double* gconv = (double*)malloc(sizeof(double) * (size_t)G * d);
+    if (!kv || !vtot || !ktot || !u || !gconv) { free(kv); free(vtot); free(ktot); free(u); free(gconv); return -1; }
+
+    for (int bh = bh_begin; bh < bh_end; ++bh) {
+        const int h = bh % H;
+        const size_t base = (size_t)bh * T * d;
+        const double* qp = q + base; const double* kp = k + base; const double* vp = v + base;
+        double* op = out + base;
+        memset(kv, 0, sizeof(double) * d * d);
+        memset(vtot, 0, sizeof(double) * d);
+        memset(ktot, 0, sizeof(double) * d);
+        for (int m = 0; m < T; ++m) {
+            unit_row(kp + (size_t)m * d, d, eps, u);
+            for (int a = 0; a < d; ++a) {
+                ktot[a] += u[a];
+                for (int c = 0; c < d; ++c) kv[a * d + c] += u[a] * vp[(size_t)m * d + c];
+            }
+            for (int c = 0; c < d; ++c) vtot[c] += vp[(size_t)m * d + c];
+        }
+        const double* vgrid = vp + (size_t)prefix * d;        /* the convolution sees the grid tokens only */
+        dwconv_head(vgrid, w, bias, h, gridH, gridW, d, ksize, gconv);
+        for (int m = 0; m < T; ++m) {
+            unit_row(qp + (size_t)m * d, d, eps, u);
+            double rowsum = 0.5 * T;                           /* sum_j (1/2 + q^_m.k^_j/pi) */
+            for (int a = 0; a < d; ++a) rowsum += u[a] * ktot[a] / M_PI;
+            for (int c = 0; c < d; ++c) {
+                double num = 0.5 * vtot[c];
+                for (int a = 0; a < d; ++a) num += u[a] * kv[a * d + c] / M_PI;
+                const double on_grid = (m >= prefix) ? gconv[(size_t)(m - prefix) * d + c] : 0.0;
+                op[(size_t)m * d + c] = num / rowsum + on_grid;
+            }
+        }
+    }
+    free(kv); free(vtot); free(ktot); free(u); free(gconv);
+    return 0;
+}
+
+/* The explicit weight matrix of one head, weights[t][j], T x T, for (a)-(c):
+ *   kernel   0: 1/2 + x/pi (Eq. 8, kept part);  1: 1 - arccos(x)/pi (Eq. 5);  x = q^_t . k^_j
+ *   rownorm  != 0: every row of that is divided by its sum (Eq. 3)
+ *   sparse   != 0: Mask_sparse_eps(Softmax_j(x)) (Eq. 10) is added afterwards */
+int castling_oracle_attention_weights(const double* q, const double* k, double* weights, int T, int d,
+                                      double eps, int kernel, int rownorm, int sparse, double sparse_eps)
+{
+    if (!q || !k || !weights || T <= 0 || d <= 0 || kernel < 0 || kernel > 1) return -1;
+    double* qu = (double*)malloc(sizeof(double) * (size_t)T * d);
+    double* ku = (double*)malloc(sizeof(double) * (size_t)T * d);
+    double* cosine = (double*)malloc(sizeof(double) * T);
+    if (!qu || !ku || !cosine) { free(qu); free(ku); free(cosine); return -1; }
+    for (int t = 0; t < T; ++t) {
+        unit_row(q + (size_t)t * d, d, eps, qu + (size_t)t * d);
+        unit_row(k + (size_t)t * d, d, eps, ku + (size_t)t * d);
+    }
+    for (int t = 0; t < T; ++t) {
+        double* row = weights + (size_t)t * T;
+        double total = 0.0;
+        for (int j = 0; j < T; ++j) {
+            double x = 0.0;
+            for (int i = 0; i < d; ++i) x += qu[(size_t)t * d + i] * ku[(size_t)j * d + i];
+            cosine[j] = x;
+            if (kernel == 0) {
+                row[j] = 0.5 + x / M_PI;
+            } else {
+                const double xc = x > 1.0 ? 1.0 : (x < -1.0 ? -1.0 : x);   /* rounding may leave [-1, 1] */
+                row[j] = castling_oracle_angular_exact(xc);
+            }
+            total += row[j];
+        }
+        if (rownorm)
+            for (int j = 0; j < T; ++j) row[j] /= total;
+        if (sparse) {
+            double z = 0.0;
+            for (int j = 0; j < T; ++j) z += exp(cosine[j]);
+            for (int j = 0; j < T; ++j) {
+                const double p = exp(cosine[j]) / z;
+                if (p > sparse_eps) row[j] += p;
+            }
+        }
+    }
+    free(qu); free(ku); free(cosine);
+    return 0;
+}
+
+/* out = weights . V + DWConv(V) with the weight matrix above; grid tokens only (no leading tokens).
+ * O(T^2 d) per head. */
+int castling_oracle_forward_matrix(const double* q, const double* k, const double* v,
+                                   const double* w, const double* bias, double* out,
+                                   int B, int H, int gridH, int gridW, int d, int ksize, double eps,
+                                   int kernel, int rownorm, int sparse, double sparse_eps,
+                                   int bh_begin, int bh_end)
+{
+    if (!q || !k || !v || !w || !out) return -1;
+    if (B <= 0 || H <= 0 || gridH <= 0 || gridW <= 0 || d <= 0) return -1;
+    if (ksize <= 0 || (ksize & 1) == 0) return -1;
+    if (bh_begin < 0 || bh_end > B * H || bh_begin > bh_end) return -1;
+    const int T = gridH * gridW;
+    double* wt = (double*)malloc(sizeof(double) * (size_t)T * T);
+    double* conv = (double*)malloc(sizeof(double) * (size_t)T * d);
+    if (!wt || !conv) { free(wt); free(conv); return -1; }
+    int rc = 0;
+    for (int bh = bh_begin; bh < bh_end && rc == 0; ++bh) {
+        const int h = bh % H;
+        const size_t base = (size_t)bh * T * d;
+        rc = castling_oracle_attention_weights(q + base, k + base, wt, T, d, eps, kernel, rownorm, sparse, sparse_eps);
+        if (rc) break;
+        dwconv_head(v + base, w, bias, h, gridH, gridW, d, ksize, conv);
+        for (int t = 0; t < T; ++t)
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int j = 0; j < T; ++j) acc += wt[(size_t)t * T + j] * v[base + (size_t)j * d + c];
+                out[base + (size_t)t * d + c] = acc + conv[(size_t)t * d + c];
+            }
+    }
+    free(wt); free(conv);
+    return rc;
+}
+
+/* Softmax_j(q^_t . k^_j) of one head, T x T: lets a test pick a mask threshold that lies in a gap
+ * of these values, so that the comparison with an fp32 implementation does not hinge on ties. */
+int castling_oracle_softmax_probs(const double* q, const double* k, double* probs, int T, int d, double eps)
+{
+    if (!q || !k || !probs || T <= 0 || d <= 0) return -1;
+    double* qu = (double*)malloc(sizeof(double) * d);
+    double* ku = (double*)malloc(sizeof(double) * (size_t)T * d);
+    if (!qu || !ku) { free(qu); free(ku); return -1; }
+    for (int j = 0; j < T; ++j) unit_row(k + (size_t)j * d, d, eps, ku + (size_t)j * d);
+    for (int t = 0; t < T; ++t) {
+        unit_row(q + (size_t)t * d, d, eps, qu);
+        double z = 0.0;
+        for (int j = 0; j < T; ++j) {
+            double x = 0.0;
+            for (int i = 0; i < d; ++i) x += qu[i] * ku[(size_t)j * d + i];
+            probs[(size_t)t * T + j] = exp(x);
+            z += exp(x);
+        }
+        for (int j = 0; j < T; ++j) probs[(size_t)t * T + j] /= z;
+    }
+    free(qu); free(ku);
+    return 0;
+}

@@ -404,11 +404,125 @@ def pin_prefix_tokens(lib):
     _close(oracle.forward(q, k, v, w, b, gh, gw, ks, lib=lib, prefix=P, threads=3), full, 0.0)
 
 
+def _worked_inputs():
+    q = np.array([[3.0, 4.0], [0.0, 2.0]]).reshape(1, 1, 2, 2)
+    k = np.array([[1.0, 0.0], [0.0, -5.0]]).reshape(1, 1, 2, 2)
+    v = np.array([[1.0, 2.0], [3.0, 4.0]]).reshape(1, 1, 2, 2)
+    w = np.array([[[9, 9, 9], [0.5, 1, 2], [9, 9, 9]], [[7, 7, 7], [-1, 0, 1], [7, 7, 7]]], dtype=np.float64)
+    return q, k, v, w, np.array([0.25, -0.5])
+
+
+def pin_variants_worked_example(lib):
+    """The 1 x 2 instance under row normalisation (Eq. 3), the exact kernel (Eq. 5) and the masked softmax
+    branch (Eq. 10): tests/golden/worked_example_1x2_variants.txt."""
+    q, k, v, w, b = _worked_inputs()
+    expect = {}
+    for name, t, c, val in _rows("worked_example_1x2_variants.txt"):
+        expect.setdefault(name, np.zeros((2, 2)))[int(t), int(c)] = float(val)
+    _close(oracle.forward_rownorm(q, k, v, w, b, 1, 2, 3, lib=lib)[0, 0], expect["rownorm"], 1e-14)
+    _close(oracle.forward_matrix(q, k, v, w, b, 1, 2, 3, rownorm=True, lib=lib)[0, 0], expect["rownorm"], 1e-14)
+    _close(oracle.forward_matrix(q, k, v, w, b, 1, 2, 3, kernel=oracle.KERNEL_EXACT, lib=lib)[0, 0], expect["exact"], 1e-14)
+    _close(oracle.forward_matrix(q, k, v, w, b, 1, 2, 3, sparse_eps=0.25, lib=lib)[0, 0], expect["sparse_0.25"], 1e-14)
+
+
+def pin_rownorm(lib):
+    """Eq. 3's denominator on the kept kernel: rows of the explicit weights sum to 1, so a constant V passes
+    through the attention term exactly; the linear form equals the explicit one, with and without leading
+    tokens; without the denominator the matrix form is the brute-force core."""
+    q, k, v, w, b = _problem(2, 3, 5, 4, 6, 3, 201)
+    wts = oracle.attention_weights(q[1, 2], k[1, 2], rownorm=True, lib=lib)
+    _close(wts.sum(axis=1), np.ones(20), 1e-13)
+    raw = oracle.attention_weights(q[1, 2], k[1, 2], lib=lib)
+    _close(raw, 0.5 + (_unit(q[1, 2]) @ _unit(k[1, 2]).T) / PI, 1e-13)
+    _close(wts, raw / raw.sum(axis=1, keepdims=True), 1e-13)
+    _close(oracle.forward_rownorm(q, k, v, w, b, 5, 4, 3, lib=lib), oracle.forward_matrix(q, k, v, w, b, 5, 4, 3, rownorm=True, lib=lib), 1e-12)
+    _close(oracle.forward_matrix(q, k, v, w, b, 5, 4, 3, lib=lib), oracle.forward_bruteforce(q, k, v, w, b, 5, 4, 3, lib=lib), 1e-13)
+    # constant V: the attention term returns the constant, whatever q and k are
+    c = np.array([1.5, -2.0, 0.25, 3.0, -0.5, 7.0])
+    vc = np.broadcast_to(c, v.shape).copy()
+    w0, b0 = _zero_filter(3, 6, 3)
+    _close(oracle.forward_rownorm(q, k, vc, w0, b0, 5, 4, 3, lib=lib), vc, 1e-13)
+    # explicit numpy evaluation of the whole variant, conv from the plain core with K = 0 (cosines 0, state 0)
+    qh, kh = _unit(q), _unit(k)
+    sim = 0.5 + np.einsum("bhtd,bhjd->bhtj", qh, kh) / PI
+    att = np.einsum("bhtj,bhjd->bhtd", sim / sim.sum(axis=-1, keepdims=True), v)
+    conv = oracle.forward(q, np.zeros_like(k), v, w, b, 5, 4, 3, lib=lib) - 0.5 * v.sum(axis=2, keepdims=True)
+    _close(oracle.forward_rownorm(q, k, v, w, b, 5, 4, 3, lib=lib), att + conv, 1e-12)
+    # leading tokens: they count in the row sums and the state, and get no convolution
+    P = 2
+    qp, kp, vp = (np.concatenate([_rand((2, 3, P, 6), 210 + i), t], axis=2) for i, t in enumerate((q, k, v)))
+    simp = 0.5 + np.einsum("bhtd,bhjd->bhtj", _unit(qp), _unit(kp)) / PI
+    attp = np.einsum("bhtj,bhjd->bhtd", simp / simp.sum(axis=-1, keepdims=True), vp)
+    got = oracle.forward_rownorm(qp, kp, vp, w, b, 5, 4, 3, lib=lib, prefix=P)
+    _close(got[:, :, :P], attp[:, :, :P], 1e-12)
+    _close(got[:, :, P:], attp[:, :, P:] + conv, 1e-12)
+    _close(oracle.forward_rownorm(q, k, v, w, b, 5, 4, 3, lib=lib, threads=3), oracle.forward_rownorm(q, k, v, w, b, 5, 4, 3, lib=lib), 0.0)
+
+
+def pin_exact_kernel_attention(lib):
+    """Eq. 4-5 as attention weights: 1 - arccos(cosine)/pi from numpy's arccos; aligned / orthogonal / opposite
+    rows give 1, 1/2, 0; the difference to the kept kernel is the odd high-order part of Eq. 8's series."""
+    q, k, v, w, b = _problem(1, 2, 4, 4, 5, 3, 221)
+    cos = np.clip(_unit(q[0, 1]) @ _unit(k[0, 1]).T, -1.0, 1.0)
+    ex = oracle.attention_weights(q[0, 1], k[0, 1], kernel=oracle.KERNEL_EXACT, lib=lib)
+    _close(ex, 1.0 - np.arccos(cos) / PI, 1e-13)
+    assert ex.min() >= 0.0 and ex.max() <= 1.0
+    lin = oracle.attention_weights(q[0, 1], k[0, 1], lib=lib)
+    resid = ex - lin
+    series = sum(oracle.angular_series_coeff(kk) * cos ** (2 * kk + 1) for kk in range(1, 400)) / PI
+    _close(resid, series, 1e-9)
+    # special rows
+    u = np.array([[2.0, 0.0, 0.0], [0.0, 3.0, 0.0], [-5.0, 0.0, 0.0]])
+    sp = oracle.attention_weights(np.repeat(u[:1], 3, axis=0), u, kernel=oracle.KERNEL_EXACT, lib=lib)
+    _close(sp[0], [1.0, 0.5, 0.0], 1e-15)
+    # whole forward = explicit numpy evaluation + the convolution of the plain core
+    full = oracle.forward_matrix(q, k, v, w, b, 4, 4, 3, kernel=oracle.KERNEL_EXACT, lib=lib)
+    cosb = np.clip(np.einsum("bhtd,bhjd->bhtj", _unit(q), _unit(k)), -1.0, 1.0)
+    conv = oracle.forward(q, np.zeros_like(k), v, w, b, 4, 4, 3, lib=lib) - 0.5 * v.sum(axis=2, keepdims=True)
+    _close(full, np.einsum("bhtj,bhjd->bhtd", 1.0 - np.arccos(cosb) / PI, v) + conv, 1e-12)
+    # d = 1: cosines are +-1, the weights 1 or 0: every query sums the values of the keys of its own sign
+    q1, k1, v1 = _rand((1, 1, 6, 1), 222), _rand((1, 1, 6, 1), 223), _rand((1, 1, 6, 1), 224)
+    w1, b1 = _zero_filter(1, 1, 3)
+    got = oracle.forward_matrix(q1, k1, v1, w1, b1, 2, 3, 3, kernel=oracle.KERNEL_EXACT, lib=lib)[0, 0, :, 0]
+    want = [sum(v1[0, 0, j, 0] for j in range(6) if np.sign(k1[0, 0, j, 0]) == np.sign(q1[0, 0, t, 0])) for t in range(6)]
+    _close(got, want, 1e-14)
+
+
+def pin_sparse_branch(lib):
+    """Eq. 10: the masked softmax over the cosines, added to the kept kernel.  A threshold of 1 or more masks
+    everything (the inference-time core, bit for bit); a negative threshold keeps everything (plain softmax
+    attention on unit rows, rows summing to 1); in between exactly the probabilities above it survive, unscaled."""
+    q, k, v, w, b = _problem(2, 2, 4, 5, 6, 3, 231)
+    base = oracle.forward_matrix(q, k, v, w, b, 4, 5, 3, lib=lib)
+    for thr in (1.0, 2.5):
+        assert np.array_equal(oracle.forward_matrix(q, k, v, w, b, 4, 5, 3, sparse_eps=thr, lib=lib), base)
+    cos = np.einsum("bhtd,bhjd->bhtj", _unit(q), _unit(k))
+    p = np.exp(cos) / np.exp(cos).sum(axis=-1, keepdims=True)
+    _close(oracle.softmax_probs(q[1, 0], k[1, 0], lib=lib), p[1, 0], 1e-14)
+    _close(oracle.softmax_probs(q[1, 0], k[1, 0], lib=lib).sum(axis=1), np.ones(20), 1e-14)
+    _close(oracle.forward_matrix(q, k, v, w, b, 4, 5, 3, sparse_eps=-1.0, lib=lib) - base, np.einsum("bhtj,bhjd->bhtd", p, v), 1e-12)
+    thr = 0.05  # p is about 1/20: some entries on either side
+    kept = p > thr
+    assert 0.1 < kept.mean() < 0.9
+    _close(oracle.forward_matrix(q, k, v, w, b, 4, 5, 3, sparse_eps=thr, lib=lib) - base,
+           np.einsum("bhtj,bhjd->bhtd", np.where(kept, p, 0.0), v), 1e-12)
+    # strictly greater: two identical keys have probability 1/2 each
+    qq = np.array([[1.0, 2.0], [3.0, -1.0]]); kk = np.array([[0.5, 0.5], [2.0, 2.0]])
+    wts_eq = oracle.attention_weights(qq, kk, sparse_eps=0.5, lib=lib) - oracle.attention_weights(qq, kk, lib=lib)
+    _close(wts_eq, np.zeros((2, 2)), 0.0)
+    wts_lt = oracle.attention_weights(qq, kk, sparse_eps=0.49, lib=lib) - oracle.attention_weights(qq, kk, lib=lib)
+    _close(wts_lt, np.full((2, 2), 0.5), 1e-15)
+    # the branch is added after the row normalisation, not inside it
+    wn = oracle.attention_weights(q[0, 0], k[0, 0], rownorm=True, sparse_eps=thr, lib=lib)
+    _close(wn, oracle.attention_weights(q[0, 0], k[0, 0], rownorm=True, lib=lib) + np.where(p[0, 0] > thr, p[0, 0], 0.0), 1e-13)
+
+
 PINS = [pin_worked_example, pin_series_coefficients, pin_angular_values, pin_series_properties,
         pin_bruteforce_equals_linear, pin_similarity_matrix, pin_constant_v, pin_equal_keys,
         pin_d_equals_one, pin_zero_rows, pin_conv_known_filters, pin_conv_head_channel_mapping,
         pin_conv_matrix_form, pin_conv_library_routine, pin_scale_invariance,
-        pin_linearity_and_symmetry, pin_threads_agree, pin_prefix_tokens]
+        pin_linearity_and_symmetry, pin_threads_agree, pin_prefix_tokens, pin_variants_worked_example,
+        pin_rownorm, pin_exact_kernel_attention, pin_sparse_branch]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -456,6 +570,21 @@ MISTAKES = [
     ("prefix_conv_row_offset", "grid_conv[(size_t)(m - prefix) * d + c] : 0.0;", "grid_conv[(size_t)(m - prefix + 1 < G ? m - prefix + 1 : 0) * d + c] : 0.0;", 1),
     ("prefix_half_term", "tok_sum[c] / 2.0 + dot / M_PI + on_grid;", "tok_sum[c] + dot / M_PI + on_grid;", 1),
     ("prefix_state_transposed", "dot += u[a] * state[a * d + c];", "dot += u[a] * state[c * d + a];", 1),
+    ("rownorm_counts_grid_only", "double rowsum = 0.5 * T;", "double rowsum = 0.5 * G;", 1),
+    ("rownorm_key_sum_not_normalised", "ktot[a] += u[a];", "ktot[a] += kp[(size_t)m * d + a];", 1),
+    ("rownorm_pi_missing", "rowsum += u[a] * ktot[a] / M_PI;", "rowsum += u[a] * ktot[a];", 1),
+    ("rownorm_divides_conv_too", "op[(size_t)m * d + c] = num / rowsum + on_grid;", "op[(size_t)m * d + c] = (num + on_grid) / rowsum;", 1),
+    ("rownorm_half_term", "double num = 0.5 * vtot[c];", "double num = vtot[c];", 1),
+    ("rownorm_state_transposed", "num += u[a] * kv[a * d + c] / M_PI;", "num += u[a] * kv[c * d + a] / M_PI;", 1),
+    ("matrix_rownorm_by_column", "for (int j = 0; j < T; ++j) row[j] /= total;", "for (int j = 0; j < T; ++j) row[j] /= (total - row[j] + row[t]);", 1),
+    ("matrix_exact_kernel_clamped_wrong", "const double xc = x > 1.0 ? 1.0 : (x < -1.0 ? -1.0 : x);", "const double xc = x > 0.5 ? 0.5 : (x < -1.0 ? -1.0 : x);", 1),
+    ("sparse_softmax_over_queries", "for (int j = 0; j < T; ++j) z += exp(cosine[j]);", "for (int j = 0; j < T; ++j) z += exp(cosine[t < T ? t : j]);", 1),
+    ("sparse_mask_not_strict", "if (p > sparse_eps) row[j] += p;", "if (p >= sparse_eps) row[j] += p;", 1),
+    ("sparse_mask_binary", "if (p > sparse_eps) row[j] += p;", "if (p > sparse_eps) row[j] += 1.0;", 1),
+    ("sparse_temperature", "const double p = exp(cosine[j]) / z;", "const double p = exp(2.0 * cosine[j]) / z;", 1),
+    ("matrix_weights_transposed", "acc += wt[(size_t)t * T + j] * v[base + (size_t)j * d + c];", "acc += wt[(size_t)j * T + t] * v[base + (size_t)j * d + c];", 1),
+    ("softmax_probs_unnormalised_keys", "for (int j = 0; j < T; ++j) unit_row(k + (size_t)j * d, d, eps, ku + (size_t)j * d);",
+     "memcpy(ku, k, sizeof(double) * (size_t)T * d);", 1),
 ]
 
 
