@@ -81,11 +81,26 @@ typedef struct {
                           /* convolution; here they enter both attention terms of Eq. 9 like any  */
                           /* token (they add to K^^T V and to the token sum, and get an output    */
                           /* row), while DWConv and its bias act on the grid tokens only.         */
+    /* Variants of the attention beyond the inference-time core; all zero selects the core.        */
+    int normalize_rows;   /* 1: every row of attention weights is divided by its sum, the denominator */
+                          /* of kernel-based linear attention (Sec. 3.1, Eq. 3) that Eq. 9 leaves out: */
+                          /* the attention term of token t is divided by N/2 + q^_t . (sum_j k^_j)/pi; */
+                          /* the convolution is added unchanged.  Runs on the CUDA-core kernels.      */
+    int exact_kernel;     /* 1: the exact angular kernel 1 - arccos(q^.k^)/pi (Eq. 4-5) instead of its  */
+                          /* kept part 1/2 + q^.k^/pi (Eq. 8).  Quadratic in N (explicit weights).     */
+    int sparse_branch;    /* 1: the auxiliary branch of training (Sec. 3.2.2, Eq. 10) is added to the   */
+                          /* weights: Mask_eps(Softmax_j(q^_t . k^_j)), Mask_eps(p) = p if p > eps else */
+                          /* 0; softmax over the keys of a query on the cosines of the unit rows, no    */
+                          /* 1/sqrt(d), survivors not renormalised.  Quadratic in N.  The comparison    */
+                          /* p > eps is taken in fp32.                                                 */
+    double sparse_eps;    /* the mask's threshold (the paper uses 0.02 for classification)             */
 } castling_attn_config_t;
 
 /*
  * castling_attn_create: make a handle bound to the CURRENT CUDA device.
- *   cfg         host pointer, read once; NULL selects {ksize 3, eps 1e-12, AUTO, no cap, no prefix}.
+ *   cfg         host pointer, read once; NULL selects {ksize 3, eps 1e-12, AUTO, no cap, no prefix, no variant}.
+ *               exact_kernel and sparse_branch take the explicit-weights kernel (any dtype and d, O(N^2 d)
+ *               time, at most 16384 tokens, no prefix tokens, contiguous or strided device tensors).
  *   out_handle  host pointer receiving the handle; set to NULL on failure.
  * Allocates nothing on the device.  Errors: INVALID_ARG, UNSUPPORTED (ksize), ARCH, CUDA.
  */

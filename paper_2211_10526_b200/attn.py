@@ -34,10 +34,14 @@ class CastlingAttn:
     """
 
     def __init__(self, ksize: int = 3, eps: float = 0.0, force_path: int = _b.PATH_AUTO, max_workspace: int = 0,
-                 prefix_tokens: int = 0):
+                 prefix_tokens: int = 0, normalize_rows: bool = False, exact_kernel: bool = False,
+                 sparse_eps: Optional[float] = None):
         self.ksize = int(ksize)
         self.prefix_tokens = int(prefix_tokens)  # leading off-grid (class) tokens: N = prefix_tokens + gridH * gridW
-        self._h = _b.castling_attn_create(ksize, eps, force_path, max_workspace, prefix_tokens)
+        # variants: rows of attention weights divided by their sums; the exact angular kernel; the masked
+        # softmax branch with threshold sparse_eps (None: off)
+        self._h = _b.castling_attn_create(ksize, eps, force_path, max_workspace, prefix_tokens, normalize_rows,
+                                          exact_kernel, sparse_eps)
 
     def close(self) -> None:
         if getattr(self, "_h", None):

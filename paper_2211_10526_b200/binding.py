@@ -23,7 +23,9 @@ STATIC_SCRATCH_BYTES = 4 << 20
 
 class castling_attn_config_t(ctypes.Structure):
     _fields_ = [("ksize", ctypes.c_int), ("eps", ctypes.c_double), ("force_path", ctypes.c_int),
-                ("max_workspace", ctypes.c_size_t), ("prefix_tokens", ctypes.c_int)]
+                ("max_workspace", ctypes.c_size_t), ("prefix_tokens", ctypes.c_int),
+                ("normalize_rows", ctypes.c_int), ("exact_kernel", ctypes.c_int), ("sparse_branch", ctypes.c_int),
+                ("sparse_eps", ctypes.c_double)]
 
 
 class castling_attn_layout_t(ctypes.Structure):
@@ -80,9 +82,13 @@ def error_string(code: int) -> str:
 
 
 def castling_attn_create(ksize: int = 3, eps: float = 0.0, force_path: int = PATH_AUTO,
-                         max_workspace: int = 0, prefix_tokens: int = 0) -> int:
-    """Returns the handle (an integer address); raises CastlingError on failure."""
-    cfg = castling_attn_config_t(int(ksize), float(eps), int(force_path), int(max_workspace), int(prefix_tokens))
+                         max_workspace: int = 0, prefix_tokens: int = 0, normalize_rows: bool = False,
+                         exact_kernel: bool = False, sparse_eps: Optional[float] = None) -> int:
+    """Returns the handle (an integer address); raises CastlingError on failure.  ``sparse_eps`` other than
+    None switches the masked softmax branch on with that threshold."""
+    cfg = castling_attn_config_t(int(ksize), float(eps), int(force_path), int(max_workspace), int(prefix_tokens),
+                                 int(bool(normalize_rows)), int(bool(exact_kernel)), int(sparse_eps is not None),
+                                 float(sparse_eps if sparse_eps is not None else 0.0))
     h = ctypes.c_void_p()
     rc = lib.castling_attn_create(ctypes.byref(cfg), ctypes.byref(h))
     if rc != OK:

@@ -50,11 +50,11 @@ size_t elem_bytes(castling_dtype_t t) { return t == CASTLING_F32 ? 4 : 2; }
 // header | state [BH] | partial [BH][P] (only when the token range is split)
 size_t workspace_words(int BH, int N, int d, bool bf16) {
     int P = castling::simt_choose_splits(BH, N);
-    size_t words = castling::state_words(d);
+    size_t words = castling::state_words_rownorm(d);  // the CUDA-core kernels' state, with room for the key-row sum
     if (bf16 && (d == 64 || d == 32)) {  // shapes the tensor-core kernels may take: they keep 64-wide states
         const int Pt = castling::tc::choose_splits(BH, castling::tc::rows_per_head(N, d));
         if (Pt > P) P = Pt;
-        words = castling::tc::kStateWords;
+        if (castling::tc::kStateWords > words) words = castling::tc::kStateWords;
     }
     size_t slots = (size_t)BH * (P > 1 ? P : 0);  // partial states behind the BH final ones
     if (bf16 && d == 32 && BH % 2 == 0) {
@@ -136,7 +136,7 @@ extern "C" {
 int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** out_handle) {
     if (!out_handle) return CASTLING_ERR_INVALID_ARG;
     *out_handle = nullptr;
-    castling_attn_config_t c = {3, 1e-12, CASTLING_PATH_AUTO, 0, 0};
+    castling_attn_config_t c = {3, 1e-12, CASTLING_PATH_AUTO, 0, 0, 0, 0, 0, 0.0};
     if (cfg) c = *cfg;
     if (c.eps <= 0.0) c.eps = 1e-12;
     if (c.ksize <= 0 || (c.ksize & 1) == 0) return CASTLING_ERR_INVALID_ARG;
@@ -144,6 +144,9 @@ int castling_attn_create(const castling_attn_config_t* cfg, castling_attn_t** ou
     if (c.force_path < CASTLING_PATH_AUTO || c.force_path > CASTLING_PATH_TENSOR) return CASTLING_ERR_INVALID_ARG;
     if (c.prefix_tokens < 0) return CASTLING_ERR_INVALID_ARG;
     if (c.prefix_tokens > 16) return CASTLING_ERR_UNSUPPORTED;
+    if ((c.normalize_rows | c.exact_kernel | c.sparse_branch) & ~1) return CASTLING_ERR_INVALID_ARG;
+    if ((c.exact_kernel || c.sparse_branch) && c.prefix_tokens > 0) return CASTLING_ERR_UNSUPPORTED;
+    if (c.sparse_branch && !(c.sparse_eps == c.sparse_eps)) return CASTLING_ERR_INVALID_ARG;  // NaN
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail_cuda(nullptr, e);
@@ -211,14 +214,29 @@ namespace {
 
 // Enqueue the kernels for one validated problem whose tensors are all on the device.
 int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
+    if (p.exact_kernel || p.sparse) {
+        // explicit attention weights: one kernel, no workspace; quadratic in the number of tokens
+        if (p.N > 16384) return CASTLING_ERR_UNSUPPORTED;
+        if (h->cfg.force_path == CASTLING_PATH_TENSOR) return CASTLING_ERR_UNSUPPORTED;
+        int launches = 0;
+        h->timer.begin(stream);
+        const cudaError_t e = castling::quad_forward(p, stream, &launches, &h->timer);
+        if (e == cudaErrorNotSupported) { (void)cudaGetLastError(); return CASTLING_ERR_UNSUPPORTED; }
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->last_path = CASTLING_PATH_SIMT;
+        h->last_launches = launches;
+        return CASTLING_OK;
+    }
     int rc = ensure_workspace(h, p.BH, p.N, p.d, p.bf16);
     if (rc != CASTLING_OK) return rc;
-    const bool tensor_ok = castling::tc::supports(p);
+    // the row-sum denominator needs the sum of the unit key rows, which only the CUDA-core kernels build
+    const bool tensor_ok = castling::tc::supports(p) && !p.rownorm;
     if (h->cfg.force_path == CASTLING_PATH_TENSOR && !tensor_ok) return CASTLING_ERR_UNSUPPORTED;
-    bool use_tensor = h->cfg.force_path == CASTLING_PATH_TENSOR ||
-                            (h->cfg.force_path == CASTLING_PATH_AUTO && castling::tc::preferred(p));
+    bool use_tensor = tensor_ok && (h->cfg.force_path == CASTLING_PATH_TENSOR ||
+                                    (h->cfg.force_path == CASTLING_PATH_AUTO && castling::tc::preferred(p)));
     float* state = h->ws + castling::kHeaderWords;
-    float* partial = state + (size_t)p.BH * (use_tensor ? (size_t)castling::tc::kStateWords : castling::state_words(p.d));
+    const size_t simt_words = p.rownorm ? castling::state_words_rownorm(p.d) : castling::state_words(p.d);
+    float* partial = state + (size_t)p.BH * (use_tensor ? (size_t)castling::tc::kStateWords : simt_words);
     int launches = 0;
     h->timer.begin(stream);
     cudaError_t e;
@@ -235,7 +253,7 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
         // the TMA descriptor could not be encoded for these strides: the CUDA-core kernels take any layout
         (void)cudaGetLastError();
         use_tensor = false;
-        partial = state + (size_t)p.BH * castling::state_words(p.d);
+        partial = state + (size_t)p.BH * simt_words;
         h->timer.begin(stream);
         e = castling::simt_forward(p, state, partial, castling::simt_choose_splits(p.BH, p.N), stream, &launches, &h->timer);
     }
@@ -255,6 +273,10 @@ Problem make_problem(const castling_attn* h, const void* q, const void* k, const
     p.N = p.prefix + gridH * gridW; p.BH = B * H; p.head0 = 0;
     p.bf16 = (dtype == CASTLING_BF16);
     p.eps2 = (float)(h->cfg.eps * h->cfg.eps);
+    p.rownorm = h->cfg.normalize_rows != 0;
+    p.exact_kernel = h->cfg.exact_kernel != 0;
+    p.sparse = h->cfg.sparse_branch != 0;
+    p.sparse_eps = (float)h->cfg.sparse_eps;
     p.set_contiguous();
     return p;
 }

@@ -42,6 +42,11 @@ struct Problem {
     bool blockdiag = false;  // tensor-core path only: a width-64 plane holds two independent width-32 heads side by
                              // side (heads h, h+1 of a layout whose head stride is 32): rows are normalised per
                              // half and only the two diagonal 32 x 32 blocks of the state are used
+    // Variants beyond the inference-time core (all off by default):
+    bool rownorm = false;       // every row of attention weights divided by its sum (Eq. 3's denominator)
+    bool exact_kernel = false;  // 1 - arccos(x)/pi (Eq. 4-5) instead of its kept part 1/2 + x/pi (Eq. 8)
+    bool sparse = false;        // plus Mask_eps(Softmax(q^ k^^T)) (Eq. 10)
+    float sparse_eps = 0.f;     // the mask's threshold
     int hdiv;          // planes per batch step of the layouts: H for a caller's strided tensors, BH for a
                        // run of contiguous planes (one uniform plane stride)
     // Contiguous [planes][N][d] tensors; needs N, d and BH.
@@ -60,6 +65,8 @@ struct Problem {
 constexpr size_t kHeaderWords = 64;
 
 inline size_t state_words(int d) { return (size_t)d * d + d; }
+// With row-sum normalisation the sum of the unit key rows follows: S, s, then sum_n k^_n (d more words).
+inline size_t state_words_rownorm(int d) { return (size_t)d * d + 2 * (size_t)d; }
 
 // Optional per-kernel timing: when `on`, an event is recorded on the stream before the first
 // kernel of a forward and after every kernel, so the host can read each kernel's duration.
@@ -106,6 +113,8 @@ int device_sm_count();
 cudaError_t simt_forward(const Problem& p, float* ws_state, float* ws_partial, int P,
                          cudaStream_t stream, int* launches, KernelTimer* timer);
 int simt_choose_splits(int BH, int N);
+// Explicit-weights forward (csrc/quad_kernels.cu): exact kernel and / or masked softmax branch; O(N^2 d).
+cudaError_t quad_forward(const Problem& p, cudaStream_t stream, int* launches, KernelTimer* timer);
 bool simt_supports(int d, int ksize);
 
 }  // namespace castling

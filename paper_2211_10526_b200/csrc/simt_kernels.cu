@@ -107,13 +107,14 @@ __device__ __forceinline__ void row_rnorm(const float* __restrict__ s, float* __
 
 // ---------------------------------------------------------------------------
 // state kernel: grid (BH * P).  CTA bh * P + p covers tokens [p*chunk, min(N,(p+1)*chunk)).
-// Writes raw sums [S (d*d, row i = key feature, col j = value feature) | s (d)].
+// Writes raw sums [S (d*d, row i = key feature, col j = value feature) | s (d)], `words` apart per split;
+// with zsum the sum of the unit key rows (d words) follows: the row-sum denominator of Eq. 3 needs it.
 // Thread (ti, tj) of a 16 x 16 arrangement owns an R x R block of S, R = D / 16.
 // ---------------------------------------------------------------------------
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 simt_state_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __restrict__ dst,
-                  int N, int chunk, int P, float eps2, Layout lk, Layout lv, int hdiv) {
+                  int N, int chunk, int P, float eps2, Layout lk, Layout lv, int hdiv, int words, int zsum) {
     constexpr int R = D / 16;
     constexpr int LD = D + 4;  // padded row, keeps 16-byte alignment
     __shared__ __align__(16) float ks[kStateTile * LD];
@@ -127,10 +128,10 @@ simt_state_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __res
     const int ti = threadIdx.x / 16, tj = threadIdx.x % 16;
 
     float acc[R][R];
-    float vsum[R];
+    float vsum[R], ksum[R];
 #pragma unroll
     for (int a = 0; a < R; ++a) {
-        vsum[a] = 0.f;
+        vsum[a] = 0.f; ksum[a] = 0.f;
 #pragma unroll
         for (int b = 0; b < R; ++b) acc[a][b] = 0.f;
     }
@@ -152,13 +153,14 @@ simt_state_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __res
 #pragma unroll
             for (int x = 0; x < R; ++x) {
                 vsum[x] += b[x];
+                ksum[x] += a[x];
 #pragma unroll
                 for (int y = 0; y < R; ++y) acc[x][y] = fmaf(a[x], b[y], acc[x][y]);
             }
         }
     }
 
-    float* out = dst + ((size_t)bh * P + p) * (D * D + D);
+    float* out = dst + ((size_t)bh * P + p) * words;
 #pragma unroll
     for (int x = 0; x < R; ++x)
 #pragma unroll
@@ -166,6 +168,10 @@ simt_state_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __res
     if (ti == 0) {
 #pragma unroll
         for (int y = 0; y < R; ++y) out[D * D + tj * R + y] = vsum[y];
+    }
+    if (zsum && tj == 0) {
+#pragma unroll
+        for (int x = 0; x < R; ++x) out[D * D + D + ti * R + x] = ksum[x];
     }
 }
 
@@ -187,7 +193,7 @@ simt_reduce_kernel(const float* __restrict__ partial, float* __restrict__ state,
 // Thread (tq, tj) owns tokens tq + 16 r (r = 0..3) and channels tj*R .. tj*R + R - 1.
 // ---------------------------------------------------------------------------
 template <int D> constexpr size_t simt_apply_smem(int ksize) {
-    return sizeof(float) * ((size_t)D * D + 2 * D + (size_t)ksize * ksize * D + kApplyTile * (D + 1) + kApplyTile);
+    return sizeof(float) * ((size_t)D * D + 3 * D + (size_t)ksize * ksize * D + kApplyTile * (D + 1) + 2 * kApplyTile);
 }
 
 template <typename T, int D>
@@ -195,7 +201,7 @@ __global__ void __launch_bounds__(kThreads)
 simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __restrict__ w,
                   const T* __restrict__ bias, const float* __restrict__ state, T* __restrict__ out,
                   int H, int head0, int prefix, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lv,
-                  Layout lo, int hdiv) {
+                  Layout lo, int hdiv, int words, int zsum) {
     constexpr int R = D / 16;
     constexpr int LDQ = D + 1;
     extern __shared__ __align__(16) float smem[];
@@ -206,17 +212,20 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
     float* w_sm = b_sm + D;             // [KK][D] filters of this head, tap-major
     float* qs = w_sm + KK * D;          // [64][D+1]
     float* rq = qs + kApplyTile * LDQ;  // [64]
+    float* rden = rq + kApplyTile;      // [64] 1 / (row sum of the similarities), or 1
+    float* z_sm = rden + kApplyTile;    // [D]  sum of the unit key rows (zsum only)
 
     const int N = prefix + gridH * gridW;
     const int tiles = (N + kApplyTile - 1) / kApplyTile;
     const int bh = blockIdx.x / tiles, h = (head0 + bh) % H;
     const int t0 = (blockIdx.x % tiles) * kApplyTile;
     const int valid = min(kApplyTile, N - t0);
-    const float* st = state + (size_t)bh * (D * D + D);
+    const float* st = state + (size_t)bh * words;
 
     for (int i = threadIdx.x; i < D * D; i += kThreads) S_sm[i] = st[i] * kInvPi;
     for (int i = threadIdx.x; i < D; i += kThreads) {
         c_sm[i] = 0.5f * st[D * D + i];
+        z_sm[i] = zsum ? st[D * D + D + i] : 0.f;
         b_sm[i] = bias ? Elem<T>::load1(bias + h * D + i) : 0.f;
     }
     for (int i = threadIdx.x; i < KK * D; i += kThreads) {
@@ -241,6 +250,17 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
     }
     __syncthreads();
     row_rnorm<D, LDQ, kApplyTile>(qs, rq, eps2);
+    __syncthreads();
+    if (threadIdx.x < kApplyTile) {
+        // Eq. 3's denominator for the kept kernel of Eq. 8: sum_j (1/2 + q^.k^_j/pi) = N/2 + q^ . (sum_j k^_j)/pi
+        float den = 1.0f;
+        if (zsum) {
+            float dot = 0.f;
+            for (int i = 0; i < D; ++i) dot = fmaf(qs[threadIdx.x * LDQ + i], z_sm[i], dot);
+            den = fmaf(dot * rq[threadIdx.x], kInvPi, 0.5f * (float)N);
+        }
+        rden[threadIdx.x] = 1.0f / den;
+    }
     __syncthreads();
 
     const int tq = threadIdx.x / 16, tj = threadIdx.x % 16;
@@ -270,10 +290,14 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
         const int tl = tq + 16 * r;
         if (tl >= valid) continue;
         const int t = t0 + tl, g = t - prefix, y = g / gridW, x = g % gridW;  // g < 0: an off-grid leading token
-        const float scale = rq[tl];
+        const float scale = rq[tl], inv_rowsum = rden[tl];
         float o[R];
 #pragma unroll
-        for (int c = 0; c < R; ++c) o[c] = fmaf(acc[r][c], scale, c_sm[tj * R + c] + (g >= 0 ? b_sm[tj * R + c] : 0.f));
+        for (int c = 0; c < R; ++c) {
+            // without the denominator: one rounding fewer, as before
+            o[c] = zsum ? fmaf(acc[r][c], scale, c_sm[tj * R + c]) * inv_rowsum + (g >= 0 ? b_sm[tj * R + c] : 0.f)
+                        : fmaf(acc[r][c], scale, c_sm[tj * R + c] + (g >= 0 ? b_sm[tj * R + c] : 0.f));
+        }
         for (int dy = -rad; dy <= rad && g >= 0; ++dy) {
             const int yy = y + dy;
             if (yy < 0 || yy >= gridH) continue;
@@ -447,7 +471,9 @@ simt_fused_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
 template <typename T, int D>
 cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, int P,
                         cudaStream_t stream, int* launches, KernelTimer* timer) {
-    if (p.N <= kFusedMaxTokens && p.BH >= kFusedMinPlanes && simt_fused_smem<D>(p.N, p.ksize) <= kFusedSmemLimit) {
+    const int zsum = p.rownorm ? 1 : 0;
+    const int words = D * D + D + (zsum ? D : 0);
+    if (!zsum && p.N <= kFusedMaxTokens && p.BH >= kFusedMinPlanes && simt_fused_smem<D>(p.N, p.ksize) <= kFusedSmemLimit) {
         const size_t smem = simt_fused_smem<D>(p.N, p.ksize);
         static PerDevice fused_opt_in;
         cudaError_t e = opt_in_smem(simt_fused_kernel<T, D>, kFusedSmemLimit, fused_opt_in);
@@ -465,13 +491,13 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     const int chunk = ((tiles + P - 1) / P) * kStateTile;
     float* dst = (P > 1) ? ws_partial : ws_state;
     simt_state_kernel<T, D><<<(unsigned)(p.BH * P), kThreads, 0, stream>>>(
-        static_cast<const T*>(p.k), static_cast<const T*>(p.v), dst, p.N, chunk, P, p.eps2, p.lk, p.lv, p.hdiv);
+        static_cast<const T*>(p.k), static_cast<const T*>(p.v), dst, p.N, chunk, P, p.eps2, p.lk, p.lv, p.hdiv, words, zsum);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     *launches = 1;
     timer->mark(stream, "simt_state");
     if (P > 1) {
-        simt_reduce_kernel<<<p.BH, kThreads, 0, stream>>>(ws_partial, ws_state, D * D + D, P);
+        simt_reduce_kernel<<<p.BH, kThreads, 0, stream>>>(ws_partial, ws_state, words, P);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         ++*launches;
@@ -485,7 +511,7 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     simt_apply_kernel<T, D><<<grid, kThreads, smem, stream>>>(
         static_cast<const T*>(p.q), static_cast<const T*>(p.v), static_cast<const T*>(p.w),
         static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.head0, p.prefix, p.gridH, p.gridW, p.ksize,
-        p.eps2, p.lq, p.lv, p.lo, p.hdiv);
+        p.eps2, p.lq, p.lv, p.lo, p.hdiv, words, zsum);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     timer->mark(stream, "simt_apply");

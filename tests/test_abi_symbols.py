@@ -44,8 +44,9 @@ def test_error_strings_and_workspace_query_need_no_gpu():
     texts = [b.error_string(c) for c in codes]
     assert len(set(texts)) == len(codes) and all(texts)
     assert "unknown" in b.error_string(-99)
-    # state + no partials for a small grid: header + BH * (d*d + d) floats
-    assert b.castling_attn_workspace_bytes(2, 4, 14, 14, 32, b.CASTLING_F32) == 4 * (64 + 8 * (32 * 32 + 32))
+    # state + no partials for a small grid: header + BH * (d*d + 2d) floats (S, s and room for the key-row sum
+    # of the row-normalised variant)
+    assert b.castling_attn_workspace_bytes(2, 4, 14, 14, 32, b.CASTLING_F32) == 4 * (64 + 8 * (32 * 32 + 2 * 32))
     # bf16 with d = 32 may run the tensor-core kernels, which keep 64-wide states
     assert b.castling_attn_workspace_bytes(2, 4, 14, 14, 32, b.CASTLING_BF16) >= 4 * (64 + 8 * (64 * 64 + 64))
     big = b.castling_attn_workspace_bytes(2, 8, 256, 256, 64, b.CASTLING_BF16)
@@ -93,9 +94,11 @@ def test_binding_structs_match_the_header_layout(tmp_path):
     src.write_text(
         '#include <stdio.h>\n#include <stddef.h>\n#include "castling_attn.h"\n'
         'int main(void) {\n'
-        '  printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(castling_attn_config_t), offsetof(castling_attn_config_t, ksize),\n'
+        '  printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(castling_attn_config_t), offsetof(castling_attn_config_t, ksize),\n'
         '         offsetof(castling_attn_config_t, eps), offsetof(castling_attn_config_t, force_path),\n'
-        '         offsetof(castling_attn_config_t, max_workspace), offsetof(castling_attn_config_t, prefix_tokens));\n'
+        '         offsetof(castling_attn_config_t, max_workspace), offsetof(castling_attn_config_t, prefix_tokens),\n'
+        '         offsetof(castling_attn_config_t, normalize_rows), offsetof(castling_attn_config_t, exact_kernel),\n'
+        '         offsetof(castling_attn_config_t, sparse_branch), offsetof(castling_attn_config_t, sparse_eps));\n'
         '  printf("%zu %zu %zu %zu\\n", sizeof(castling_attn_layout_t), offsetof(castling_attn_layout_t, q_batch),\n'
         '         offsetof(castling_attn_layout_t, v_head), offsetof(castling_attn_layout_t, out_token));\n'
         '  printf("%d %d %d %u\\n", CASTLING_ERR_SCRATCH_LIMIT, CASTLING_PATH_TENSOR, CASTLING_BF16, CASTLING_STATIC_SCRATCH_BYTES);\n'
@@ -105,6 +108,8 @@ def test_binding_structs_match_the_header_layout(tmp_path):
     lines = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
     cfg, lay = b.castling_attn_config_t, b.castling_attn_layout_t
     assert [int(x) for x in lines[0].split()] == [ctypes.sizeof(cfg), cfg.ksize.offset, cfg.eps.offset, cfg.force_path.offset,
-                                                 cfg.max_workspace.offset, cfg.prefix_tokens.offset]
+                                                 cfg.max_workspace.offset, cfg.prefix_tokens.offset,
+                                                 cfg.normalize_rows.offset, cfg.exact_kernel.offset, cfg.sparse_branch.offset,
+                                                 cfg.sparse_eps.offset]
     assert [int(x) for x in lines[1].split()] == [ctypes.sizeof(lay), lay.q_batch.offset, lay.v_head.offset, lay.out_token.offset]
     assert [int(x) for x in lines[2].split()] == [b.ERR_SCRATCH_LIMIT, b.PATH_TENSOR, b.CASTLING_BF16, b.STATIC_SCRATCH_BYTES]

@@ -1,0 +1,188 @@
+"""GPU parity of the variants of the attention beyond the inference-time core, against the CPU oracle:
+
+* rows of attention weights divided by their sums (Eq. 3's denominator on the kept kernel of Eq. 8),
+* the exact angular kernel of Eq. 4-5 in place of its kept part,
+* the masked softmax branch of training, Eq. 10,
+
+on the named configurations (the quadratic variants up to 4096 tokens, the size their kernel is meant for,
+and once at its limit of 16384), with the same bounds as the core: 1e-5 of the largest reference value for fp32,
+2e-2 for bf16.  The mask of Eq. 10 compares a probability with a threshold; the kernel does that in fp32 and the
+oracle in float64, so thresholds are placed in a gap of the oracle's probabilities wherever all of them can be
+listed (then no comparison is close); elsewhere a borderline probability may fall on either side, which moves an
+output by at most threshold * |v|, far inside the bf16 bound.
+"""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-2}
+
+
+def gpu_forward(c, layout="head_major", prefix=0, grid=None, **variant):
+    from paper_2211_10526_b200 import CastlingAttn
+    s = c.shape
+    gh, gw = grid if grid else (s.gridH, s.gridW)
+    dev = torch.device("cuda:0")
+    if layout == "head_major":
+        q, k, v = (t.to(dev) for t in (c.q, c.k, c.v))
+        out = torch.full_like(q, float("nan"))
+    else:
+        mk = lambda t: t.permute(0, 2, 1, 3).contiguous().to(dev).permute(0, 2, 1, 3)
+        q, k, v = mk(c.q), mk(c.k), mk(c.v)
+        out = torch.full((s.B, s.N, s.H, s.d), float("nan"), dtype=q.dtype, device=dev).permute(0, 2, 1, 3)
+    with CastlingAttn(ksize=s.ksize, prefix_tokens=prefix, **variant) as attn:
+        attn.forward(q, k, v, c.dw_weight.to(dev), c.dw_bias.to(dev), gh, gw, out=out)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+    got = out.double().cpu().numpy()
+    assert np.all(np.isfinite(got)), "an output element was never written"
+    return got
+
+
+def check(got, ref, dtype, what):
+    scale = float(np.max(np.abs(ref)))
+    err = float(np.max(np.abs(got - ref))) / scale
+    assert err <= TOL[dtype], f"{what}: max-rel error {err:.3e} (largest reference value {scale:.3g})"
+
+
+def gap_threshold(c, lo=0.1, hi=0.9, require=True):
+    """A threshold inside the widest gap between neighbouring softmax probabilities (all planes) in the middle of
+    their distribution: no probability is closer to it than half that gap.  With `require` the gap has to be
+    wide against fp32 rounding (the fp32 cases, whose bound a single borderline probability would break)."""
+    s = c.shape
+    ps = [oracle.softmax_probs(c.q[b, h], c.k[b, h]).ravel() for b in range(s.B) for h in range(s.H)]
+    p = np.sort(np.concatenate(ps))
+    a, b = int(lo * p.size), int(hi * p.size)
+    i = a + int(np.argmax(np.diff(p[a:b])))
+    thr = 0.5 * (p[i] + p[i + 1])
+    assert not require or (p[i + 1] - p[i]) / thr > 1e-5, "no usable gap"
+    return float(thr)
+
+
+CONFIG_CALLS = [("c1_fp32_tiny", 0), ("c2_levit_bf16", 0), ("c2_levit_bf16", 1), ("c2_levit_bf16", 2),
+                ("c3_deit_base_bf16", 0), ("c4_detection_bf16", 0), ("c5_sweep_bf16", 0), ("c5_sweep_bf16", 1),
+                ("c5_sweep_bf16", 2), ("c5_sweep_bf16", 3)]
+IDS = [f"{n}-{i}" for n, i in CONFIG_CALLS]
+
+
+@pytest.mark.parametrize("name,idx", CONFIG_CALLS, ids=IDS)
+def test_row_normalised_configurations(name, idx):
+    (c,) = list(workloads.iter_workload(name, only=[idx]))
+    s = c.shape
+    ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, threads=16)
+    check(gpu_forward(c, normalize_rows=True), ref, s.dtype, f"{s.label()} row-normalised")
+
+
+def test_row_normalised_attention_term_alone():
+    """Zero filters and bias: the output is the normalised attention term, a weighted mean of V, on its own scale."""
+    for dtype, shape in (("f32", (2, 3, 20, 24, 32, 3)), ("bf16", (2, 2, 48, 40, 64, 3))):
+        c = workloads.custom_call(*shape, dtype, seed=8100)
+        c.dw_weight.zero_(); c.dw_bias.zero_()
+        s = c.shape
+        ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, threads=8)
+        check(gpu_forward(c, normalize_rows=True), ref, dtype, f"{s.label()} normalised attention term")
+        # rows of weights sum to one: a constant V comes back
+        c.v[:] = 1.25
+        got = gpu_forward(c, normalize_rows=True)
+        assert np.max(np.abs(got - 1.25)) <= (2e-6 if dtype == "f32" else 1e-2)
+
+
+def test_row_normalised_with_leading_tokens_and_strides():
+    c = workloads.custom_call(2, 4, 1, 2 + 9 * 10, 32, 3, "f32", seed=8101)
+    ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, 9, 10, 3, prefix=2)
+    check(gpu_forward(c, prefix=2, grid=(9, 10), normalize_rows=True), ref, "f32", "leading tokens")
+    c = workloads.custom_call(2, 4, 12, 14, 64, 5, "bf16", seed=8102)
+    ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, 12, 14, 5)
+    check(gpu_forward(c, layout="token_major", normalize_rows=True), ref, "bf16", "token-major")
+
+
+QUAD_CALLS = [("c1_fp32_tiny", 0), ("c2_levit_bf16", 0), ("c2_levit_bf16", 1), ("c2_levit_bf16", 2),
+              ("c3_deit_base_bf16", 0), ("c4_detection_bf16", 0), ("c5_sweep_bf16", 0), ("c5_sweep_bf16", 1)]
+QUAD_IDS = [f"{n}-{i}" for n, i in QUAD_CALLS]
+
+
+@pytest.mark.parametrize("name,idx", QUAD_CALLS, ids=QUAD_IDS)
+def test_exact_angular_kernel_configurations(name, idx):
+    (c,) = list(workloads.iter_workload(name, only=[idx]))
+    s = c.shape
+    ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize,
+                                kernel=oracle.KERNEL_EXACT, threads=16)
+    check(gpu_forward(c, exact_kernel=True), ref, s.dtype, f"{s.label()} exact kernel")
+
+
+@pytest.mark.parametrize("name,idx", QUAD_CALLS, ids=QUAD_IDS)
+def test_sparse_branch_configurations(name, idx):
+    (c,) = list(workloads.iter_workload(name, only=[idx]))
+    s = c.shape
+    # a threshold that keeps about half of the probabilities (the paper's 0.02 masks everything on such inputs:
+    # with unit rows no probability exceeds e^2 / N); in a gap of all probabilities where they can be listed
+    thr = gap_threshold(c, require=(s.dtype == "f32")) if s.B * s.H * s.N * s.N <= 4_000_000 else 1.0 / s.N
+    ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, sparse_eps=thr, threads=16)
+    check(gpu_forward(c, sparse_eps=thr), ref, s.dtype, f"{s.label()} masked softmax branch, threshold {thr:.3e}")
+
+
+def test_castling_all_zero_mask_is_the_inference_core():
+    """With the paper's threshold the mask is empty on these inputs, and the explicit-weights kernel then computes
+    the inference-time core: same result as the oracle's linear form, and as the linear kernels to rounding."""
+    (c,) = list(workloads.iter_workload("c1_fp32_tiny", only=[0]))
+    s = c.shape
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize)
+    assert np.array_equal(oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, sparse_eps=0.02),
+                          oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize))
+    quad = gpu_forward(c, sparse_eps=0.02)
+    check(quad, ref, "f32", "empty mask")
+    check(quad, gpu_forward(c), "f32", "explicit weights against the linear kernels")
+
+
+def test_variant_terms_alone_fp32():
+    """The masked softmax term and the high-order residual of the exact kernel, each as the difference of two fp32
+    runs, on its own scale; thresholds in a gap of the probabilities."""
+    c = workloads.custom_call(2, 3, 16, 16, 32, 3, "f32", seed=8103)
+    s = c.shape
+    core = gpu_forward(c, sparse_eps=2.0)      # explicit weights, empty mask
+    thr = gap_threshold(c)
+    o = lambda **kw: oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, threads=6, **kw)
+    base = o()
+    for what, got, ref in (("masked softmax term", gpu_forward(c, sparse_eps=thr) - core, o(sparse_eps=thr) - base),
+                           ("plain softmax term", gpu_forward(c, sparse_eps=-1.0) - core, o(sparse_eps=-1.0) - base),
+                           ("high-order residual", gpu_forward(c, exact_kernel=True) - core, o(kernel=oracle.KERNEL_EXACT) - base)):
+        scale = float(np.max(np.abs(ref)))
+        err = float(np.max(np.abs(got - ref)))
+        # each run is good to 1e-5 of its own largest value, which is larger than this term's
+        assert err <= 2e-5 * float(np.max(np.abs(base))), f"{what}: {err:.3e} on a term of size {scale:.3g}"
+        assert err <= 5e-3 * scale, f"{what}: {err:.3e} on a term of size {scale:.3g}"
+
+
+def test_all_variants_together_and_limits():
+    from paper_2211_10526_b200 import CastlingAttn, binding as b
+    c = workloads.custom_call(2, 2, 16, 20, 48, 5, "f32", seed=8104)
+    s = c.shape
+    thr = gap_threshold(c)
+    ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, kernel=oracle.KERNEL_EXACT,
+                                rownorm=True, sparse_eps=thr)
+    check(gpu_forward(c, exact_kernel=True, normalize_rows=True, sparse_eps=thr), ref, "f32", "all variants")
+    ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, rownorm=True, sparse_eps=thr)
+    check(gpu_forward(c, normalize_rows=True, sparse_eps=thr), ref, "f32", "row sums and mask")
+    # leading tokens and the quadratic variants do not combine; nor do more than 16384 tokens
+    with pytest.raises(b.CastlingError):
+        CastlingAttn(prefix_tokens=1, exact_kernel=True)
+    dev = torch.device("cuda:0")
+    with CastlingAttn(exact_kernel=True) as attn:
+        t = torch.zeros(1, 1, 129 * 128, 32, dtype=torch.bfloat16, device=dev)
+        w, bias = torch.zeros(32, 3, 3, dtype=torch.bfloat16, device=dev), torch.zeros(32, dtype=torch.bfloat16, device=dev)
+        with pytest.raises(b.CastlingError):
+            attn.forward(t, t, t, w, bias, 129, 128, out=torch.empty_like(t))
+
+
+def test_exact_kernel_at_the_token_limit():
+    c = workloads.custom_call(1, 2, 128, 128, 32, 3, "bf16", seed=8105)
+    s = c.shape
+    ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, kernel=oracle.KERNEL_EXACT, threads=2)
+    check(gpu_forward(c, exact_kernel=True), ref, "bf16", "16384 tokens")
