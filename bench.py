@@ -77,6 +77,9 @@ def parse_args():
     ap.add_argument("--force-path", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     ap.add_argument("--layout", default="head_major", choices=["head_major", "token_major"],
                     help="memory layout of q, k, v, out: [B,H,N,d] contiguous, or [B,N,H,d] passed as strided views")
+    ap.add_argument("--repeats", type=int, default=REPEATS, help="timed repeats (the median is reported)")
+    ap.add_argument("--min-forwards", type=int, default=MIN_FORWARDS,
+                    help="forwards per repeat, at least; a profiler run passes 1 here and to --repeats")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -315,12 +318,12 @@ def main():
     # ---- timed region: REPEATS repeats of max(K, MIN_FORWARDS) forwards each, device time between two events
     # on the launching stream, maximum over the ranks per repeat; the median repeat is the reported one.  The
     # clock sampler runs across all repeats.
-    n_fwd = max(args.steps, MIN_FORWARDS)
+    n_fwd = max(args.steps, args.min_forwards)
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.25)
     rep_ms = []
-    for _ in range(REPEATS):
+    for _ in range(max(1, args.repeats)):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier(world)
         torch.cuda.synchronize()
@@ -409,9 +412,9 @@ def main():
                        "parallelism": "independent replicas" if world > 1 else "single GPU",
                        "arithmetic": "bf16 tensor-core operands, fp32 accumulation" if s.dtype == "bf16" else "fp32",
                        "kernel_path": {1: "cuda-core", 2: "tensor-core"}.get(path, str(path))},
-            "timing": {"repeats": REPEATS, "forwards_per_repeat": n_fwd, "ms_per_step_min": rep_sorted[0],
+            "timing": {"repeats": len(rep_ms), "forwards_per_repeat": n_fwd, "ms_per_step_min": rep_sorted[0],
                        "ms_per_step_median": ms_per_step, "ms_per_step_max": rep_sorted[-1]},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * n_fwd * REPEATS,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * n_fwd * len(rep_ms),
             "roofline": roofline, "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)
