@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC = {
     ("c5_sweep_bf16:3", "tc_apply"): {"bytes": 252.5e6 + 98.8e6, "profile": "profiles/tc_kernels_c5_sweep.md",
                                       "source": "paper_2211_10526_b200/csrc/tc_apply.cu", "commit": "d209734"},
-    ("c3_deit_base_bf16", "tc_fused"): {"bytes": 57.9e6 + 1.8e6, "profile": "profiles/tc_fused_c3_deit_base.md",
+    ("c3_deit_base_bf16", "tc_fused"): {"bytes": 57.9e6 + 2.0e6, "profile": "profiles/tc_fused_c3_deit_base.md",
                                         "source": "paper_2211_10526_b200/csrc/tc_fused.cu", "commit": "d209734"},
 }
 REPEATS = 5          # timed repeats; the median is reported
