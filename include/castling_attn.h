@@ -219,9 +219,22 @@ CASTLING_API int castling_attn_last_path(const castling_attn_t* handle, int* ker
 /*
  * castling_attn_device_status: read back the handle's device-side status word
  * (synchronises `stream`).  0 = every bounded wait in the kernels completed; otherwise
- * returns CASTLING_ERR_DEVICE and stores the raw word in *raw (may be NULL).
+ * returns CASTLING_ERR_DEVICE and stores the raw word in *raw (may be NULL); a non-zero word is
+ * reported once and cleared, together with the arrival counters a kernel may have left half way.
  */
 CASTLING_API int castling_attn_device_status(castling_attn_t* handle, void* stream, unsigned int* raw);
+
+/*
+ * castling_attn_selftest_wait: check the mechanism behind that status word without any fault.  Launches one
+ * small kernel on `stream` whose threads wait, with a limit of `limit_us` microseconds (1 .. 1 000 000), on a
+ * shared-memory barrier that nothing completes -- the situation of a pipeline whose copy or partner never
+ * arrives.  The wait must give up, raise a bit in the status word and let the kernel return; the call
+ * synchronises `stream` and returns CASTLING_OK when the kernel ran to its end that way.  Afterwards
+ * castling_attn_device_status reports CASTLING_ERR_DEVICE once (raw word 16) and clears the word; the handle
+ * stays usable.  May allocate the workspace header on first use.  (The paper has no counterpart: this
+ * verifies the failure behaviour of the kernels' bounded waits.)
+ */
+CASTLING_API int castling_attn_selftest_wait(castling_attn_t* handle, unsigned int limit_us, void* stream);
 
 /*
  * castling_attn_set_profiling: with enable != 0 every later forward on this handle records a

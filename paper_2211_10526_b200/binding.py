@@ -65,6 +65,8 @@ def _load() -> ctypes.CDLL:
     lib.castling_attn_last_path.argtypes = [vp, ctypes.POINTER(i)]
     lib.castling_attn_device_status.restype = i
     lib.castling_attn_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint)]
+    lib.castling_attn_selftest_wait.restype = i
+    lib.castling_attn_selftest_wait.argtypes = [vp, ctypes.c_uint, vp]
     lib.castling_attn_set_profiling.restype = i
     lib.castling_attn_set_profiling.argtypes = [vp, i]
     lib.castling_attn_kernel_times.restype = i
@@ -142,6 +144,11 @@ def castling_attn_device_status(handle, stream: int = 0):
     raw = ctypes.c_uint(0)
     rc = lib.castling_attn_device_status(handle, stream or None, ctypes.byref(raw))
     return rc, raw.value
+
+
+def castling_attn_selftest_wait(handle, limit_us: int = 2000, stream: int = 0) -> int:
+    """Runs the kernel whose bounded wait must give up; returns the C return code (OK when it did)."""
+    return lib.castling_attn_selftest_wait(handle, int(limit_us), stream or None)
 
 
 def castling_attn_set_profiling(handle, enable: bool) -> int:

@@ -466,9 +466,30 @@ int castling_attn_device_status(castling_attn_t* h, void* stream, unsigned int* 
         if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(h, e);
     }
     if (raw) *raw = word;
-    if (word && h->counters)  // a kernel that gave up may have left arrival counters half way
-        cudaMemset(h->counters, 0, h->counters_cap * sizeof(unsigned));
+    if (word) {
+        // reported once: the word is cleared, and so are arrival counters that a kernel which gave up may have
+        // left half way
+        cudaMemset(h->ws, 0, sizeof(unsigned));
+        if (h->counters) cudaMemset(h->counters, 0, h->counters_cap * sizeof(unsigned));
+    }
     return word ? CASTLING_ERR_DEVICE : CASTLING_OK;
+}
+
+int castling_attn_selftest_wait(castling_attn_t* h, unsigned int limit_us, void* stream) {
+    if (!h || limit_us == 0 || limit_us > 1000000u) return CASTLING_ERR_INVALID_ARG;
+    int rc = ensure_workspace(h, 1, 64, 64, true);  // the status word lives at the head of the workspace
+    if (rc != CASTLING_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned* status = reinterpret_cast<unsigned*>(h->ws);
+    unsigned* reached = status + 1;  // header word 1 is free
+    cudaError_t e = cudaMemsetAsync(reached, 0, sizeof(unsigned), st);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    e = castling::tc::launch_selftest_wait(status, (unsigned long long)limit_us * 1000ull, reached, st);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    unsigned end = 0;
+    if ((e = cudaMemcpyAsync(&end, reached, sizeof(end), cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_cuda(h, e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail_cuda(h, e);
+    return end == 1u ? CASTLING_OK : CASTLING_ERR_DEVICE;  // 1: the kernel ran to its end after the wait gave up
 }
 
 int castling_attn_set_profiling(castling_attn_t* h, int enable) {

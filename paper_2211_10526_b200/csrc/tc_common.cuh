@@ -15,6 +15,7 @@ enum : unsigned {
     kStatusApplyTimeout = 1u << 1,
     kStatusFusedTimeout = 1u << 2,
     kStatusPipeTimeout = 1u << 3,
+    kStatusSelfTestTimeout = 1u << 4,
 };
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait, then give up
@@ -61,7 +62,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // global status word and the CTA's abort flag, if the wait outlasts kWaitLimitNs or another
 // thread of the CTA has already given up; the caller then leaves its loop for the common exit.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned* status, unsigned bit) {
+                                          unsigned* status, unsigned bit, unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     uint32_t spins = 0;
@@ -69,7 +70,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 255u) == 0) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            if (global_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicOr(status, bit);
                 return false;

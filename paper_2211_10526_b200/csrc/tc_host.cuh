@@ -77,6 +77,10 @@ cudaError_t launch_pipe(const Problem& p, float* state, float* ready, unsigned* 
 bool fused_supports(const Problem& p);
 cudaError_t launch_fused(const Problem& p, unsigned* status, cudaStream_t st);
 
+// A one-CTA kernel whose bounded wait (limit_ns) can never be satisfied: it has to raise kStatusSelfTestTimeout in
+// *status and return; *reached_end becomes 1 (2 if the wait claimed success).
+cudaError_t launch_selftest_wait(unsigned* status, unsigned long long limit_ns, unsigned* reached_end, cudaStream_t st);
+
 }  // namespace tc
 
 // Shared with the CUDA-core path: sums P partial states per (b,h) in index order.

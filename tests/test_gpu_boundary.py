@@ -287,3 +287,33 @@ def test_forward_inside_a_cuda_graph(shape):
     assert np.all(np.isfinite(g))
     err = float(np.max(np.abs(g - ref)) / np.max(np.abs(ref)))
     assert err <= (1e-5 if dtype == "f32" else 2e-2), err
+
+
+def test_bounded_wait_gives_up_and_the_handle_stays_usable():
+    """A wait that can never be satisfied (a barrier nothing completes) runs into its limit, the kernel returns,
+    the status word reports it once as CASTLING_ERR_DEVICE, and a forward on the same handle is correct after."""
+    import time
+    import workloads
+    from paper_2211_10526_b200 import CastlingAttn, binding as b
+    dev = torch.device("cuda:0")
+    c = workloads.custom_call(2, 2, 24, 20, 64, 3, "bf16", seed=910)
+    s = c.shape
+    ref = oracle.forward(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize)
+    args = tuple(t.to(dev) for t in (c.q, c.k, c.v, c.dw_weight, c.dw_bias))
+    with CastlingAttn(ksize=3) as attn:
+        out = attn.forward(*args, s.gridH, s.gridW)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+        t0 = time.perf_counter()
+        assert b.castling_attn_selftest_wait(attn.handle, 3000) == b.OK     # 3 ms limit
+        waited = time.perf_counter() - t0
+        assert 0.002 <= waited < 1.0, waited                                 # it did wait, and it did stop
+        rc, raw = attn.device_status()
+        assert rc == b.ERR_DEVICE and raw == 16
+        assert attn.device_status() == (0, 0)                                # reported once, then cleared
+        assert b.castling_attn_selftest_wait(attn.handle, 0) == b.ERR_INVALID_ARG
+        out = attn.forward(*args, s.gridH, s.gridW)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+    err = float(np.max(np.abs(out.double().cpu().numpy() - ref)) / np.max(np.abs(ref)))
+    assert err <= 2e-2
