@@ -225,6 +225,39 @@ CASTLING_API int castling_attn_last_path(const castling_attn_t* handle, int* ker
 CASTLING_API int castling_attn_device_status(castling_attn_t* handle, void* stream, unsigned int* raw);
 
 /*
+ * A forward whose token grid is cut into bands of rows held by different devices ("sequence sharding").  The
+ * paper's complexity paragraph (Sec. 3.2.1) is what makes this cheap: everything the keys and values of the
+ * whole sequence contribute to Eq. 9 is the d x d matrix K^^T V and the token sum of V, so the devices exchange
+ * B*H*(d*d + d) floats, not tokens; the depthwise convolution needs the (ksize-1)/2 grid rows on either side
+ * of a band from its neighbours.  The library does the two local halves; the caller sums the states over the
+ * devices in between (one all-reduce) and supplies the neighbour rows of V.
+ *
+ * castling_attn_state_words(d) = d*d + d: floats per (b,h) of a state: S row-major [key feature][value
+ * feature], then the token sum s.  Raw sums: the states of the bands of one sequence simply add up.
+ *
+ * castling_attn_shard_state: this band's sums.
+ *   k, v        DEVICE, [B, H, n_tokens, d] contiguous: the band's tokens (their grid position does not matter).
+ *   state_out   DEVICE, float [B*H][d*d + d], overwritten.
+ * castling_attn_shard_apply: the band's output rows from a state summed over all bands.
+ *   q, out      DEVICE, [B, H, gridH_local*gridW, d] contiguous: the band's queries / outputs.
+ *   v_halo      DEVICE, [B, H, (halo_top + gridH_local + halo_bottom)*gridW, d]: the band's rows of V preceded by
+ *               the last halo_top rows of the band above and followed by the first halo_bottom rows of the band
+ *               below; each of the two is 0 at the edge of the whole grid (zero padding applies there) and at
+ *               most (ksize-1)/2, and must be (ksize-1)/2 wherever a neighbouring band exists.
+ *   state       DEVICE, float [B*H][d*d + d]: the sum over all bands of what castling_attn_shard_state wrote.
+ * Both enqueue on `stream` and return (the first call of a larger shape may allocate the workspace).  They run
+ * on the CUDA-core kernels for every dtype.  A handle created with prefix tokens or any variant flag:
+ * UNSUPPORTED.  Pointers 16-byte aligned.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, OOM, CUDA.
+ */
+CASTLING_API size_t castling_attn_state_words(int d);
+CASTLING_API int castling_attn_shard_state(castling_attn_t* handle, const void* k, const void* v, float* state_out,
+                          int B, int H, int n_tokens, int d, castling_dtype_t dtype, void* stream);
+CASTLING_API int castling_attn_shard_apply(castling_attn_t* handle, const void* q, const void* v_halo,
+                          const void* dw_weight, const void* dw_bias, const float* state, void* out,
+                          int B, int H, int gridH_local, int gridW, int halo_top, int halo_bottom, int d,
+                          castling_dtype_t dtype, void* stream);
+
+/*
  * castling_attn_selftest_wait: check the mechanism behind that status word without any fault.  Launches one
  * small kernel on `stream` whose threads wait, with a limit of `limit_us` microseconds (1 .. 1 000 000), on a
  * shared-memory barrier that nothing completes -- the situation of a pipeline whose copy or partner never

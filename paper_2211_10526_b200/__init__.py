@@ -8,12 +8,12 @@ run before it exists) and loading raises if it has not been built.
 """
 import importlib
 
-__all__ = ["binding", "CastlingAttn", "build"]
+__all__ = ["binding", "CastlingAttn", "build", "sharded"]
 
 
 def __getattr__(name):
     if name == "CastlingAttn":
         return importlib.import_module(".attn", __name__).CastlingAttn
-    if name in ("binding", "build", "attn"):
+    if name in ("binding", "build", "attn", "sharded"):
         return importlib.import_module("." + name, __name__)
     raise AttributeError(f"module {__name__!r} has no attribute {name!r}")

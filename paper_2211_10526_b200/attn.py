@@ -126,6 +126,42 @@ class CastlingAttn:
             raise _b.CastlingError(rc, "castling_attn_forward_host")
         return out
 
+    def shard_state(self, k, v, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Sums over this band's tokens (k, v: contiguous [B, H, n, d] on the device) -> fp32 [B*H, d*d + d]:
+        K^^T V row-major, then the token sum of V.  The states of the bands of one sequence add up."""
+        if k.shape != v.shape or k.dim() != 4 or not (k.is_contiguous() and v.is_contiguous()) or k.dtype != v.dtype:
+            raise ValueError("k, v: contiguous [B, H, n, d] tensors of one dtype")
+        B, H, n, d = k.shape
+        if out is None:
+            out = torch.empty(B * H, _b.castling_attn_state_words(d), dtype=torch.float32, device=k.device)
+        rc = _b.castling_attn_shard_state(self._h, k.data_ptr(), v.data_ptr(), out.data_ptr(), B, H, n, d, _dtype_code(k),
+                                          _current_raw_stream(k.device))
+        if rc != _b.OK:
+            raise _b.CastlingError(rc, "castling_attn_shard_state")
+        return out
+
+    def shard_apply(self, q, v_halo, dw_weight, dw_bias: Optional[torch.Tensor], state, gridH_local: int, gridW: int,
+                    halo_top: int, halo_bottom: int, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Output rows of one band of grid rows from a state summed over all bands; v_halo holds the band's rows of
+        V between halo_top rows of the band above and halo_bottom rows of the band below."""
+        B, H, n, d = q.shape
+        rows = halo_top + gridH_local + halo_bottom
+        if n != gridH_local * gridW or tuple(v_halo.shape) != (B, H, rows * gridW, d):
+            raise ValueError("q: [B, H, gridH_local*gridW, d]; v_halo: [B, H, (halo_top+gridH_local+halo_bottom)*gridW, d]")
+        if not (q.is_contiguous() and v_halo.is_contiguous() and dw_weight.is_contiguous() and state.is_contiguous()):
+            raise ValueError("contiguous tensors expected")
+        if tuple(state.shape) != (B * H, _b.castling_attn_state_words(d)) or state.dtype != torch.float32:
+            raise ValueError("state: fp32 [B*H, d*d + d]")
+        if out is None:
+            out = torch.empty_like(q)
+        rc = _b.castling_attn_shard_apply(self._h, q.data_ptr(), v_halo.data_ptr(), dw_weight.data_ptr(),
+                                          None if dw_bias is None else dw_bias.data_ptr(), state.data_ptr(), out.data_ptr(),
+                                          B, H, gridH_local, gridW, halo_top, halo_bottom, d, _dtype_code(q),
+                                          _current_raw_stream(q.device))
+        if rc != _b.OK:
+            raise _b.CastlingError(rc, "castling_attn_shard_apply")
+        return out
+
     def last_path(self):
         return _b.castling_attn_last_path(self._h)
 

@@ -65,6 +65,12 @@ def _load() -> ctypes.CDLL:
     lib.castling_attn_last_path.argtypes = [vp, ctypes.POINTER(i)]
     lib.castling_attn_device_status.restype = i
     lib.castling_attn_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint)]
+    lib.castling_attn_state_words.restype = sz
+    lib.castling_attn_state_words.argtypes = [i]
+    lib.castling_attn_shard_state.restype = i
+    lib.castling_attn_shard_state.argtypes = [vp] * 4 + [i] * 4 + [i, vp]
+    lib.castling_attn_shard_apply.restype = i
+    lib.castling_attn_shard_apply.argtypes = [vp] * 7 + [i] * 7 + [i, vp]
     lib.castling_attn_selftest_wait.restype = i
     lib.castling_attn_selftest_wait.argtypes = [vp, ctypes.c_uint, vp]
     lib.castling_attn_set_profiling.restype = i
@@ -144,6 +150,22 @@ def castling_attn_device_status(handle, stream: int = 0):
     raw = ctypes.c_uint(0)
     rc = lib.castling_attn_device_status(handle, stream or None, ctypes.byref(raw))
     return rc, raw.value
+
+
+def castling_attn_state_words(d: int) -> int:
+    return int(lib.castling_attn_state_words(int(d)))
+
+
+def castling_attn_shard_state(handle, k: int, v: int, state_out: int, B: int, H: int, n_tokens: int, d: int, dtype: int,
+                              stream: int = 0) -> int:
+    return lib.castling_attn_shard_state(handle, k, v, state_out, B, H, n_tokens, d, dtype, stream or None)
+
+
+def castling_attn_shard_apply(handle, q: int, v_halo: int, dw_weight: int, dw_bias: Optional[int], state: int, out: int,
+                              B: int, H: int, gridH_local: int, gridW: int, halo_top: int, halo_bottom: int, d: int,
+                              dtype: int, stream: int = 0) -> int:
+    return lib.castling_attn_shard_apply(handle, q, v_halo, dw_weight, dw_bias, state, out, B, H, gridH_local, gridW,
+                                         halo_top, halo_bottom, d, dtype, stream or None)
 
 
 def castling_attn_selftest_wait(handle, limit_us: int = 2000, stream: int = 0) -> int:

@@ -475,6 +475,62 @@ int castling_attn_device_status(castling_attn_t* h, void* stream, unsigned int* 
     return word ? CASTLING_ERR_DEVICE : CASTLING_OK;
 }
 
+size_t castling_attn_state_words(int d) { return d > 0 ? castling::state_words(d) : 0; }
+
+// The two halves of a forward whose token grid is cut into bands of rows held by different devices.
+static int shard_config_ok(const castling_attn* h) {
+    if (!h) return CASTLING_ERR_INVALID_ARG;
+    if (h->cfg.prefix_tokens || h->cfg.normalize_rows || h->cfg.exact_kernel || h->cfg.sparse_branch) return CASTLING_ERR_UNSUPPORTED;
+    return CASTLING_OK;
+}
+
+int castling_attn_shard_state(castling_attn_t* h, const void* k, const void* v, float* state_out,
+                              int B, int H, int n_tokens, int d, castling_dtype_t dtype, void* stream) {
+    int rc = shard_config_ok(h);
+    if (rc != CASTLING_OK) return rc;
+    rc = check_shape(h, B, H, 1, n_tokens, d, dtype);
+    if (rc != CASTLING_OK) return rc;
+    if (!k || !v || !state_out) return CASTLING_ERR_INVALID_ARG;
+    if (((uintptr_t)k | (uintptr_t)v | (uintptr_t)state_out) & 15) return CASTLING_ERR_ALIGNMENT;
+    Problem p = make_problem(h, nullptr, k, v, nullptr, nullptr, nullptr, B, H, 1, n_tokens, d, dtype);
+    p.phase = castling::kPhaseStateOnly;
+    rc = ensure_workspace(h, p.BH, p.N, p.d, p.bf16);
+    if (rc != CASTLING_OK) return rc;
+    float* partial = h->ws + castling::kHeaderWords + (size_t)p.BH * castling::state_words(p.d);
+    int launches = 0;
+    h->timer.begin(static_cast<cudaStream_t>(stream));
+    const cudaError_t e = castling::simt_forward(p, state_out, partial, castling::simt_choose_splits(p.BH, p.N),
+                                                 static_cast<cudaStream_t>(stream), &launches, &h->timer);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->last_path = CASTLING_PATH_SIMT; h->last_launches = launches;
+    return CASTLING_OK;
+}
+
+int castling_attn_shard_apply(castling_attn_t* h, const void* q, const void* v_halo, const void* dw_weight,
+                              const void* dw_bias, const float* state, void* out, int B, int H, int gridH_local,
+                              int gridW, int halo_top, int halo_bottom, int d, castling_dtype_t dtype, void* stream) {
+    int rc = shard_config_ok(h);
+    if (rc != CASTLING_OK) return rc;
+    rc = check_shape(h, B, H, gridH_local, gridW, d, dtype);
+    if (rc != CASTLING_OK) return rc;
+    if (!q || !v_halo || !dw_weight || !state || !out) return CASTLING_ERR_INVALID_ARG;
+    const int r = (h->cfg.ksize - 1) / 2;
+    if (halo_top < 0 || halo_bottom < 0 || halo_top > r || halo_bottom > r) return CASTLING_ERR_INVALID_ARG;
+    if (((uintptr_t)q | (uintptr_t)v_halo | (uintptr_t)out | (uintptr_t)state) & 15) return CASTLING_ERR_ALIGNMENT;
+    Problem p = make_problem(h, q, nullptr, v_halo, dw_weight, dw_bias, out, B, H, gridH_local, gridW, d, dtype);
+    p.phase = castling::kPhaseApplyOnly;
+    p.v_row0 = halo_top;
+    p.v_rows = halo_top + gridH_local + halo_bottom;
+    p.lv.head = (long long)p.v_rows * gridW * d;   // planes of the taller V tensor
+    int launches = 0;
+    h->timer.begin(static_cast<cudaStream_t>(stream));
+    const cudaError_t e = castling::simt_forward(p, const_cast<float*>(state), nullptr, 1, static_cast<cudaStream_t>(stream),
+                                                 &launches, &h->timer);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->last_path = CASTLING_PATH_SIMT; h->last_launches = launches;
+    return CASTLING_OK;
+}
+
 int castling_attn_selftest_wait(castling_attn_t* h, unsigned int limit_us, void* stream) {
     if (!h || limit_us == 0 || limit_us > 1000000u) return CASTLING_ERR_INVALID_ARG;
     int rc = ensure_workspace(h, 1, 64, 64, true);  // the status word lives at the head of the workspace

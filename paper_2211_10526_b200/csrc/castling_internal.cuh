@@ -11,6 +11,7 @@
 namespace castling {
 
 constexpr float kInvPi = 0.31830988618379067154f;
+constexpr int kPhaseAll = 0, kPhaseStateOnly = 1, kPhaseApplyOnly = 2;
 
 // Element strides of one [B, H, N, d] tensor whose d elements are contiguous.
 struct Layout {
@@ -47,6 +48,11 @@ struct Problem {
     bool exact_kernel = false;  // 1 - arccos(x)/pi (Eq. 4-5) instead of its kept part 1/2 + x/pi (Eq. 8)
     bool sparse = false;        // plus Mask_eps(Softmax(q^ k^^T)) (Eq. 10)
     float sparse_eps = 0.f;     // the mask's threshold
+    // A forward cut in two for sequences sharded over devices (CUDA-core kernels): the state of this shard's tokens
+    // only, or the apply pass only with a state summed over all shards given in the workspace's place.
+    int phase = 0;              // kPhaseAll / kPhaseStateOnly / kPhaseApplyOnly
+    int v_row0 = 0, v_rows = 0; // apply of a shard: V holds v_rows grid rows and its row v_row0 is the shard's row 0
+                                // (v_rows = 0: V holds exactly the gridH rows)
     int hdiv;          // planes per batch step of the layouts: H for a caller's strided tensors, BH for a
                        // run of contiguous planes (one uniform plane stride)
     // Contiguous [planes][N][d] tensors; needs N, d and BH.

@@ -201,7 +201,9 @@ __global__ void __launch_bounds__(kThreads)
 simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __restrict__ w,
                   const T* __restrict__ bias, const float* __restrict__ state, T* __restrict__ out,
                   int H, int head0, int prefix, int gridH, int gridW, int ksize, float eps2, Layout lq, Layout lv,
-                  Layout lo, int hdiv, int words, int zsum) {
+                  Layout lo, int hdiv, int words, int zsum, int v_row0, int v_rows) {
+    // v_row0, v_rows: the V tensor holds v_rows grid rows, of which row v_row0 is this call's grid row 0 (a shard of
+    // a taller grid brings the rows of its neighbours that the filters reach; otherwise 0 and gridH)
     constexpr int R = D / 16;
     constexpr int LDQ = D + 1;
     extern __shared__ __align__(16) float smem[];
@@ -299,8 +301,8 @@ simt_apply_kernel(const T* __restrict__ q, const T* __restrict__ v, const T* __r
                         : fmaf(acc[r][c], scale, c_sm[tj * R + c] + (g >= 0 ? b_sm[tj * R + c] : 0.f));
         }
         for (int dy = -rad; dy <= rad && g >= 0; ++dy) {
-            const int yy = y + dy;
-            if (yy < 0 || yy >= gridH) continue;
+            const int yy = y + dy + v_row0;
+            if (yy < 0 || yy >= v_rows) continue;
             for (int dx = -rad; dx <= rad; ++dx) {
                 const int xx = x + dx;
                 if (xx < 0 || xx >= gridW) continue;
@@ -473,7 +475,8 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
                         cudaStream_t stream, int* launches, KernelTimer* timer) {
     const int zsum = p.rownorm ? 1 : 0;
     const int words = D * D + D + (zsum ? D : 0);
-    if (!zsum && p.N <= kFusedMaxTokens && p.BH >= kFusedMinPlanes && simt_fused_smem<D>(p.N, p.ksize) <= kFusedSmemLimit) {
+    if (!zsum && p.phase == kPhaseAll && p.N <= kFusedMaxTokens && p.BH >= kFusedMinPlanes &&
+        simt_fused_smem<D>(p.N, p.ksize) <= kFusedSmemLimit) {
         const size_t smem = simt_fused_smem<D>(p.N, p.ksize);
         static PerDevice fused_opt_in;
         cudaError_t e = opt_in_smem(simt_fused_kernel<T, D>, kFusedSmemLimit, fused_opt_in);
@@ -487,21 +490,25 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
         timer->mark(stream, "simt_fused");
         return e;
     }
-    const int tiles = (p.N + kStateTile - 1) / kStateTile;
-    const int chunk = ((tiles + P - 1) / P) * kStateTile;
-    float* dst = (P > 1) ? ws_partial : ws_state;
-    simt_state_kernel<T, D><<<(unsigned)(p.BH * P), kThreads, 0, stream>>>(
-        static_cast<const T*>(p.k), static_cast<const T*>(p.v), dst, p.N, chunk, P, p.eps2, p.lk, p.lv, p.hdiv, words, zsum);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    *launches = 1;
-    timer->mark(stream, "simt_state");
-    if (P > 1) {
-        simt_reduce_kernel<<<p.BH, kThreads, 0, stream>>>(ws_partial, ws_state, words, P);
+    cudaError_t e = cudaSuccess;
+    if (p.phase != kPhaseApplyOnly) {
+        const int tiles = (p.N + kStateTile - 1) / kStateTile;
+        const int chunk = ((tiles + P - 1) / P) * kStateTile;
+        float* dst = (P > 1) ? ws_partial : ws_state;
+        simt_state_kernel<T, D><<<(unsigned)(p.BH * P), kThreads, 0, stream>>>(
+            static_cast<const T*>(p.k), static_cast<const T*>(p.v), dst, p.N, chunk, P, p.eps2, p.lk, p.lv, p.hdiv, words, zsum);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         ++*launches;
-        timer->mark(stream, "simt_reduce");
+        timer->mark(stream, "simt_state");
+        if (P > 1) {
+            simt_reduce_kernel<<<p.BH, kThreads, 0, stream>>>(ws_partial, ws_state, words, P);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+            ++*launches;
+            timer->mark(stream, "simt_reduce");
+        }
+        if (p.phase == kPhaseStateOnly) return cudaSuccess;
     }
     const size_t smem = simt_apply_smem<D>(p.ksize);
     static PerDevice apply_opt_in;
@@ -511,7 +518,7 @@ cudaError_t launch_simt(const Problem& p, float* ws_state, float* ws_partial, in
     simt_apply_kernel<T, D><<<grid, kThreads, smem, stream>>>(
         static_cast<const T*>(p.q), static_cast<const T*>(p.v), static_cast<const T*>(p.w),
         static_cast<const T*>(p.bias), ws_state, static_cast<T*>(p.out), p.H, p.head0, p.prefix, p.gridH, p.gridW, p.ksize,
-        p.eps2, p.lq, p.lv, p.lo, p.hdiv, words, zsum);
+        p.eps2, p.lq, p.lv, p.lo, p.hdiv, words, zsum, p.v_row0, p.v_rows > 0 ? p.v_rows : p.gridH);
     e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     timer->mark(stream, "simt_apply");
