@@ -64,6 +64,21 @@ struct ApplyParams {
     unsigned* status;
 };
 
+// Position of a CTA's current patch, advanced without divisions (one step per patch in every role).
+struct PatchWalk {
+    int bh, py, px;
+    __device__ __forceinline__ PatchWalk(int g, int tilesX, int tilesY) {
+        const int per = tilesX * tilesY;
+        bh = g / per;
+        const int rem = g - bh * per;
+        py = rem / tilesX;
+        px = rem - py * tilesX;
+    }
+    __device__ __forceinline__ void step(int tilesX, int tilesY) {
+        if (++px == tilesX) { px = 0; if (++py == tilesY) { py = 0; ++bh; } }
+    }
+};
+
 // MODE 0: width-64 heads; 1: width-32 heads, two adjacent tokens per 128-byte row (the PAIR geometry);
 // 2: two width-32 heads side by side in the one-token-per-row geometry (block-diagonal state).
 template <int KS, int MODE>
@@ -90,7 +105,6 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int tiles_per_bh = prm.tilesX * prm.tilesY;
     // contiguous share of the patches for this CTA
     const int g_begin = (int)((long long)prm.n_tiles * blockIdx.x / gridDim.x);
     const int g_end = (int)((long long)prm.n_tiles * (blockIdx.x + 1) / gridDim.x);
@@ -110,16 +124,19 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tcgen05_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
     constexpr unsigned kBit = kStatusApplyTimeout;
+    // the next forward's state kernel (launched programmatically dependent) may set itself up on multiprocessors
+    // this grid has left; it waits for this grid's completion before it touches global memory
+    pdl_launch_dependents();
 
     if (warp == 0) {
         if (lane == 0) {
             int issued = 0;
             const uint64_t pol_q = l2_policy_evict_first();  // Q is read once
-            for (int it = 0; it < my_tiles; ++it) {
+            PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
+            for (int it = 0; it < my_tiles; ++it, pw.step(prm.tilesX, prm.tilesY)) {
                 const int s = it % NS, use = it / NS;
                 if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) break;
-                const int g = g_begin + it, bh = g / tiles_per_bh, rem = g % tiles_per_bh;
-                const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
+                const int bh = pw.bh, y0 = pw.py * kTY, x0 = pw.px * kTX;
                 uint8_t* qs = stages + s * G::kStage;
                 mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
                 if (prm.flat) {
@@ -142,9 +159,10 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             constexpr uint32_t idesc = umma_idesc_bf16(128, kD, false, true);
             const uint32_t s_addr = smem_u32(S_s);
             int prev_bh = -1, seg = 0;
-            for (int it = 0; it < my_tiles; ++it) {
+            PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
+            for (int it = 0; it < my_tiles; ++it, pw.step(prm.tilesX, prm.tilesY)) {
                 const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
-                const int bh = (g_begin + it) / tiles_per_bh;
+                const int bh = pw.bh;
                 if (bh != prev_bh) {
                     if (!mbar_wait(s_ready, seg & 1, abort_flag, prm.status, kBit)) break;
                     ++seg; prev_bh = bh;
@@ -171,10 +189,10 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
         int prev_bh = -1;
         pdl_wait_primary();  // the state kernel's results are read below
-        for (int it = 0; it < my_tiles; ++it) {
+        PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
+        for (int it = 0; it < my_tiles; ++it, pw.step(prm.tilesX, prm.tilesY)) {
             const int b = it & 1, ub = it >> 1;
-            const int g = g_begin + it, bh = g / tiles_per_bh, rem = g % tiles_per_bh;
-            const int y0 = (rem / prm.tilesX) * kTY, x0 = (rem % prm.tilesX) * kTX;
+            const int bh = pw.bh, y0 = pw.py * kTY, x0 = pw.px * kTX;
             if (bh != prev_bh) {
                 // every UMMA that read the previous S' has retired (its acc_full was waited on below)
                 prev_bh = bh;
@@ -291,9 +309,10 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         float2 cinit = make_float2(0.f, 0.f);
         int prev_bh = -1;
         pdl_wait_primary();  // the token sums of the state kernel are read below
-        for (int it = 0; it < my_tiles; ++it) {
+        PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
+        for (int it = 0; it < my_tiles; ++it, pw.step(prm.tilesX, prm.tilesY)) {
             const int s = it % NS, use = it / NS, b = it & 1, ub = it >> 1;
-            const int bh = (g_begin + it) / tiles_per_bh;
+            const int bh = pw.bh;
             if (bh != prev_bh) {
                 prev_bh = bh;
                 // this lane's channel pair: 2*lane of 64 channels, or (PAIR) 2*(lane & 15) of 32 channels

@@ -60,6 +60,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int n_tiles = min(total_tiles, t_begin + tiles_per_cta) - t_begin;  // per item
     const int bh = bh0;  // the (b,h) of the split reduction below (P > 1: the only item)
     if (n_tiles <= 0 || n_items <= 0) {  // the host never makes such a CTA; keep the partial well defined anyway
+        pdl_wait_primary();
         if (P > 1) {
             float* out = dst + ((size_t)bh * P + p) * (kD * kD + kD);
             for (int i = tid; i < kD * kD + kD; i += kThreads) out[i] = 0.f;
@@ -102,6 +103,11 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             // K is read once; V is read again by the apply kernel: keep it in L2 as long as possible
             const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_last();
             bool ok = true;
+            // Launched programmatically dependent on the kernel before it in the stream (the apply kernel of the
+            // previous forward lets its dependents start early): everything above ran while that kernel drained.
+            // Global memory is first touched here; the partial states and arrival counters are written only after
+            // these loads have landed.
+            pdl_wait_primary();
             for (int item = 0; item < n_items && ok; ++item) {
                 for (int it = 0; it < n_tiles; ++it, ++issued) {
                     const int s = issued % kStages, use = issued / kStages;
@@ -347,13 +353,17 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
         items = (p.BH + resident - 1) / resident;
         grid = (p.BH + items - 1) / items;
     }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
     if (halves)
-        tc_state_kernel<true><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(
-            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, p.hdiv, items, p.eps2, status);
-    else
-        tc_state_kernel<false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(
-            tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, p.hdiv, items, p.eps2, status);
-    return cudaGetLastError();
+        return cudaLaunchKernelEx(&cfg, tc_state_kernel<true>, tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P,
+                                  p.BH, p.hdiv, items, p.eps2, status);
+    return cudaLaunchKernelEx(&cfg, tc_state_kernel<false>, tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P,
+                              p.BH, p.hdiv, items, p.eps2, status);
 }
 
 }  // namespace tc
