@@ -57,6 +57,12 @@ static bool two_kernels() {
     return !one;
 }
 
+// CASTLING_TC_CLUSTER=1 in the environment selects the cluster-per-plane forward where the shape allows it.
+static bool cluster_enabled() {
+    static const bool on = [] { const char* e = getenv("CASTLING_TC_CLUSTER"); return e && e[0] == '1'; }();
+    return on;
+}
+
 cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer) {
     *launches = 0;
@@ -75,6 +81,13 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
         return cudaSuccess;
     }
     cudaError_t e;
+    if (const int C = cluster_enabled() ? cluster_size(p) : 0) {
+        e = launch_cluster(p, C, status, stream);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        timer->mark(stream, "tc_cluster");
+        return cudaSuccess;
+    }
     if (!two_kernels() && pipe_supports(p)) {
         // state and apply pipelines in one persistent kernel: V is read from memory once
         e = launch_pipe(p, ws_state, ws_partial, counters, status, stream);

@@ -72,6 +72,12 @@ bool pipe_supports(const Problem& p);
 size_t pipe_ready_words(int BH);
 cudaError_t launch_pipe(const Problem& p, float* state, float* ready, unsigned* ctr, unsigned* status, cudaStream_t st);
 
+// Forward with one thread-block cluster per plane (csrc/tc_cluster.cu): every CTA builds the state of its share of
+// the plane, the cluster adds the shares up through distributed shared memory, every CTA applies the sum to its
+// share of the patches.  One launch, no workspace.  cluster_size: CTAs per plane, 0 when the shape is not taken.
+int cluster_size(const Problem& p);
+cudaError_t launch_cluster(const Problem& p, int C, unsigned* status, cudaStream_t st);
+
 // Single-kernel forward for short sequences (bf16, 3x3 or 5x5 filters, at most 256 128-byte rows per plane:
 // d = 64 with N <= 256, two width-32 heads per row with N <= 256, or width-32 token pairs with N <= 512): no workspace.
 bool fused_supports(const Problem& p);
