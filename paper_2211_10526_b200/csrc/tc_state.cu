@@ -100,8 +100,10 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (warp == 0) {
         if (lane == 0) {
             int issued = 0;
-            // K is read once; V is read again by the apply kernel: keep it in L2 as long as possible
-            const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_last();
+            // Both tensors stream through L2 once here.  V is read again by the apply kernel, but at long sequences it
+            // does not survive until then whatever the hint, and lines marked evict-last pile up and slow the streams
+            // of both kernels (measured: 132 -> 125 us per forward at 2 x 8 planes of 256 x 256 tokens).
+            const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_first();
             bool ok = true;
             // Launched programmatically dependent on the kernel before it in the stream (the apply kernel of the
             // previous forward lets its dependents start early): everything above ran while that kernel drained.
