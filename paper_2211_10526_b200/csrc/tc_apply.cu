@@ -131,6 +131,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 0) {
         if (lane == 0) {
             int issued = 0;
+            const uint64_t pol_q = l2_policy_evict_first();  // Q is read once
             PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
             for (int it = 0; it < my_tiles; ++it, pw.step(prm.tilesX, prm.tilesY)) {
                 const int s = it % NS, use = it / NS;
@@ -139,11 +140,11 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 uint8_t* qs = stages + s * G::kStage;
                 mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
                 if (prm.flat) {
-                    tma_load_4d(qs, &tmQ, &full[s], 0, x0, y0, bh);
+                    tma_load_4d_hint(qs, &tmQ, &full[s], 0, x0, y0, bh, pol_q);
                     tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, bh);
                 } else {
                     const int pb = bh / prm.hdiv, ph = bh - pb * prm.hdiv;
-                    tma_load_5d(qs, &tmQ, &full[s], 0, x0, y0, ph, pb);
+                    tma_load_5d_hint(qs, &tmQ, &full[s], 0, x0, y0, ph, pb, pol_q);
                     tma_load_5d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, ph, pb);
                 }
                 ++issued;
@@ -185,6 +186,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int quarter = warp & 3, row = quarter * 32 + lane, et = tid - 64;
         const int half = (warp - 2) >> 2;  // channels half*32 .. half*32 + 31
         const bool leader = (et == 0);
+        const uint64_t pol_o = l2_policy_evict_first();  // the output is not read back here
         int prev_bh = -1;
         pdl_wait_primary();  // the state kernel's results are read below
         PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
@@ -289,10 +291,10 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             named_barrier_sync(1, kEpiThreads);
             if (leader) {
                 if (prm.flat) {
-                    tma_store_4d(&tmO, out_s, 0, x0, y0, bh);
+                    tma_store_4d_hint(&tmO, out_s, 0, x0, y0, bh, pol_o);
                 } else {
                     const int pb = bh / prm.hdiv;
-                    tma_store_5d(&tmO, out_s, 0, x0, y0, bh - pb * prm.hdiv, pb);
+                    tma_store_5d_hint(&tmO, out_s, 0, x0, y0, bh - pb * prm.hdiv, pb, pol_o);
                 }
                 tma_store_commit();
             }

@@ -172,11 +172,6 @@ __device__ __forceinline__ void tma_load_5d_hint(void* dst, const CUtensorMap* m
         "r"(c3), "r"(c4), "l"(policy)
         : "memory");
 }
-__device__ __forceinline__ void tma_store_5d(const CUtensorMap* m, const void* src, int c0, int c1, int c2, int c3, int c4) {
-    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-                 : "memory");
-}
 __device__ __forceinline__ void tma_store_5d_hint(const CUtensorMap* m, const void* src, int c0, int c1, int c2, int c3,
                                                   int c4, uint64_t policy) {
     asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3, %4, %5, %6}], [%1], %7;"
