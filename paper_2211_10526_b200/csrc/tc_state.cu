@@ -231,8 +231,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (ok) ok = flush(n_items - 1);
     }
     tcgen05_fence_before_sync();
-    __threadfence();  // this split's partial state is visible device-wide before the arrival below
-    __syncthreads();
+    __syncthreads();  // every thread's part of this split's partial state has been stored
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 
     // Cross-split reduction without a second launch and without any waiting, as a two-level tree
@@ -248,10 +247,16 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const int n_groups = (P + kGroup - 1) / kGroup, grp = p / kGroup;
         const int first = grp * kGroup, members = min(kGroup, P - first);
         float4* base = reinterpret_cast<float4*>(dst + (size_t)bh * P * kWords);
-        if (tid == 0) is_last = (atomicAdd(&cnt[grp], 1u) == (unsigned)(members - 1));
+        // One thread publishes for the CTA: its device-wide fence after the CTA barrier covers the stores the other
+        // threads made before that barrier; its fence after the atomic, followed by a CTA barrier, lets every thread
+        // read what the other CTAs of the group published the same way.
+        if (tid == 0) {
+            __threadfence();
+            is_last = (atomicAdd(&cnt[grp], 1u) == (unsigned)(members - 1));
+            __threadfence();
+        }
         __syncthreads();
         if (!is_last) return;
-        __threadfence();
         if (members > 1) {
             float4 acc[kIter];
 #pragma unroll
@@ -281,15 +286,15 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (i < kWords4) base[(size_t)first * kWords4 + i] = acc[j];
             }
         }
-        __threadfence();
         __syncthreads();
         if (tid == 0) {
             cnt[grp] = 0;
+            __threadfence();
             is_last = (atomicAdd(&cnt[kCountersPerHead - 1], 1u) == (unsigned)(n_groups - 1));
+            __threadfence();
         }
         __syncthreads();
         if (!is_last) return;
-        __threadfence();
         float4* fin = reinterpret_cast<float4*>(final_state + (size_t)bh * kWords);
         float4 acc[kIter];
 #pragma unroll
