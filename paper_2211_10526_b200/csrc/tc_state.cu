@@ -257,6 +257,9 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         __syncthreads();
         if (!is_last) return;
+        // a single group (at most kGroup splits): its sum is the final state, no second level
+        float4* fin = reinterpret_cast<float4*>(final_state + (size_t)bh * kWords);
+        float4* level1 = (n_groups == 1) ? fin : base + (size_t)first * kWords4;
         if (members > 1) {
             float4 acc[kIter];
 #pragma unroll
@@ -283,8 +286,12 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
             for (int j = 0; j < kIter; ++j) {
                 const int i = tid + j * kThreads;
-                if (i < kWords4) base[(size_t)first * kWords4 + i] = acc[j];
+                if (i < kWords4) level1[i] = acc[j];
             }
+        }
+        if (n_groups == 1) {
+            if (tid == 0) cnt[grp] = 0;
+            return;
         }
         __syncthreads();
         if (tid == 0) {
@@ -295,7 +302,6 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         __syncthreads();
         if (!is_last) return;
-        float4* fin = reinterpret_cast<float4*>(final_state + (size_t)bh * kWords);
         float4 acc[kIter];
 #pragma unroll
         for (int j = 0; j < kIter; ++j) {
