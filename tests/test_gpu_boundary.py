@@ -122,6 +122,40 @@ def test_bitwise_reproducible(name, idx):
         assert torch.equal(o.view(torch.uint8), outs[0].view(torch.uint8))
 
 
+@pytest.mark.parametrize("shape", [(2, 8, 64, 64, 64, 3), (2, 4, 96, 128, 64, 3), (4, 8, 64, 64, 32, 5)],
+                         ids=lambda t: "x".join(map(str, t)))
+def test_forwards_queued_back_to_back_do_not_disturb_each_other(shape):
+    """On the tensor-core path the state kernel of a forward starts while the apply kernel of the previous one is
+    still draining (programmatic dependent launch).  Forwards on alternating, different inputs are queued without
+    any synchronisation, each into its own output; every output has to equal, bit for bit, the output of the same
+    inputs run alone (the path is bitwise reproducible), so a state written too early, or read too late, shows."""
+    b = _b()
+    sets = []
+    for seed in (431, 432, 433):
+        c = workloads.custom_call(*shape, "bf16", seed=seed)
+        sets.append((c, _dev(c)))
+    s = sets[0][0].shape
+    h = b.castling_attn_create(s.ksize)
+    alone = []
+    for c, (q, k, v, w, bias) in sets:
+        out = torch.empty_like(q)
+        assert _raw_forward(b, h, q, k, v, w, bias, out, s) == b.OK
+        torch.cuda.synchronize()
+        alone.append(out)
+    assert not torch.equal(alone[0], alone[1])
+    rounds = 12
+    outs = [[torch.full_like(alone[0], float("nan")) for _ in sets] for _ in range(rounds)]
+    for r in range(rounds):
+        for i, (c, (q, k, v, w, bias)) in enumerate(sets):
+            assert _raw_forward(b, h, q, k, v, w, bias, outs[r][i], s) == b.OK
+    torch.cuda.synchronize()
+    assert b.castling_attn_device_status(h)[0] == b.OK
+    b.castling_attn_destroy(h)
+    for r in range(rounds):
+        for i in range(len(sets)):
+            assert torch.equal(outs[r][i].view(torch.uint8), alone[i].view(torch.uint8)), (r, i)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_host_entry_point_matches_device_entry_point(dtype):
     from paper_2211_10526_b200 import CastlingAttn
