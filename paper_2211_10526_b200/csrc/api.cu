@@ -54,7 +54,7 @@ size_t workspace_words(int BH, int N, int d, bool bf16) {
     if (bf16 && (d == 64 || d == 32)) {  // shapes the tensor-core kernels may take: they keep 64-wide states
         const int Pt = castling::tc::choose_splits(BH, castling::tc::rows_per_head(N, d));
         if (Pt > P) P = Pt;
-        if (castling::tc::kStateWords > words) words = castling::tc::kStateWords;
+        if (castling::tc::kStateWordsRownorm > words) words = castling::tc::kStateWordsRownorm;
     }
     size_t slots = (size_t)BH * (P > 1 ? P : 0);  // partial states behind the BH final ones
     if (bf16 && d == 32 && BH % 2 == 0) {
@@ -229,14 +229,13 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     }
     int rc = ensure_workspace(h, p.BH, p.N, p.d, p.bf16);
     if (rc != CASTLING_OK) return rc;
-    // the row-sum denominator needs the sum of the unit key rows, which only the CUDA-core kernels build
-    const bool tensor_ok = castling::tc::supports(p) && !p.rownorm;
+    const bool tensor_ok = castling::tc::supports(p);
     if (h->cfg.force_path == CASTLING_PATH_TENSOR && !tensor_ok) return CASTLING_ERR_UNSUPPORTED;
     bool use_tensor = tensor_ok && (h->cfg.force_path == CASTLING_PATH_TENSOR ||
                                     (h->cfg.force_path == CASTLING_PATH_AUTO && castling::tc::preferred(p)));
     float* state = h->ws + castling::kHeaderWords;
     const size_t simt_words = p.rownorm ? castling::state_words_rownorm(p.d) : castling::state_words(p.d);
-    float* partial = state + (size_t)p.BH * (use_tensor ? (size_t)castling::tc::kStateWords : simt_words);
+    float* partial = state + (size_t)p.BH * (use_tensor ? (size_t)castling::tc::state_words_of(p) : simt_words);
     int launches = 0;
     h->timer.begin(stream);
     cudaError_t e;

@@ -51,6 +51,10 @@ template <int KS, bool PAIR> struct Geo {
     static constexpr int kOffRq = kOffStg + 2 * kStgBytes;   // sum of squares of each half of a Q row
     static constexpr int kOffBar = kOffRq + 2 * kTile * 4;
     static constexpr size_t kSmem = 1024 + kOffBar + 256;
+    // row-sum normalisation: a second 64-wide block of the operand (its first columns hold sum k^ / pi) and 1/2 s per
+    // staging buffer
+    static constexpr int kOffS2 = ((kOffBar + 256 + 1023) / 1024) * 1024, kOffHs = kOffS2 + 8192;
+    static constexpr size_t kSmemRN = 1024 + kOffHs + 2 * kD * 4;
 };
 
 struct ApplyParams {
@@ -62,6 +66,7 @@ struct ApplyParams {
     int H, head0, bh0, hdiv, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
+    int n_tokens;                  // tokens per sequence (row-sum normalisation: the sum of the constant 1/2 terms is n_tokens / 2)
 };
 
 // Position of a CTA's current patch, advanced without divisions (one step per patch in every role).
@@ -81,13 +86,20 @@ struct PatchWalk {
 
 // MODE 0: width-64 heads; 1: width-32 heads, two adjacent tokens per 128-byte row (the PAIR geometry);
 // 2: two width-32 heads side by side in the one-token-per-row geometry (block-diagonal state).
-template <int KS, int MODE>
+// RN: row-sum normalisation (Eq. 3's denominator on the kept kernel of Eq. 8).  The state carries sum_n k^_n behind s; the
+// operand gets one or two more columns (sum k^ / pi per head or token of the row), so that column 64 (65) of the
+// accumulator is q . sum k^ / pi; the attention term (acc / ||q|| + 1/2 s) is divided by n_tokens / 2 + that product
+// / ||q|| before the convolution and the bias are added.
+template <int KS, int MODE, bool RN>
 __global__ void __launch_bounds__((Geo<KS, MODE == 1>::kThreads), 1)
 tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmO, const ApplyParams prm) {
     constexpr bool PAIR = (MODE == 1), BLOCKDIAG = (MODE == 2);
     using G = Geo<KS, PAIR>;
     constexpr int NS = G::kStages;
+    constexpr int kSW = kD * kD + kD + (RN ? kD : 0);   // words of one state
+    constexpr int kAcc = RN ? 2 * kD : kD;              // TMEM columns per accumulator
+    constexpr int kAccN = RN ? kD + 16 : kD;            // columns the UMMAs write
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* S_s = smem + G::kOffS;
@@ -95,6 +107,8 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     uint8_t* stages = smem + G::kOffStages;
     uint8_t* stg = smem + G::kOffStg;
     float* rq_s = reinterpret_cast<float*>(smem + G::kOffRq);
+    uint8_t* S2_s = smem + G::kOffS2;                                  // RN only
+    float* hs_s = reinterpret_cast<float*>(smem + G::kOffHs);          // RN only: [2][64]
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + G::kOffBar);  // [NS] TMA landed
     uint64_t* empty = full + NS;                                      // [NS] stage consumed (conv + epilogue warps, UMMA commit)
     uint64_t* acc_full = empty + NS;                                  // [2]  UMMAs retired
@@ -118,7 +132,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO);
     }
-    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 1) tmem_alloc(tmem_slot, RN ? 2 * kTmemCols : kTmemCols);
     tcgen05_fence_before_sync();
     __syncthreads();
     tcgen05_fence_after_sync();
@@ -156,8 +170,9 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, kD, false, true);
+            constexpr uint32_t idesc = umma_idesc_bf16(128, kAccN, false, true);
             const uint32_t s_addr = smem_u32(S_s);
+            const uint32_t lbo = RN ? smem_u32(S2_s) - s_addr : 0;     // to the operand's second 64-wide block
             int prev_bh = -1, seg = 0;
             PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
             for (int it = 0; it < my_tiles; ++it, pw.step(prm.tilesX, prm.tilesY)) {
@@ -174,8 +189,8 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) {
                     const uint64_t a = umma_desc_sw128(q_addr + k * 32, 0, 1024);        // K-major rows of 128 B
-                    const uint64_t bd = umma_desc_sw128(s_addr + k * 2048, 0, 1024);     // N-major, 16 K-rows per step
-                    umma_bf16(tmem + b * kD, a, bd, idesc, k != 0);
+                    const uint64_t bd = umma_desc_sw128(s_addr + k * 2048, lbo, 1024);   // N-major, 16 K-rows per step
+                    umma_bf16(tmem + b * kAcc, a, bd, idesc, k != 0);
                 }
                 umma_commit(&acc_full[b]);
                 umma_commit(&empty[s]);  // the same UMMAs have finished reading the Q patch
@@ -197,7 +212,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 // every UMMA that read the previous S' has retired (its acc_full was waited on below)
                 prev_bh = bh;
                 const int i = et >> 2, part = et & 3;  // row i of the operand, 16 columns part*16 ..
-                const float* st = prm.state + (size_t)(prm.bh0 + bh) * prm.P * (kD * kD + kD);
+                const float* st = prm.state + (size_t)(prm.bh0 + bh) * prm.P * kSW;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     float4 lo, hi;
@@ -205,8 +220,8 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         const float4* src = reinterpret_cast<const float4*>(st + i * kD + part * 16);
                         lo = __ldg(src + 2 * c); hi = __ldg(src + 2 * c + 1);
                         for (int pp = 1; pp < prm.P; ++pp) {  // fixed order: bitwise reproducible
-                            const float4 l2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c);
-                            const float4 h2 = __ldg(src + pp * ((kD * kD + kD) / 4) + 2 * c + 1);
+                            const float4 l2 = __ldg(src + pp * (kSW / 4) + 2 * c);
+                            const float4 h2 = __ldg(src + pp * (kSW / 4) + 2 * c + 1);
                             lo.x += l2.x; lo.y += l2.y; lo.z += l2.z; lo.w += l2.w;
                             hi.x += h2.x; hi.y += h2.y; hi.z += h2.z; hi.w += h2.w;
                         }
@@ -231,6 +246,20 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     o.x = pack_bf16x2(lo.x * kInvPi, lo.y * kInvPi); o.y = pack_bf16x2(lo.z * kInvPi, lo.w * kInvPi);
                     o.z = pack_bf16x2(hi.x * kInvPi, hi.y * kInvPi); o.w = pack_bf16x2(hi.z * kInvPi, hi.w * kInvPi);
                     *reinterpret_cast<uint4*>(S_s + i * 128 + (((part * 2 + c) ^ (i & 7)) << 4)) = o;
+                    if (RN) {
+                        // second block of the operand: row i (a key feature) holds sum k^[i] / pi in column 0, or, where a
+                        // row carries two tokens or two heads, in the column of its half; the rest is zero
+                        uint4 z = make_uint4(0, 0, 0, 0);
+                        if (part == 0 && c == 0) {
+                            const float* sk = st + kD * kD + kD;
+                            float val;
+                            if (PAIR) val = __ldg(sk + (i & 31)) + __ldg(sk + 32 + (i & 31));   // both token parities
+                            else val = __ldg(sk + i);
+                            const uint32_t hv = pack_bf16x2(val * kInvPi, 0.f) & 0xffffu;
+                            z.x = (MODE != 0 && i >= 32) ? (hv << 16) : hv;
+                        }
+                        *reinterpret_cast<uint4*>(S2_s + i * 128 + (((part * 2 + c) ^ (i & 7)) << 4)) = z;
+                    }
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(s_ready);
@@ -258,11 +287,18 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             float a[32];
             {
                 float a0[16], a1[16];
-                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kD + half * 32, a0);
-                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kD + half * 32 + 16, a1);
+                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kAcc + half * 32, a0);
+                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kAcc + half * 32 + 16, a1);
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 16; ++e) { a[e] = a0[e]; a[16 + e] = a1[e]; }
+            }
+            float qk = 0.f;  // RN: q . sum k^ / pi of this thread's token
+            if (RN) {
+                float x[16];
+                tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + b * kAcc + kD, x);
+                tmem_ld_wait();
+                qk = (MODE != 0 && half == 1) ? x[1] : x[0];
             }
             if (!mbar_wait(&conv_full[b], ub & 1, abort_flag, prm.status, kBit)) break;
             // the previous patch's TMA store must have read out_s before it is rewritten; the same
@@ -274,15 +310,27 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                                  : rsqrtf(fmaxf(rq_s[row] + rq_s[kTile + row], prm.eps2));
             const uint8_t* srow = stg + b * kStgBytes + row * kStgStride + half * 128;
             uint8_t* orow = out_s + row * 128;
+            if (RN) {
+                // (acc / ||q|| + 1/2 s) / (n / 2 + q^ . sum k^ / pi); the staged value is convolution + bias only
+                const float inv = 1.0f / fmaf(qk, rq, 0.5f * (float)prm.n_tokens);
+                const float* hrow = hs_s + b * kD + half * 32;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float4 hv = *reinterpret_cast<const float4*>(hrow + 4 * e);
+                    a[4 * e + 0] = fmaf(a[4 * e + 0], rq, hv.x) * inv; a[4 * e + 1] = fmaf(a[4 * e + 1], rq, hv.y) * inv;
+                    a[4 * e + 2] = fmaf(a[4 * e + 2], rq, hv.z) * inv; a[4 * e + 3] = fmaf(a[4 * e + 3], rq, hv.w) * inv;
+                }
+            }
+            const float rqm = RN ? 1.0f : rq;  // RN: the scale has been applied above
 #pragma unroll
             for (int e = 0; e < 4; ++e) {  // 8 channels -> one 16-byte chunk of the bf16 row
                 const float4 c0 = *reinterpret_cast<const float4*>(srow + e * 32);
                 const float4 c1 = *reinterpret_cast<const float4*>(srow + e * 32 + 16);
                 uint4 pk;
-                pk.x = pack_bf16x2(fmaf(a[8 * e + 0], rq, c0.x), fmaf(a[8 * e + 1], rq, c0.y));
-                pk.y = pack_bf16x2(fmaf(a[8 * e + 2], rq, c0.z), fmaf(a[8 * e + 3], rq, c0.w));
-                pk.z = pack_bf16x2(fmaf(a[8 * e + 4], rq, c1.x), fmaf(a[8 * e + 5], rq, c1.y));
-                pk.w = pack_bf16x2(fmaf(a[8 * e + 6], rq, c1.z), fmaf(a[8 * e + 7], rq, c1.w));
+                pk.x = pack_bf16x2(fmaf(a[8 * e + 0], rqm, c0.x), fmaf(a[8 * e + 1], rqm, c0.y));
+                pk.y = pack_bf16x2(fmaf(a[8 * e + 2], rqm, c0.z), fmaf(a[8 * e + 3], rqm, c0.w));
+                pk.z = pack_bf16x2(fmaf(a[8 * e + 4], rqm, c1.x), fmaf(a[8 * e + 5], rqm, c1.y));
+                pk.w = pack_bf16x2(fmaf(a[8 * e + 6], rqm, c1.z), fmaf(a[8 * e + 7], rqm, c1.w));
                 *reinterpret_cast<uint4*>(orow + (((half * 4 + e) ^ (row & 7)) << 4)) = pk;
             }
             tcgen05_fence_before_sync();
@@ -306,7 +354,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         constexpr int kCX = kTX / 2;
         constexpr int R = G::R, RO = G::kConvRows, ROWS = RO + 2 * R;
         float2 wreg[KS][KS];
-        float2 cinit = make_float2(0.f, 0.f);
+        float2 cinit = make_float2(0.f, 0.f), hs2 = make_float2(0.f, 0.f);
         int prev_bh = -1;
         pdl_wait_primary();  // the token sums of the state kernel are read below
         PatchWalk pw(g_begin, prm.tilesX, prm.tilesY);
@@ -320,7 +368,7 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const int gbh = prm.bh0 + bh;
                 const int cp2 = PAIR ? 2 * (lane & 15) : 2 * lane;
                 const int ch = ((prm.head0 + gbh) % prm.H) * (PAIR ? 32 : kD) + cp2;
-                const float* sv = prm.state + (size_t)gbh * prm.P * (kD * kD + kD) + kD * kD;
+                const float* sv = prm.state + (size_t)gbh * prm.P * kSW + kD * kD;
                 float s0, s1;
                 if (PAIR) {  // token sum = sum of the two halves of the paired sums
                     s0 = __ldg(sv + cp2) + __ldg(sv + 32 + cp2);
@@ -328,11 +376,12 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 } else {
                     s0 = __ldg(sv + cp2); s1 = __ldg(sv + cp2 + 1);
                     for (int pp = 1; pp < prm.P; ++pp) {
-                        s0 += __ldg(sv + pp * (kD * kD + kD) + cp2);
-                        s1 += __ldg(sv + pp * (kD * kD + kD) + cp2 + 1);
+                        s0 += __ldg(sv + pp * kSW + cp2);
+                        s1 += __ldg(sv + pp * kSW + cp2 + 1);
                     }
                 }
-                cinit.x = 0.5f * s0; cinit.y = 0.5f * s1;
+                cinit.x = RN ? 0.f : 0.5f * s0; cinit.y = RN ? 0.f : 0.5f * s1;
+                hs2 = make_float2(0.5f * s0, 0.5f * s1);
                 if (prm.bias) { cinit.x += __bfloat162float(prm.bias[ch]); cinit.y += __bfloat162float(prm.bias[ch + 1]); }
 #pragma unroll
                 for (int dy = 0; dy < KS; ++dy)
@@ -384,16 +433,21 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int r = 0; r < RO; ++r) *reinterpret_cast<float2*>(so + (r * kTX + x) * kStgStride) = acc[r];
             }
+            if (RN && cw == 0 && xh == 0) {
+                // 1/2 s of the plane this patch belongs to, per column of a 128-byte row, beside the staging buffer
+                const int col = PAIR ? (lane >> 4) * 32 + 2 * (lane & 15) : 2 * lane;
+                *reinterpret_cast<float2*>(hs_s + b * kD + col) = hs2;
+            }
             mbar_arrive(&empty[s]);      // the V patch of this stage is no longer needed
             mbar_arrive(&conv_full[b]);
         }
     }
     tcgen05_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 1) tmem_dealloc(tmem, RN ? 2 * kTmemCols : kTmemCols);
 }
 
-template <int KS, int MODE>
+template <int KS, int MODE, bool RN>
 cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigned* status, cudaStream_t st) {
     constexpr bool PAIR = (MODE == 1);
     using G = Geo<KS, PAIR>;
@@ -430,10 +484,11 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0; prm.hdiv = p.hdiv;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
-    prm.eps2 = p.eps2; prm.status = status;
+    prm.eps2 = p.eps2; prm.status = status; prm.n_tokens = p.N;
+    constexpr size_t kSmemBytes = RN ? G::kSmemRN : G::kSmem;
     static PerDevice opt_in;  // one per instantiation
     {
-        const cudaError_t e = opt_in_smem(tc_apply_kernel<KS, MODE>, G::kSmem, opt_in);
+        const cudaError_t e = opt_in_smem(tc_apply_kernel<KS, MODE, RN>, kSmemBytes, opt_in);
         if (e != cudaSuccess) return e;
     }
     const int sms = device_sm_count();  // one persistent CTA per multiprocessor
@@ -441,12 +496,12 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     // programmatic dependent launch: this grid's prologue and first Q / V loads overlap the tail of
     // the state kernel; the warps that read its results wait for it (griddepcontrol.wait) first
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(G::kThreads); cfg.dynamicSmemBytes = G::kSmem; cfg.stream = st;
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(G::kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS, MODE>, tmQ, tmV, tmO, prm);
+    return cudaLaunchKernelEx(&cfg, tc_apply_kernel<KS, MODE, RN>, tmQ, tmV, tmO, prm);
 }
 
 // Output rows of the off-grid leading tokens: out = q^ S / pi + 1/2 s (no convolution, no bias), from the
@@ -501,15 +556,22 @@ cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_
     return cudaGetLastError();
 }
 
-cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st) {
+namespace {
+template <bool RN>
+cudaError_t launch_apply_rn(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st) {
     if (p.d == 32)
-        return p.ksize == 3 ? launch_apply_ks<3, 1>(p, partial, P, status, st)
-                            : launch_apply_ks<5, 1>(p, partial, P, status, st);
+        return p.ksize == 3 ? launch_apply_ks<3, 1, RN>(p, partial, P, status, st)
+                            : launch_apply_ks<5, 1, RN>(p, partial, P, status, st);
     if (p.blockdiag)
-        return p.ksize == 3 ? launch_apply_ks<3, 2>(p, partial, P, status, st)
-                            : launch_apply_ks<5, 2>(p, partial, P, status, st);
-    return p.ksize == 3 ? launch_apply_ks<3, 0>(p, partial, P, status, st)
-                        : launch_apply_ks<5, 0>(p, partial, P, status, st);
+        return p.ksize == 3 ? launch_apply_ks<3, 2, RN>(p, partial, P, status, st)
+                            : launch_apply_ks<5, 2, RN>(p, partial, P, status, st);
+    return p.ksize == 3 ? launch_apply_ks<3, 0, RN>(p, partial, P, status, st)
+                        : launch_apply_ks<5, 0, RN>(p, partial, P, status, st);
+}
+}  // namespace
+
+cudaError_t launch_apply(const Problem& p, const float* partial, int P, unsigned* status, cudaStream_t st) {
+    return p.rownorm ? launch_apply_rn<true>(p, partial, P, status, st) : launch_apply_rn<false>(p, partial, P, status, st);
 }
 
 }  // namespace tc

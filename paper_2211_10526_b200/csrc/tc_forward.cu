@@ -24,6 +24,7 @@ bool head_pairs(const Problem& p) {
 // bf16, 3x3 or 5x5 filters, head width 64 or one of the two width-32 arrangements above.
 bool supports(const Problem& p) {
     if (!p.bf16 || (p.ksize != 3 && p.ksize != 5)) return false;
+    if (p.rownorm && p.prefix != 0) return false;  // the rows of leading tokens are not written with the row-sum division
     return p.d == 64 || token_pairs(p) || head_pairs(p);
 }
 
@@ -73,7 +74,7 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
         p.lq.head = p.lk.head = p.lv.head = p.lo.head = 64;
         P = choose_splits(p.BH, p.N);
     }
-    if (fused_supports(p)) {  // a whole (b,h) fits in shared memory: one kernel, no workspace
+    if (!p.rownorm && fused_supports(p)) {  // a whole (b,h) fits in shared memory: one kernel, no workspace
         const cudaError_t e = launch_fused(p, status, stream);
         if (e != cudaSuccess) return e;
         ++*launches;
@@ -81,14 +82,14 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
         return cudaSuccess;
     }
     cudaError_t e;
-    if (const int C = cluster_enabled() ? cluster_size(p) : 0) {
+    if (const int C = (cluster_enabled() && !p.rownorm) ? cluster_size(p) : 0) {
         e = launch_cluster(p, C, status, stream);
         if (e != cudaSuccess) return e;
         ++*launches;
         timer->mark(stream, "tc_cluster");
         return cudaSuccess;
     }
-    if (!two_kernels() && pipe_supports(p)) {
+    if (!two_kernels() && !p.rownorm && pipe_supports(p)) {
         // state and apply pipelines in one persistent kernel: V is read from memory once
         e = launch_pipe(p, ws_state, ws_partial, counters, status, stream);
         if (e != cudaSuccess) return e;

@@ -29,8 +29,11 @@ bool preferred(const Problem& p);
 // 128-byte rows per (b,h): N for d = 64, N / 2 for d = 32 (two tokens per row).
 int rows_per_head(int N, int d);
 
-// Words of one (b,h) state as the tensor-core kernels store it (always the 64-wide form).
+// Words of one (b,h) state as the tensor-core kernels store it (always the 64-wide form): S, s, and with row-sum
+// normalisation the sum of the unit key rows behind them.
 constexpr int kStateWords = 64 * 64 + 64;
+constexpr int kStateWordsRownorm = kStateWords + 64;
+inline int state_words_of(const Problem& p) { return p.rownorm ? kStateWordsRownorm : kStateWords; }
 
 // Token splits of the tensor-core state kernel and the workspace words it needs beyond the state.
 int choose_splits(int BH, int N);

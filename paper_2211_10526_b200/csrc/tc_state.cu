@@ -7,6 +7,9 @@
 // features, row 64 is all ones, which makes row 64 of the accumulator the token sum of V) and
 // B = V (tokens x 64, N-major).  The fp32 accumulator lives in TMEM for the CTA's whole token
 // range and is written once, as this split's partial state.
+// RN (row-sum normalisation, Eq. 3's denominator on the kept kernel of Eq. 8) also needs sum_n k^_n: B gets a
+// second 64-wide block along N from the same constant block ([V | 1 0 0 ...]), so column 64 of the accumulator is
+// the row sum of A: rows 0..63 of it are sum_n k^_n, and the state has 64 more words.
 #include "tc_common.cuh"
 #include "tc_host.cuh"
 
@@ -21,7 +24,7 @@ constexpr int kTileBytes = kTile * kD * 2;   // 16 KiB per operand tile
 constexpr int kStageBytes = 2 * kTileBytes;  // K then V
 constexpr int kOnesBytes = 2048;             // 16 token rows x 128 B: feature 64 = 1, 65..127 = 0
 constexpr int kThreads = 192;                // warp 0 TMA, warp 1 UMMA, warps 2..5 scale + epilogue
-constexpr int kTmemCols = 128;                // two 64-column accumulators: a CTA may serve several (b,h)
+constexpr int kTmemCols = 128;                // two 64-column accumulators: a CTA may serve several (b,h) (RN: twice that)
 constexpr int kGroup = 4;                    // splits per first-level reduction group
 constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 
@@ -32,7 +35,7 @@ constexpr size_t kSmemBytes = 1024 + kStages * kStageBytes + kOnesBytes + 256;
 // reads them.  Each half row is normalised by its own token's norm.
 // The same instantiation serves two width-32 heads stored side by side in one 128-byte row (head
 // stride 32): identical arithmetic; there the consumers keep the two diagonal blocks apart, one per head.
-template <bool PAIR>
+template <bool PAIR, bool RN>
 __global__ void __launch_bounds__(kThreads, 2)
 tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 float* __restrict__ dst, float* __restrict__ final_state, unsigned* __restrict__ counters,
@@ -48,6 +51,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_free + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+    constexpr int kAcc = RN ? 2 * kD : kD;                 // accumulator columns
+    constexpr int kStateW = kD * kD + kD + (RN ? kD : 0);  // words of one state: S, s, (RN) sum of the unit key rows
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // Work items.  With P > 1 a CTA serves one (b,h, split).  With P == 1 (many heads, few tokens) a CTA
     // serves items_per_cta consecutive (b,h) one after another, so that barrier set-up, TMEM allocation
@@ -62,8 +67,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (n_tiles <= 0 || n_items <= 0) {  // the host never makes such a CTA; keep the partial well defined anyway
         pdl_wait_primary();
         if (P > 1) {
-            float* out = dst + ((size_t)bh * P + p) * (kD * kD + kD);
-            for (int i = tid; i < kD * kD + kD; i += kThreads) out[i] = 0.f;
+            float* out = dst + ((size_t)bh * P + p) * kStateW;
+            for (int i = tid; i < kStateW; i += kThreads) out[i] = 0.f;
         }
         return;
     }
@@ -81,7 +86,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmV);
     }
-    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 1) tmem_alloc(tmem_slot, RN ? 2 * kTmemCols : kTmemCols);
     if (warp >= 2) {
         // constant block of A: for each of 16 token rows, element 64 (first of the second 64-wide
         // block along M) is 1.0 and the rest 0; 16-byte chunk c of row r sits at chunk c ^ (r & 7)
@@ -129,7 +134,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, kD, true, true);
+            constexpr uint32_t idesc = umma_idesc_bf16(128, kAcc, true, true);
             const uint32_t ones_addr = smem_u32(ones);
             bool ok = true;
             int gt = 0;  // tiles issued so far, over all items
@@ -146,8 +151,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     for (int j = 0; j < kTile / 16; ++j) {  // one UMMA per 16 tokens (K = 16)
                         const uint32_t a0 = ka + j * 2048, b0 = va + j * 2048;
                         const uint64_t a = umma_desc_sw128(a0, ones_addr - a0, 1024);
-                        const uint64_t b = umma_desc_sw128(b0, 0, 1024);
-                        umma_bf16(tmem + buf * kD, a, b, idesc, (it | j) != 0);
+                        const uint64_t b = umma_desc_sw128(b0, RN ? ones_addr - b0 : 0, 1024);
+                        umma_bf16(tmem + buf * kAcc, a, b, idesc, (it | j) != 0);
                     }
                     umma_commit(&empty[s]);
                 }
@@ -166,18 +171,24 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             if (!mbar_wait(&accum[buf], (item >> 1) & 1, abort_flag, status, kStatusStateTimeout)) return false;
             tcgen05_fence_after_sync();
             if (quarter < 3) {
-                float* out = dst + ((size_t)(bh0 + item) * P + p) * (kD * kD + kD);
+                float* out = dst + ((size_t)(bh0 + item) * P + p) * kStateW;
                 const int row = quarter * 32 + lane;
 #pragma unroll
                 for (int cc = 0; cc < kD / 16; ++cc) {
                     float v[16];
-                    tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + buf * kD + cc * 16, v);
+                    tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + buf * kAcc + cc * 16, v);
                     tmem_ld_wait();
                     if (row <= kD) {
                         float4* o4 = reinterpret_cast<float4*>(out + row * kD + cc * 16);  // row 64 lands on s
 #pragma unroll
                         for (int e = 0; e < 4; ++e) o4[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
                     }
+                }
+                if (RN) {  // column 64: the row sums of A; rows 0..63 are sum_n k^_n, stored behind s
+                    float v[16];
+                    tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + buf * kAcc + kD, v);
+                    tmem_ld_wait();
+                    if (row < kD) out[kD * kD + kD + row] = v[0];
                 }
             }
             tcgen05_fence_before_sync();
@@ -232,7 +243,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
     tcgen05_fence_before_sync();
     __syncthreads();  // every thread's part of this split's partial state has been stored
-    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 1) tmem_dealloc(tmem, RN ? 2 * kTmemCols : kTmemCols);
 
     // Cross-split reduction without a second launch and without any waiting, as a two-level tree
     // driven by arrival counters: the splits of a (b,h) form groups of kGroup; the CTA that arrives
@@ -242,7 +253,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // Every counter is put back to zero by the CTA that consumed it.
     if (P > 1 && !*abort_flag) {
         __shared__ int is_last;
-        constexpr int kWords = kD * kD + kD, kWords4 = kWords / 4, kIter = (kWords4 + kThreads - 1) / kThreads;
+        constexpr int kWords = kStateW, kWords4 = kWords / 4, kIter = (kWords4 + kThreads - 1) / kThreads;
         unsigned* cnt = counters + (size_t)bh * kCountersPerHead;
         const int n_groups = (P + kGroup - 1) / kGroup, grp = p / kGroup;
         const int first = grp * kGroup, members = min(kGroup, P - first);
@@ -352,10 +363,12 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
                             (uint64_t)(nb > 1 ? p.lv.batch : p.lv.head * p.hdiv)};
     if (!make_tensor_map_bf16(&tmK, p.k, 4, dims, sk, box, true) || !make_tensor_map_bf16(&tmV, p.v, 4, dims, sv, box, true))
         return cudaErrorNotSupported;
-    static PerDevice opt_in[2];
+    static PerDevice opt_in[4];
     {
-        const cudaError_t e = halves ? opt_in_smem(tc_state_kernel<true>, kSmemBytes, opt_in[1])
-                                     : opt_in_smem(tc_state_kernel<false>, kSmemBytes, opt_in[0]);
+        const cudaError_t e = p.rownorm ? (halves ? opt_in_smem(tc_state_kernel<true, true>, kSmemBytes, opt_in[3])
+                                                  : opt_in_smem(tc_state_kernel<false, true>, kSmemBytes, opt_in[2]))
+                                        : (halves ? opt_in_smem(tc_state_kernel<true, false>, kSmemBytes, opt_in[1])
+                                                  : opt_in_smem(tc_state_kernel<false, false>, kSmemBytes, opt_in[0]));
         if (e != cudaSuccess) return e;
     }
     float* dst = P > 1 ? partial : final_state;
@@ -372,11 +385,12 @@ cudaError_t launch_state(const Problem& p, float* partial, float* final_state, u
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (halves)
-        return cudaLaunchKernelEx(&cfg, tc_state_kernel<true>, tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P,
-                                  p.BH, p.hdiv, items, p.eps2, status);
-    return cudaLaunchKernelEx(&cfg, tc_state_kernel<false>, tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P,
-                              p.BH, p.hdiv, items, p.eps2, status);
+    auto launch = [&](auto kernel) {
+        return cudaLaunchKernelEx(&cfg, kernel, tmK, tmV, dst, final_state, counters, rows, tiles_per_cta, P, p.BH, p.hdiv, items,
+                                  p.eps2, status);
+    };
+    if (p.rownorm) return halves ? launch(tc_state_kernel<true, true>) : launch(tc_state_kernel<false, true>);
+    return halves ? launch(tc_state_kernel<true, false>) : launch(tc_state_kernel<false, false>);
 }
 
 }  // namespace tc

@@ -103,6 +103,41 @@ def test_row_normalised_with_leading_tokens_and_strides():
     check(gpu_forward(c, layout="token_major", normalize_rows=True), ref, "bf16", "token-major")
 
 
+@pytest.mark.parametrize("path", [1, 2], ids=["cuda-core", "tensor-core"])
+@pytest.mark.parametrize("case", [(2, 8, 64, 64, 64, 3, "head_major"), (3, 4, 40, 56, 64, 5, "head_major"),
+                                  (2, 4, 64, 64, 32, 3, "head_major"), (2, 6, 48, 64, 32, 5, "head_major"),
+                                  (2, 6, 48, 64, 32, 3, "token_major")], ids=lambda t: "x".join(map(str, t)))
+def test_row_normalised_on_both_kernel_families(case, path):
+    """The row-sum division on the tensor-core kernels (sum of the unit key rows as one more accumulator column of the
+    state contraction, q . sum k^ as one more column of the apply contraction) and on the CUDA-core kernels, for every
+    packing of the tensor-core kernels; once with the filters and bias as drawn and once without them, so that the
+    divided attention term is the whole output."""
+    from paper_2211_10526_b200 import CastlingAttn
+    *shape, layout = case
+    for zero_conv in (False, True):
+        c = workloads.custom_call(*shape, "bf16", seed=8150 + shape[2])
+        if zero_conv:
+            c.dw_weight.zero_(); c.dw_bias.zero_()
+        s = c.shape
+        ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, threads=16)
+        dev = torch.device("cuda:0")
+        if layout == "head_major":
+            q, k, v = (t.to(dev) for t in (c.q, c.k, c.v))
+            out = torch.full_like(q, float("nan"))
+        else:
+            mk = lambda t: t.permute(0, 2, 1, 3).contiguous().to(dev).permute(0, 2, 1, 3)
+            q, k, v = mk(c.q), mk(c.k), mk(c.v)
+            out = torch.full((s.B, s.N, s.H, s.d), float("nan"), dtype=q.dtype, device=dev).permute(0, 2, 1, 3)
+        with CastlingAttn(ksize=s.ksize, normalize_rows=True, force_path=path) as attn:
+            attn.forward(q, k, v, c.dw_weight.to(dev), c.dw_bias.to(dev), s.gridH, s.gridW, out=out)
+            torch.cuda.synchronize()
+            assert attn.device_status() == (0, 0)
+            assert attn.last_path()[0] == path
+        got = out.double().cpu().numpy()
+        assert np.all(np.isfinite(got))
+        check(got, ref, "bf16", f"{s.label()} {layout} path {path} zero_conv={zero_conv}")
+
+
 QUAD_CALLS = [("c1_fp32_tiny", 0), ("c2_levit_bf16", 0), ("c2_levit_bf16", 1), ("c2_levit_bf16", 2),
               ("c3_deit_base_bf16", 0), ("c4_detection_bf16", 0), ("c5_sweep_bf16", 0), ("c5_sweep_bf16", 1)]
 QUAD_IDS = [f"{n}-{i}" for n, i in QUAD_CALLS]
