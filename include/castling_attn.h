@@ -246,8 +246,9 @@ CASTLING_API int castling_attn_device_status(castling_attn_t* handle, void* stre
  *               below; each of the two is 0 at the edge of the whole grid (zero padding applies there) and at
  *               most (ksize-1)/2, and must be (ksize-1)/2 wherever a neighbouring band exists.
  *   state       DEVICE, float [B*H][d*d + d]: the sum over all bands of what castling_attn_shard_state wrote.
- * Both enqueue on `stream` and return (the first call of a larger shape may allocate the workspace).  They run
- * on the CUDA-core kernels for every dtype.  A handle created with prefix tokens or any variant flag:
+ * Both enqueue on `stream` and return (the first call of a larger shape may allocate the workspace).  bf16 bands of
+ * width-64 heads with at least 48 tokens run on the tensor-core kernels (unless the handle is pinned to
+ * CASTLING_PATH_SIMT), everything else on the CUDA-core kernels.  A handle created with prefix tokens or any variant flag:
  * UNSUPPORTED.  Pointers 16-byte aligned.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, OOM, CUDA.
  */
 CASTLING_API size_t castling_attn_state_words(int d);

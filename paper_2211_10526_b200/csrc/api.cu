@@ -498,10 +498,24 @@ int castling_attn_shard_state(castling_attn_t* h, const void* k, const void* v, 
     float* partial = h->ws + castling::kHeaderWords + (size_t)p.BH * castling::state_words(p.d);
     int launches = 0;
     h->timer.begin(static_cast<cudaStream_t>(stream));
-    const cudaError_t e = castling::simt_forward(p, state_out, partial, castling::simt_choose_splits(p.BH, p.N),
-                                                 static_cast<cudaStream_t>(stream), &launches, &h->timer);
+    bool tensor = h->cfg.force_path != CASTLING_PATH_SIMT && castling::tc::shard_supports(p);
+    cudaError_t e = cudaSuccess;
+    if (tensor) {
+        rc = ensure_counters(h, p.BH);
+        if (rc != CASTLING_OK) return rc;
+        // the partial states of the tensor-core kernel follow BH final-state slots of its own size
+        partial = h->ws + castling::kHeaderWords + (size_t)p.BH * castling::tc::kStateWords;
+        e = castling::tc::shard_state(p, state_out, partial, h->counters, reinterpret_cast<unsigned*>(h->ws),
+                                      static_cast<cudaStream_t>(stream), &launches, &h->timer);
+        if (e == cudaErrorNotSupported) { (void)cudaGetLastError(); tensor = false; h->timer.begin(static_cast<cudaStream_t>(stream)); }
+    }
+    if (!tensor) {
+        partial = h->ws + castling::kHeaderWords + (size_t)p.BH * castling::state_words(p.d);
+        e = castling::simt_forward(p, state_out, partial, castling::simt_choose_splits(p.BH, p.N),
+                                   static_cast<cudaStream_t>(stream), &launches, &h->timer);
+    }
     if (e != cudaSuccess) return fail_cuda(h, e);
-    h->last_path = CASTLING_PATH_SIMT; h->last_launches = launches;
+    h->last_path = tensor ? CASTLING_PATH_TENSOR : CASTLING_PATH_SIMT; h->last_launches = launches;
     return CASTLING_OK;
 }
 
@@ -523,10 +537,20 @@ int castling_attn_shard_apply(castling_attn_t* h, const void* q, const void* v_h
     p.lv.head = (long long)p.v_rows * gridW * d;   // planes of the taller V tensor
     int launches = 0;
     h->timer.begin(static_cast<cudaStream_t>(stream));
-    const cudaError_t e = castling::simt_forward(p, const_cast<float*>(state), nullptr, 1, static_cast<cudaStream_t>(stream),
-                                                 &launches, &h->timer);
+    bool tensor = h->cfg.force_path != CASTLING_PATH_SIMT && castling::tc::shard_supports(p);
+    cudaError_t e = cudaSuccess;
+    if (tensor) {
+        rc = ensure_workspace(h, 1, 64, 64, true);  // the status word lives at the head of the workspace
+        if (rc != CASTLING_OK) return rc;
+        e = castling::tc::shard_apply(p, state, reinterpret_cast<unsigned*>(h->ws), static_cast<cudaStream_t>(stream),
+                                      &launches, &h->timer);
+        if (e == cudaErrorNotSupported) { (void)cudaGetLastError(); tensor = false; h->timer.begin(static_cast<cudaStream_t>(stream)); }
+    }
+    if (!tensor)
+        e = castling::simt_forward(p, const_cast<float*>(state), nullptr, 1, static_cast<cudaStream_t>(stream), &launches,
+                                   &h->timer);
     if (e != cudaSuccess) return fail_cuda(h, e);
-    h->last_path = CASTLING_PATH_SIMT; h->last_launches = launches;
+    h->last_path = tensor ? CASTLING_PATH_TENSOR : CASTLING_PATH_SIMT; h->last_launches = launches;
     return CASTLING_OK;
 }
 

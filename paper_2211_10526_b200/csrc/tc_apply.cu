@@ -66,6 +66,8 @@ struct ApplyParams {
     int H, head0, bh0, hdiv, tilesX, tilesY, n_tiles;  // tiles of (b,h) in [bh0, bh0 + n_tiles / (tilesX*tilesY))
     float eps2;
     unsigned* status;
+    int v_row0;                    // V holds more grid rows than the plane has (a band of a sharded sequence with its
+                                   // neighbours' rows): its row v_row0 is grid row 0
     int n_tokens;                  // tokens per sequence (row-sum normalisation: the sum of the constant 1/2 terms is n_tokens / 2)
 };
 
@@ -155,11 +157,11 @@ tc_apply_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 mbar_expect_tx(&full[s], kQBytes + G::kVBytes);
                 if (prm.flat) {
                     tma_load_4d_hint(qs, &tmQ, &full[s], 0, x0, y0, bh, pol_q);
-                    tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, bh);
+                    tma_load_4d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R + prm.v_row0, bh);
                 } else {
                     const int pb = bh / prm.hdiv, ph = bh - pb * prm.hdiv;
                     tma_load_5d_hint(qs, &tmQ, &full[s], 0, x0, y0, ph, pb, pol_q);
-                    tma_load_5d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R, ph, pb);
+                    tma_load_5d(qs + kQBytes, &tmV, &full[s], 0, x0 - G::HC, y0 - G::R + prm.v_row0, ph, pb);
                 }
                 ++issued;
             }
@@ -472,8 +474,11 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + p.prefix * p.lq.token;
     const __nv_bfloat16* vg = static_cast<const __nv_bfloat16*>(p.v) + p.prefix * p.lv.token;
     __nv_bfloat16* og = static_cast<__nv_bfloat16*>(p.out) + p.prefix * p.lo.token;
+    // V may hold more grid rows than the plane (the neighbours' rows of a band of a sharded sequence): rows outside
+    // that taller tensor, not outside the band, are the zero padding
+    uint64_t dimsv[5] = {dims[0], dims[1], (uint64_t)(p.v_rows > 0 ? p.v_rows : p.gridH), dims[3], dims[4]};
     if (!make_tensor_map_bf16(&tmQ, qg, rank, dims, sq, box, true) || !make_tensor_map_bf16(&tmO, og, rank, dims, so, box, true) ||
-        !make_tensor_map_bf16(&tmV, vg, rank, dims, sv, boxv, false))
+        !make_tensor_map_bf16(&tmV, vg, rank, dimsv, sv, boxv, false))
         return cudaErrorNotSupported;
     ApplyParams prm;
     prm.state = state;
@@ -484,7 +489,7 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
     prm.H = p.H; prm.head0 = p.head0; prm.bh0 = 0; prm.hdiv = p.hdiv;
     prm.tilesX = (cols + kTX - 1) / kTX; prm.tilesY = (p.gridH + kTY - 1) / kTY;
     prm.n_tiles = p.BH * prm.tilesX * prm.tilesY;
-    prm.eps2 = p.eps2; prm.status = status; prm.n_tokens = p.N;
+    prm.eps2 = p.eps2; prm.status = status; prm.n_tokens = p.N; prm.v_row0 = p.v_rows > 0 ? p.v_row0 : 0;
     constexpr size_t kSmemBytes = RN ? G::kSmemRN : G::kSmem;
     static PerDevice opt_in;  // one per instantiation
     {

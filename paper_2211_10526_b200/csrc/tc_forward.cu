@@ -116,5 +116,31 @@ cudaError_t forward(const Problem& p_in, float* ws_state, float* ws_partial, uns
     return cudaSuccess;
 }
 
+bool shard_supports(const Problem& p) {
+    return p.bf16 && p.d == 64 && (p.ksize == 3 || p.ksize == 5) && p.prefix == 0 && !p.rownorm && p.N >= 48;
+}
+
+cudaError_t shard_state(const Problem& p, float* state_out, float* ws_partial, unsigned* counters, unsigned* status,
+                        cudaStream_t stream, int* launches, KernelTimer* timer) {
+    *launches = 0;
+    const int P = choose_splits(p.BH, p.N);
+    const int tiles = (p.N + kStateTile - 1) / kStateTile;
+    const cudaError_t e = launch_state(p, ws_partial, state_out, counters, P, (tiles + P - 1) / P, status, stream);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    timer->mark(stream, "tc_state");
+    return cudaSuccess;
+}
+
+cudaError_t shard_apply(const Problem& p, const float* state, unsigned* status, cudaStream_t stream, int* launches,
+                        KernelTimer* timer) {
+    *launches = 0;
+    const cudaError_t e = launch_apply(p, state, 1, status, stream);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    timer->mark(stream, "tc_apply");
+    return cudaSuccess;
+}
+
 }  // namespace tc
 }  // namespace castling

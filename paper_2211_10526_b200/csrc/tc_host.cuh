@@ -44,6 +44,15 @@ int choose_splits(int BH, int N);
 cudaError_t forward(const Problem& p, float* ws_state, float* ws_partial, unsigned* counters, int P,
                     unsigned* status, cudaStream_t stream, int* launches, KernelTimer* timer);
 
+// The two halves of a forward on their own (a sequence sharded over devices): the state of a shard's tokens, written
+// to state_out in the documented layout (S row-major, then s), and the apply pass over a band of grid rows with a
+// state summed over all shards.  Head width 64 only (the width-32 packings keep their states in another form).
+bool shard_supports(const Problem& p);
+cudaError_t shard_state(const Problem& p, float* state_out, float* ws_partial, unsigned* counters, unsigned* status,
+                        cudaStream_t stream, int* launches, KernelTimer* timer);
+cudaError_t shard_apply(const Problem& p, const float* state, unsigned* status, cudaStream_t stream, int* launches,
+                        KernelTimer* timer);
+
 // Launchers of the individual kernels (each in its own file).
 cudaError_t launch_state(const Problem& p, float* partial, float* final_state, unsigned* counters, int P,
                          int tiles_per_cta, unsigned* status, cudaStream_t st);
