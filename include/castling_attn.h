@@ -86,7 +86,7 @@ typedef struct {
                           /* of kernel-based linear attention (Sec. 3.1, Eq. 3) that Eq. 9 leaves out: */
                           /* the attention term of token t is divided by N/2 + q^_t . (sum_j k^_j)/pi; */
                           /* the convolution is added unchanged.  bf16 shapes that the tensor-core    */
-                          /* kernels take run there (without leading tokens); the rest on CUDA cores. */
+                          /* kernels take run there; the rest on the CUDA-core kernels.               */
     int exact_kernel;     /* 1: the exact angular kernel 1 - arccos(q^.k^)/pi (Eq. 4-5) instead of its  */
                           /* kept part 1/2 + q^.k^/pi (Eq. 8).  Quadratic in N (explicit weights).     */
     int sparse_branch;    /* 1: the auxiliary branch of training (Sec. 3.2.2, Eq. 10) is added to the   */

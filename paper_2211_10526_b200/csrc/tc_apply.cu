@@ -516,7 +516,7 @@ cudaError_t launch_apply_ks(const Problem& p, const float* state, int P, unsigne
 __global__ void __launch_bounds__(64)
 tc_prefix_rows_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
                       const float* __restrict__ state, Layout lq, Layout lo, int hdiv, int prefix, int mode,
-                      float eps2) {
+                      float eps2, int rownorm, int n_tokens) {
     __shared__ float qs[kD];
     __shared__ float part[2];
     const int plane = blockIdx.x / prefix, t = blockIdx.x % prefix, j = threadIdx.x;
@@ -530,23 +530,29 @@ tc_prefix_rows_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __rest
     if ((j & 31) == 0) part[j >> 5] = ss;
     __syncthreads();
     if (j >= width) return;
-    const float* st = state + (size_t)plane * (kD * kD + kD);
-    float nrm2, acc = 0.f, sum;
+    const float* st = state + (size_t)plane * (kD * kD + kD + (rownorm ? kD : 0));
+    const float* sk = st + kD * kD + kD;  // row-sum normalisation: sum of the unit key rows (per token parity / head)
+    float nrm2, acc = 0.f, sum, qk = 0.f;
     if (mode == 0) {
         nrm2 = part[0] + part[1];
         for (int i = 0; i < kD; ++i) acc = fmaf(qs[i], st[i * kD + j], acc);
         sum = st[kD * kD + j];
+        if (rownorm) for (int i = 0; i < kD; ++i) qk = fmaf(qs[i], sk[i], qk);
     } else if (mode == 1) {
         nrm2 = part[0];
         for (int i = 0; i < 32; ++i) acc = fmaf(qs[i], st[i * kD + j] + st[(32 + i) * kD + 32 + j], acc);
         sum = st[kD * kD + j] + st[kD * kD + 32 + j];
+        if (rownorm) for (int i = 0; i < 32; ++i) qk = fmaf(qs[i], sk[i] + sk[32 + i], qk);
     } else {
         const int h0 = j & 32;  // first channel of this thread's head within the row
         nrm2 = part[j >> 5];
         for (int i = 0; i < 32; ++i) acc = fmaf(qs[h0 + i], st[(h0 + i) * kD + j], acc);
         sum = st[kD * kD + j];
+        if (rownorm) for (int i = 0; i < 32; ++i) qk = fmaf(qs[h0 + i], sk[h0 + i], qk);
     }
-    const float o = fmaf(acc * kInvPi, rsqrtf(fmaxf(nrm2, eps2)), 0.5f * sum);
+    const float rq = rsqrtf(fmaxf(nrm2, eps2));
+    float o = fmaf(acc * kInvPi, rq, 0.5f * sum);
+    if (rownorm) o /= fmaf(qk * kInvPi, rq, 0.5f * (float)n_tokens);
     out[plane_offset(lo, plane, hdiv) + t * lo.token + j] = __float2bfloat16_rn(o);
 }
 
@@ -557,7 +563,7 @@ cudaError_t launch_prefix_rows(const Problem& p, const float* state, cudaStream_
     const int mode = p.d == 32 ? 1 : (p.blockdiag ? 2 : 0);
     tc_prefix_rows_kernel<<<(unsigned)(p.BH * p.prefix), 64, 0, st>>>(
         static_cast<const __nv_bfloat16*>(p.q), static_cast<__nv_bfloat16*>(p.out), state, p.lq, p.lo, p.hdiv,
-        p.prefix, mode, p.eps2);
+        p.prefix, mode, p.eps2, p.rownorm ? 1 : 0, p.N);
     return cudaGetLastError();
 }
 

@@ -24,7 +24,6 @@ bool head_pairs(const Problem& p) {
 // bf16, 3x3 or 5x5 filters, head width 64 or one of the two width-32 arrangements above.
 bool supports(const Problem& p) {
     if (!p.bf16 || (p.ksize != 3 && p.ksize != 5)) return false;
-    if (p.rownorm && p.prefix != 0) return false;  // the rows of leading tokens are not written with the row-sum division
     return p.d == 64 || token_pairs(p) || head_pairs(p);
 }
 

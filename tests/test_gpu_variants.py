@@ -98,6 +98,11 @@ def test_row_normalised_with_leading_tokens_and_strides():
     c = workloads.custom_call(2, 4, 1, 2 + 9 * 10, 32, 3, "f32", seed=8101)
     ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, 9, 10, 3, prefix=2)
     check(gpu_forward(c, prefix=2, grid=(9, 10), normalize_rows=True), ref, "f32", "leading tokens")
+    # bf16 with leading tokens on the tensor-core kernels: width 64, and width-32 token pairs (even number of leading tokens)
+    for d, prefix, gh, gw in ((64, 1, 20, 24), (32, 2, 20, 24)):
+        c = workloads.custom_call(2, 4, 1, prefix + gh * gw, d, 3, "bf16", seed=8103 + d)
+        ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, gh, gw, 3, prefix=prefix)
+        check(gpu_forward(c, prefix=prefix, grid=(gh, gw), normalize_rows=True, force_path=2), ref, "bf16", f"leading tokens, d={d}")
     c = workloads.custom_call(2, 4, 12, 14, 64, 5, "bf16", seed=8102)
     ref = oracle.forward_rownorm(c.q, c.k, c.v, c.dw_weight, c.dw_bias, 12, 14, 5)
     check(gpu_forward(c, layout="token_major", normalize_rows=True), ref, "bf16", "token-major")
