@@ -217,9 +217,25 @@ int run_device(castling_attn* h, const Problem& p, cudaStream_t stream) {
     if (p.exact_kernel || p.sparse) {
         // explicit attention weights: one kernel, no workspace; quadratic in the number of tokens
         if (p.N > 16384) return CASTLING_ERR_UNSUPPORTED;
-        if (h->cfg.force_path == CASTLING_PATH_TENSOR) return CASTLING_ERR_UNSUPPORTED;
+        const bool tensor_quad = castling::tc::quad_supports(p) && h->cfg.force_path != CASTLING_PATH_SIMT;
+        if (h->cfg.force_path == CASTLING_PATH_TENSOR && !tensor_quad) return CASTLING_ERR_UNSUPPORTED;
         int launches = 0;
         h->timer.begin(stream);
+        if (tensor_quad) {
+            // the exact kernel alone on bf16 heads of width 64: cosines and weighted sums on the tensor cores
+            const int rc = ensure_workspace(h, 1, 64, 64, true);  // the status word lives at the head of the workspace
+            if (rc != CASTLING_OK) return rc;
+            const cudaError_t eq = castling::tc::launch_quad(p, reinterpret_cast<unsigned*>(h->ws), stream);
+            if (eq == cudaSuccess) {
+                h->timer.mark(stream, "tc_quad");
+                h->last_path = CASTLING_PATH_TENSOR;
+                h->last_launches = 1;
+                return CASTLING_OK;
+            }
+            if (eq != cudaErrorNotSupported || h->cfg.force_path == CASTLING_PATH_TENSOR) return fail_cuda(h, eq);
+            (void)cudaGetLastError();  // strides the tensor maps cannot take: the CUDA-core kernel takes any layout
+            h->timer.begin(stream);
+        }
         const cudaError_t e = castling::quad_forward(p, stream, &launches, &h->timer);
         if (e == cudaErrorNotSupported) { (void)cudaGetLastError(); return CASTLING_ERR_UNSUPPORTED; }
         if (e != cudaSuccess) return fail_cuda(h, e);

@@ -95,6 +95,10 @@ cudaError_t launch_cluster(const Problem& p, int C, unsigned* status, cudaStream
 bool fused_supports(const Problem& p);
 cudaError_t launch_fused(const Problem& p, unsigned* status, cudaStream_t st);
 
+// Attention with the exact angular kernel on the tensor cores (csrc/tc_quad.cu): explicit weights, bf16, head width 64.
+bool quad_supports(const Problem& p);
+cudaError_t launch_quad(const Problem& p, unsigned* status, cudaStream_t st);
+
 // A one-CTA kernel whose bounded wait (limit_ns) can never be satisfied: it has to raise kStatusSelfTestTimeout in
 // *status and return; *reached_end becomes 1 (2 if the wait claimed success).
 cudaError_t launch_selftest_wait(unsigned* status, unsigned long long limit_ns, unsigned* reached_end, cudaStream_t st);

@@ -157,6 +157,42 @@ def test_exact_angular_kernel_configurations(name, idx):
     check(gpu_forward(c, exact_kernel=True), ref, s.dtype, f"{s.label()} exact kernel")
 
 
+@pytest.mark.parametrize("path", [1, 2], ids=["cuda-core", "tensor-core"])
+@pytest.mark.parametrize("case", [(2, 3, 16, 16, 64, 3, "head_major"), (1, 4, 25, 31, 64, 5, "head_major"),
+                                  (2, 2, 40, 48, 64, 3, "token_major"), (1, 2, 9, 11, 64, 3, "head_major")],
+                         ids=lambda t: "x".join(map(str, t)))
+def test_exact_kernel_on_both_kernel_families(case, path):
+    """The exact angular kernel on the tensor cores (cosines and weighted sums as UMMAs, weights through shared
+    memory) and on the CUDA cores: whole tiles, a ragged last tile of queries and keys, a plane smaller than a tile,
+    both filter sizes, a strided layout; with the filters as drawn, and without them, so that the attention term is
+    the whole output."""
+    from paper_2211_10526_b200 import CastlingAttn
+    *shape, layout = case
+    for zero_conv in (False, True):
+        c = workloads.custom_call(*shape, "bf16", seed=8300 + shape[2])
+        if zero_conv:
+            c.dw_weight.zero_(); c.dw_bias.zero_()
+        s = c.shape
+        ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize,
+                                    kernel=oracle.KERNEL_EXACT, threads=16)
+        dev = torch.device("cuda:0")
+        if layout == "head_major":
+            q, k, v = (t.to(dev) for t in (c.q, c.k, c.v))
+            out = torch.full_like(q, float("nan"))
+        else:
+            mk = lambda t: t.permute(0, 2, 1, 3).contiguous().to(dev).permute(0, 2, 1, 3)
+            q, k, v = mk(c.q), mk(c.k), mk(c.v)
+            out = torch.full((s.B, s.N, s.H, s.d), float("nan"), dtype=q.dtype, device=dev).permute(0, 2, 1, 3)
+        with CastlingAttn(ksize=s.ksize, exact_kernel=True, force_path=path) as attn:
+            attn.forward(q, k, v, c.dw_weight.to(dev), c.dw_bias.to(dev), s.gridH, s.gridW, out=out)
+            torch.cuda.synchronize()
+            assert attn.device_status() == (0, 0)
+            assert attn.last_path() == (path, 1)
+        got = out.double().cpu().numpy()
+        assert np.all(np.isfinite(got))
+        check(got, ref, "bf16", f"{s.label()} {layout} path {path} zero_conv={zero_conv}")
+
+
 @pytest.mark.parametrize("name,idx", QUAD_CALLS, ids=QUAD_IDS)
 def test_sparse_branch_configurations(name, idx):
     (c,) = list(workloads.iter_workload(name, only=[idx]))
