@@ -88,8 +88,9 @@ typedef struct {
                           /* the convolution is added unchanged.  bf16 shapes that the tensor-core    */
                           /* kernels take run there; the rest on the CUDA-core kernels.               */
     int exact_kernel;     /* 1: the exact angular kernel 1 - arccos(q^.k^)/pi (Eq. 4-5) instead of its  */
-                          /* kept part 1/2 + q^.k^/pi (Eq. 8).  Quadratic in N (explicit weights); on  */
-                          /* its own, for bf16 heads of width 64, it runs on the tensor cores.         */
+                          /* kept part 1/2 + q^.k^/pi (Eq. 8).  Quadratic in N (explicit weights).     */
+                          /* This flag and sparse_branch run on the tensor cores for bf16 heads of     */
+                          /* width 64 (without normalize_rows and leading tokens), else on CUDA cores. */
     int sparse_branch;    /* 1: the auxiliary branch of training (Sec. 3.2.2, Eq. 10) is added to the   */
                           /* weights: Mask_eps(Softmax_j(q^_t . k^_j)), Mask_eps(p) = p if p > eps else */
                           /* 0; softmax over the keys of a query on the cosines of the unit rows, no    */

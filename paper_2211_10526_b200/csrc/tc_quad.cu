@@ -11,6 +11,9 @@
 //                of the weights), bf16 weights into the shared-memory operand of the second contraction
 // and at the end of the item warps 6..9 (thread = query) read O, add bias and the depthwise convolution of V taken
 // from global memory, and store the row.  Keys beyond the plane have k^ = 0, weight 1/2 and v = 0: no masking.
+// With the auxiliary branch of training (Eq. 10) every item takes a first sweep over the keys that only forms the
+// cosines and adds up exp(cosine) per query (keys beyond the plane excluded); in the second sweep the weight of a pair
+// is the base weight (exact kernel, or its kept part 1/2 + x/pi) plus Mask_eps of its softmax probability.
 // No workspace; every wait is bounded.
 #include "tc_common.cuh"
 #include "tc_host.cuh"
@@ -29,7 +32,8 @@ constexpr int kThreads = 14 * 32;
 constexpr int kNormThreads = 128, kWThreads = 256;
 constexpr int kTmemCols = 512;                      // cosines: 2 x 128 columns; output: 64 columns at 256
 constexpr int kOffQ = 0, kOffStages = kTileBytes, kOffP = kOffStages + kStages * kStageBytes;
-constexpr int kOffBar = kOffP + 2 * kPBytes;
+constexpr int kOffDen = kOffP + 2 * kPBytes;        // softmax denominators: one partial sum per weight thread
+constexpr int kOffBar = kOffDen + 2 * kTile * 4;
 constexpr size_t kSmem = 1024 + kOffBar + 256;
 static_assert(kSmem <= 227 * 1024, "shared memory");
 
@@ -42,6 +46,8 @@ struct QuadParams {
     int hdiv, H, head0, BH, N, gridH, gridW, q_tiles, k_tiles, n_items;
     float eps2;
     unsigned* status;
+    int exact;              // base weight: 1 - arccos(x)/pi, else 1/2 + x/pi
+    float sparse_eps;       // threshold of the mask (sparse sweeps only)
 };
 
 // 1 - arccos(x) / pi for x in [-1, 1]
@@ -56,7 +62,7 @@ __device__ __forceinline__ float angular_weight(float x) {
     return x >= 0.f ? 1.0f - r : r;                           // arccos(-a) = pi - arccos(a)
 }
 
-template <int KS>
+template <int KS, bool SPARSE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const QuadParams prm) {
@@ -65,6 +71,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint8_t* Q_s = smem + kOffQ;
     uint8_t* stages = smem + kOffStages;
     uint8_t* P_s = smem + kOffP;
+    float* den_s = reinterpret_cast<float*>(smem + kOffDen);
     uint64_t* q_full = reinterpret_cast<uint64_t*>(smem + kOffBar);
     uint64_t* q_ready = q_full + 1;      // Q rows scaled (128)
     uint64_t* q_free = q_ready + 1;      // the item's last cosine UMMAs have read Q
@@ -77,12 +84,14 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint64_t* p_free = p_full + 2;           // [2]
     uint64_t* o_full = p_free + 2;
     uint64_t* o_free = o_full + 1;           // (128)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_free + 1);
+    uint64_t* den_bar = o_free + 1;          // (256) both halves of every query's denominator are in shared memory
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(den_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int my_items = ((int)blockIdx.x < prm.n_items) ? (prm.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
     const int KT = prm.k_tiles;
+    const int sweeps = SPARSE ? 2 : 1;   // key tiles per item: sweeps * KT; the last sweep feeds the second contraction
     constexpr unsigned kBit = kStatusFusedTimeout;
 
     if (tid == 0) {
@@ -91,7 +100,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         for (int b = 0; b < 2; ++b) {
             mbar_init(&c_full[b], 1); mbar_init(&c_free[b], kWThreads); mbar_init(&p_full[b], kWThreads); mbar_init(&p_free[b], 1);
         }
-        mbar_init(o_full, 1); mbar_init(o_free, kNormThreads);
+        mbar_init(o_full, 1); mbar_init(o_free, kNormThreads); mbar_init(den_bar, kWThreads);
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -112,13 +121,15 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (i > 0 && !mbar_wait(q_free, (i - 1) & 1, abort_flag, prm.status, kBit)) break;
                 mbar_expect_tx(q_full, kTileBytes);
                 tma_load_4d(Q_s, &tmQ, q_full, 0, qt * kTile, ph, pb);
-                for (int jt = 0; jt < KT; ++jt, ++g) {
+                for (int tt = 0; tt < sweeps * KT; ++tt, ++g) {
+                    const int jt = tt % KT;
+                    const bool with_v = tt >= (sweeps - 1) * KT;   // the first sweep of two needs the keys only
                     const int s = (int)(g % kStages), use = (int)(g / kStages);
                     if (use > 0 && !mbar_wait(&kv_empty[s], (use - 1) & 1, abort_flag, prm.status, kBit)) { ok = false; break; }
                     uint8_t* ks = stages + s * kStageBytes;
-                    mbar_expect_tx(&kv_full[s], kStageBytes);
+                    mbar_expect_tx(&kv_full[s], with_v ? kStageBytes : kTileBytes);
                     tma_load_4d(ks, &tmK, &kv_full[s], 0, jt * kTile, ph, pb);
-                    tma_load_4d(ks + kTileBytes, &tmV, &kv_full[s], 0, jt * kTile, ph, pb);
+                    if (with_v) tma_load_4d(ks + kTileBytes, &tmV, &kv_full[s], 0, jt * kTile, ph, pb);
                 }
             }
             if (*abort_flag) {  // giving up: let the copies in flight land before shared memory goes away
@@ -131,12 +142,12 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             constexpr uint32_t idesc_c = umma_idesc_bf16(128, 128, false, false);   // Q^ (K-major) x K^ (K-major)
             constexpr uint32_t idesc_o = umma_idesc_bf16(128, kD, false, true);     // W (K-major) x V (N-major)
             const uint32_t q_addr = smem_u32(Q_s), p_addr = smem_u32(P_s);
-            long long g = 0;
+            long long g = 0, gp = 0;   // key tiles so far: all of them / those that feed the second contraction
             bool ok = true;
-            // the second contraction of key tile g (of this CTA's sequence); first: the item's first tile
-            auto second = [&](long long gg, bool first) -> bool {
-                const int s = (int)(gg % kStages), pbuf = (int)(gg & 1);
-                if (!mbar_wait(&p_full[pbuf], (uint32_t)((gg >> 1) & 1), abort_flag, prm.status, kBit)) return false;
+            // the second contraction of the tile with ring number gg and weight-buffer number pp; first: the item's first
+            auto second = [&](long long gg, long long pp, bool first) -> bool {
+                const int s = (int)(gg % kStages), pbuf = (int)(pp & 1);
+                if (!mbar_wait(&p_full[pbuf], (uint32_t)((pp >> 1) & 1), abort_flag, prm.status, kBit)) return false;
                 tcgen05_fence_after_sync();
                 const uint32_t va = smem_u32(stages + s * kStageBytes + kTileBytes), pa = p_addr + pbuf * kPBytes;
 #pragma unroll
@@ -153,7 +164,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!mbar_wait(q_ready, i & 1, abort_flag, prm.status, kBit)) break;
                 // the previous item's output has been read out of TMEM before this item's first accumulation
                 if (i > 0 && !mbar_wait(o_free, (i - 1) & 1, abort_flag, prm.status, kBit)) break;
-                for (int jt = 0; jt < KT && ok; ++jt, ++g) {
+                for (int tt = 0; tt < sweeps * KT && ok; ++tt, ++g) {
+                    const bool last_sweep = tt >= (sweeps - 1) * KT;
+                    const int jt = tt % KT;
                     const int s = (int)(g % kStages), use = (int)(g / kStages), cb = (int)(g & 1);
                     ok = mbar_wait(&k_scaled[s], use & 1, abort_flag, prm.status, kBit);
                     if (ok && g >= 2) ok = mbar_wait(&c_free[cb], (uint32_t)(((g >> 1) - 1) & 1), abort_flag, prm.status, kBit);
@@ -167,10 +180,11 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         umma_bf16(tmem + cb * 128, a, b, idesc_c, k != 0);
                     }
                     umma_commit(&c_full[cb]);
+                    if (!last_sweep) { umma_commit(&kv_empty[s]); continue; }   // cosines only: the stage is free again
                     if (jt == KT - 1) umma_commit(q_free);
-                    if (jt > 0) ok = second(g - 1, jt == 1);   // one tile behind: the weight warps work meanwhile
+                    if (jt > 0) { ok = second(g - 1, gp, jt == 1); ++gp; }   // one tile behind: the weight warps work meanwhile
                 }
-                if (ok) ok = second(g - 1, KT == 1);
+                if (ok) { ok = second(g - 1, gp, KT == 1); ++gp; }
                 if (ok) umma_commit(o_full);
             }
         }
@@ -209,7 +223,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (!mbar_wait(q_full, i & 1, abort_flag, prm.status, kBit)) break;
             scale_row(Q_s + t * 128);
             mbar_arrive(q_ready);
-            for (int jt = 0; jt < KT; ++jt, ++g) {
+            for (int tt = 0; tt < sweeps * KT; ++tt, ++g) {
                 const int s = (int)(g % kStages), use = (int)(g / kStages);
                 if (!mbar_wait(&kv_full[s], use & 1, abort_flag, prm.status, kBit)) { ok = false; break; }
                 scale_row(stages + s * kStageBytes + t * 128);
@@ -220,15 +234,53 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // ---- weights: thread = (query row, 64 of the tile's 128 keys); at the end of an item half 0 writes the rows ----
         const int quarter = warp & 3, half = (warp - 6) >> 2, row = quarter * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
-        long long g = 0;
+        long long g = 0, gp = 0;
         bool ok = true;
+        const bool exact = prm.exact != 0;
         for (int i = 0; i < my_items && ok; ++i) {
             const int item = blockIdx.x + i * gridDim.x, bh = item / prm.q_tiles, qt = item - bh * prm.q_tiles;
-            for (int jt = 0; jt < KT; ++jt, ++g) {
-                const int cb = (int)(g & 1), pbuf = cb;
+            float inv_den = 0.f;
+            if (SPARSE) {
+                // first sweep: sum over the plane's keys of exp(cosine) for this thread's query, half of every tile
+                float den = 0.f;
+                for (int jt = 0; jt < KT; ++jt, ++g) {
+                    const int cb = (int)(g & 1);
+                    if (!mbar_wait(&c_full[cb], (uint32_t)((g >> 1) & 1), abort_flag, prm.status, kBit)) { ok = false; break; }
+                    tcgen05_fence_after_sync();
+                    const int key0 = jt * kTile + half * 64;
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        float x[16];
+                        tmem_ld16(lane_base + cb * 128 + half * 64 + cc * 16, x);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (key0 + cc * 16 + e < prm.N) den += __expf(fminf(fmaxf(x[e], -1.0f), 1.0f));
+                    }
+                    tcgen05_fence_before_sync();
+                    mbar_arrive(&c_free[cb]);
+                }
+                if (!ok) break;
+                den_s[half * kTile + row] = den;
+                mbar_arrive(den_bar);
+                if (!mbar_wait(den_bar, i & 1, abort_flag, prm.status, kBit)) break;
+                inv_den = 1.0f / (den_s[row] + den_s[kTile + row]);
+            }
+            // weight of a pair from its cosine
+            auto weight = [&](float xr) -> float {
+                const float x = fminf(fmaxf(xr, -1.0f), 1.0f);
+                float wv = exact ? angular_weight(x) : fmaf(x, kInvPi, 0.5f);
+                if (SPARSE) {
+                    const float pr = __expf(x) * inv_den;
+                    if (pr > prm.sparse_eps) wv += pr;
+                }
+                return wv;
+            };
+            for (int jt = 0; jt < KT; ++jt, ++g, ++gp) {
+                const int cb = (int)(g & 1), pbuf = (int)(gp & 1);
                 if (!mbar_wait(&c_full[cb], (uint32_t)((g >> 1) & 1), abort_flag, prm.status, kBit)) { ok = false; break; }
                 tcgen05_fence_after_sync();
-                if (g >= 2 && !mbar_wait(&p_free[pbuf], (uint32_t)(((g >> 1) - 1) & 1), abort_flag, prm.status, kBit)) { ok = false; break; }
+                if (gp >= 2 && !mbar_wait(&p_free[pbuf], (uint32_t)(((gp >> 1) - 1) & 1), abort_flag, prm.status, kBit)) { ok = false; break; }
                 uint8_t* prow = P_s + pbuf * kPBytes + half * kTileBytes + row * 128;
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
@@ -236,14 +288,14 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tmem_ld16(lane_base + cb * 128 + half * 64 + cc * 16, x);
                     tmem_ld_wait();
                     uint4 o0, o1;
-                    o0.x = pack_bf16x2(angular_weight(x[0]), angular_weight(x[1]));
-                    o0.y = pack_bf16x2(angular_weight(x[2]), angular_weight(x[3]));
-                    o0.z = pack_bf16x2(angular_weight(x[4]), angular_weight(x[5]));
-                    o0.w = pack_bf16x2(angular_weight(x[6]), angular_weight(x[7]));
-                    o1.x = pack_bf16x2(angular_weight(x[8]), angular_weight(x[9]));
-                    o1.y = pack_bf16x2(angular_weight(x[10]), angular_weight(x[11]));
-                    o1.z = pack_bf16x2(angular_weight(x[12]), angular_weight(x[13]));
-                    o1.w = pack_bf16x2(angular_weight(x[14]), angular_weight(x[15]));
+                    o0.x = pack_bf16x2(weight(x[0]), weight(x[1]));
+                    o0.y = pack_bf16x2(weight(x[2]), weight(x[3]));
+                    o0.z = pack_bf16x2(weight(x[4]), weight(x[5]));
+                    o0.w = pack_bf16x2(weight(x[6]), weight(x[7]));
+                    o1.x = pack_bf16x2(weight(x[8]), weight(x[9]));
+                    o1.y = pack_bf16x2(weight(x[10]), weight(x[11]));
+                    o1.z = pack_bf16x2(weight(x[12]), weight(x[13]));
+                    o1.w = pack_bf16x2(weight(x[14]), weight(x[15]));
                     *reinterpret_cast<uint4*>(prow + (((2 * cc) ^ (row & 7)) << 4)) = o0;
                     *reinterpret_cast<uint4*>(prow + (((2 * cc + 1) ^ (row & 7)) << 4)) = o1;
                 }
@@ -316,7 +368,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int KS>
+template <int KS, bool SPARSE>
 cudaError_t launch_quad_ks(const Problem& p, unsigned* status, cudaStream_t st) {
     CUtensorMap tmQ, tmK, tmV;
     const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
@@ -341,28 +393,30 @@ cudaError_t launch_quad_ks(const Problem& p, unsigned* status, cudaStream_t st) 
     prm.q_tiles = (p.N + kTile - 1) / kTile; prm.k_tiles = prm.q_tiles;
     prm.n_items = p.BH * prm.q_tiles;
     prm.eps2 = p.eps2; prm.status = status;
+    prm.exact = p.exact_kernel ? 1 : 0; prm.sparse_eps = p.sparse_eps;
     static PerDevice opt_in;
     {
-        const cudaError_t e = opt_in_smem(tc_quad_kernel<KS>, kSmem, opt_in);
+        const cudaError_t e = opt_in_smem(tc_quad_kernel<KS, SPARSE>, kSmem, opt_in);
         if (e != cudaSuccess) return e;
     }
     const int sms = device_sm_count();
     const int grid = prm.n_items < sms ? prm.n_items : sms;
-    tc_quad_kernel<KS><<<(unsigned)grid, kThreads, kSmem, st>>>(tmQ, tmK, tmV, prm);
+    tc_quad_kernel<KS, SPARSE><<<(unsigned)grid, kThreads, kSmem, st>>>(tmQ, tmK, tmV, prm);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-// bf16, head width 64 (16-byte aligned token rows), 3x3 or 5x5 filters, the exact kernel alone (no masked softmax branch,
-// no row-sum division), no leading tokens.
+// bf16, head width 64 (16-byte aligned token rows), 3x3 or 5x5 filters, explicit weights (exact kernel and / or the
+// masked softmax branch) without row-sum division, no leading tokens.
 bool quad_supports(const Problem& p) {
-    return p.bf16 && p.d == kD && (p.ksize == 3 || p.ksize == 5) && p.exact_kernel && !p.sparse && !p.rownorm &&
+    return p.bf16 && p.d == kD && (p.ksize == 3 || p.ksize == 5) && (p.exact_kernel || p.sparse) && !p.rownorm &&
            p.prefix == 0 && !p.blockdiag && (p.lv.token % 8) == 0 && (p.lo.token % 8) == 0;
 }
 
 cudaError_t launch_quad(const Problem& p, unsigned* status, cudaStream_t st) {
-    return p.ksize == 3 ? launch_quad_ks<3>(p, status, st) : launch_quad_ks<5>(p, status, st);
+    if (p.sparse) return p.ksize == 3 ? launch_quad_ks<3, true>(p, status, st) : launch_quad_ks<5, true>(p, status, st);
+    return p.ksize == 3 ? launch_quad_ks<3, false>(p, status, st) : launch_quad_ks<5, false>(p, status, st);
 }
 
 }  // namespace tc

@@ -193,6 +193,41 @@ def test_exact_kernel_on_both_kernel_families(case, path):
         check(got, ref, "bf16", f"{s.label()} {layout} path {path} zero_conv={zero_conv}")
 
 
+@pytest.mark.parametrize("path", [1, 2], ids=["cuda-core", "tensor-core"])
+@pytest.mark.parametrize("exact", [False, True], ids=["kept-kernel", "exact-kernel"])
+@pytest.mark.parametrize("case", [(2, 3, 2, 3, 64, 3), (2, 3, 4, 4, 64, 3), (1, 4, 5, 6, 64, 5), (2, 3, 16, 16, 64, 3),
+                                  (1, 4, 25, 31, 64, 5)], ids=lambda t: "x".join(map(str, t)))
+def test_sparse_branch_on_both_kernel_families(case, exact, path):
+    """The masked softmax branch on the tensor cores (a first sweep over the keys for the denominators, the masked
+    probabilities added to the weights in the second) and on the CUDA cores, on top of either base kernel.  The
+    threshold sits in a gap of the oracle's probabilities; with bf16 cosines a probability next to it may still fall
+    on the other side, which moves an output by at most the threshold times |v|."""
+    from paper_2211_10526_b200 import CastlingAttn
+    c = workloads.custom_call(*case, "bf16", seed=8400 + case[2])
+    s = c.shape
+    thr = gap_threshold(c, lo=0.0, hi=0.2, require=False)   # most probabilities pass
+    ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize,
+                                kernel=oracle.KERNEL_EXACT if exact else oracle.KERNEL_LINEAR, sparse_eps=thr, threads=16)
+    base = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize,
+                                 kernel=oracle.KERNEL_EXACT if exact else oracle.KERNEL_LINEAR, threads=16)
+    # With unit rows a probability is about 1/N, so the branch is a small term of long sequences (the bound on the whole
+    # output could hide it there); on the planes of a few tokens it is several times the bound, and a defect in the
+    # denominators or the mask fails the comparison below.
+    if s.N <= 32:
+        assert np.max(np.abs(ref - base)) > 2.5 * TOL["bf16"] * np.max(np.abs(ref)), "the branch is too small to be seen"
+    dev = torch.device("cuda:0")
+    q, k, v = (t.to(dev) for t in (c.q, c.k, c.v))
+    out = torch.full_like(q, float("nan"))
+    with CastlingAttn(ksize=s.ksize, exact_kernel=exact, sparse_eps=thr, force_path=path) as attn:
+        attn.forward(q, k, v, c.dw_weight.to(dev), c.dw_bias.to(dev), s.gridH, s.gridW, out=out)
+        torch.cuda.synchronize()
+        assert attn.device_status() == (0, 0)
+        assert attn.last_path() == (path, 1)
+    got = out.double().cpu().numpy()
+    assert np.all(np.isfinite(got))
+    check(got, ref, "bf16", f"{s.label()} exact={exact} path {path}")
+
+
 @pytest.mark.parametrize("name,idx", QUAD_CALLS, ids=QUAD_IDS)
 def test_sparse_branch_configurations(name, idx):
     (c,) = list(workloads.iter_workload(name, only=[idx]))
