@@ -46,7 +46,6 @@ struct QuadParams {
     int hdiv, H, head0, BH, N, gridH, gridW, q_tiles, k_tiles, n_items;
     float eps2;
     unsigned* status;
-    int exact;              // base weight: 1 - arccos(x)/pi, else 1/2 + x/pi
     float sparse_eps;       // threshold of the mask (sparse sweeps only)
 };
 
@@ -62,7 +61,7 @@ __device__ __forceinline__ float angular_weight(float x) {
     return x >= 0.f ? 1.0f - r : r;                           // arccos(-a) = pi - arccos(a)
 }
 
-template <int KS, bool SPARSE>
+template <int KS, bool SPARSE, bool EXACT>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const QuadParams prm) {
@@ -236,7 +235,6 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         long long g = 0, gp = 0;
         bool ok = true;
-        const bool exact = prm.exact != 0;
         for (int i = 0; i < my_items && ok; ++i) {
             const int item = blockIdx.x + i * gridDim.x, bh = item / prm.q_tiles, qt = item - bh * prm.q_tiles;
             float inv_den = 0.f;
@@ -253,9 +251,14 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         float x[16];
                         tmem_ld16(lane_base + cb * 128 + half * 64 + cc * 16, x);
                         tmem_ld_wait();
+                        if (jt < KT - 1) {   // only the last tile can reach beyond the plane
 #pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            if (key0 + cc * 16 + e < prm.N) den += __expf(fminf(fmaxf(x[e], -1.0f), 1.0f));
+                            for (int e = 0; e < 16; ++e) den += __expf(fminf(fmaxf(x[e], -1.0f), 1.0f));
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e)
+                                if (key0 + cc * 16 + e < prm.N) den += __expf(fminf(fmaxf(x[e], -1.0f), 1.0f));
+                        }
                     }
                     tcgen05_fence_before_sync();
                     mbar_arrive(&c_free[cb]);
@@ -268,8 +271,9 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
             // weight of a pair from its cosine
             auto weight = [&](float xr) -> float {
-                const float x = fminf(fmaxf(xr, -1.0f), 1.0f);
-                float wv = exact ? angular_weight(x) : fmaf(x, kInvPi, 0.5f);
+                // rounding can leave a cosine just outside [-1, 1]; the exact kernel's function clamps |x| itself
+                const float x = (EXACT && !SPARSE) ? xr : fminf(fmaxf(xr, -1.0f), 1.0f);
+                float wv = EXACT ? angular_weight(x) : fmaf(x, kInvPi, 0.5f);
                 if (SPARSE) {
                     const float pr = __expf(x) * inv_den;
                     if (pr > prm.sparse_eps) wv += pr;
@@ -368,7 +372,7 @@ tc_quad_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int KS, bool SPARSE>
+template <int KS, bool SPARSE, bool EXACT>
 cudaError_t launch_quad_ks(const Problem& p, unsigned* status, cudaStream_t st) {
     CUtensorMap tmQ, tmK, tmV;
     const uint64_t nb = (uint64_t)(p.BH / p.hdiv);
@@ -393,15 +397,15 @@ cudaError_t launch_quad_ks(const Problem& p, unsigned* status, cudaStream_t st) 
     prm.q_tiles = (p.N + kTile - 1) / kTile; prm.k_tiles = prm.q_tiles;
     prm.n_items = p.BH * prm.q_tiles;
     prm.eps2 = p.eps2; prm.status = status;
-    prm.exact = p.exact_kernel ? 1 : 0; prm.sparse_eps = p.sparse_eps;
+    prm.sparse_eps = p.sparse_eps;
     static PerDevice opt_in;
     {
-        const cudaError_t e = opt_in_smem(tc_quad_kernel<KS, SPARSE>, kSmem, opt_in);
+        const cudaError_t e = opt_in_smem(tc_quad_kernel<KS, SPARSE, EXACT>, kSmem, opt_in);
         if (e != cudaSuccess) return e;
     }
     const int sms = device_sm_count();
     const int grid = prm.n_items < sms ? prm.n_items : sms;
-    tc_quad_kernel<KS, SPARSE><<<(unsigned)grid, kThreads, kSmem, st>>>(tmQ, tmK, tmV, prm);
+    tc_quad_kernel<KS, SPARSE, EXACT><<<(unsigned)grid, kThreads, kSmem, st>>>(tmQ, tmK, tmV, prm);
     return cudaGetLastError();
 }
 
@@ -415,8 +419,11 @@ bool quad_supports(const Problem& p) {
 }
 
 cudaError_t launch_quad(const Problem& p, unsigned* status, cudaStream_t st) {
-    if (p.sparse) return p.ksize == 3 ? launch_quad_ks<3, true>(p, status, st) : launch_quad_ks<5, true>(p, status, st);
-    return p.ksize == 3 ? launch_quad_ks<3, false>(p, status, st) : launch_quad_ks<5, false>(p, status, st);
+    if (p.sparse && p.exact_kernel)
+        return p.ksize == 3 ? launch_quad_ks<3, true, true>(p, status, st) : launch_quad_ks<5, true, true>(p, status, st);
+    if (p.sparse)
+        return p.ksize == 3 ? launch_quad_ks<3, true, false>(p, status, st) : launch_quad_ks<5, true, false>(p, status, st);
+    return p.ksize == 3 ? launch_quad_ks<3, false, true>(p, status, st) : launch_quad_ks<5, false, true>(p, status, st);
 }
 
 }  // namespace tc
