@@ -297,3 +297,8 @@ def test_exact_kernel_at_the_token_limit():
     s = c.shape
     ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, kernel=oracle.KERNEL_EXACT, threads=2)
     check(gpu_forward(c, exact_kernel=True), ref, "bf16", "16384 tokens")
+    # the same limit on the tensor-core kernel (width-64 heads): 128 query tiles x 128 key tiles for one plane
+    c = workloads.custom_call(1, 1, 128, 128, 64, 3, "bf16", seed=8106)
+    s = c.shape
+    ref = oracle.forward_matrix(c.q, c.k, c.v, c.dw_weight, c.dw_bias, s.gridH, s.gridW, s.ksize, kernel=oracle.KERNEL_EXACT, threads=2)
+    check(gpu_forward(c, exact_kernel=True, force_path=2), ref, "bf16", "16384 tokens, tensor cores")
